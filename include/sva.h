@@ -1,0 +1,145 @@
+/*
+ * sva.h -- C ABI of the block-sparse spatiotemporal attention library (sm_100a).
+ *
+ * The path follows the sparse-attention description of the paper (Sec. "Sparse
+ * Attention": critical key blocks are chosen per query block and "computed
+ * exactly"; LTX-2.3 pipeline paragraph: "score-based routing", block-wise
+ * sparsity, "FlashAttention dense fallback"):
+ *
+ *   route   : mean-pool Q and K per block, block scores, per-row top-k or
+ *             cumulative-mass cut  ->  CSR list of kept key blocks per query block
+ *   attend  : softmax attention of every query over the keys of its kept blocks only
+ *   dense   : the same with every block kept
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller.  The structs
+ *     and the returned strings live on the host.
+ *   - Q, K, V, O are [B, H, N, d] with d contiguous; strides for b, h, n are given in
+ *     ELEMENTS.  N counts the valid tokens: tokens >= N do not exist (they are never
+ *     read as keys and never written as queries), so buffers need not be padded.
+ *   - Row index of the block structure: r = (b*H + h)*Nb + I with Nb = ceil(N/block),
+ *     R = B*H*Nb.  CSR entries are key-block indices J in [0, Nb), ascending and
+ *     unique inside a row.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*), never
+ *     synchronise the device and may be issued back to back on one stream.
+ *   - The library allocates no device memory; scratch is the caller's `workspace`.
+ *   - Every call validates its arguments on the host first and returns a non-zero
+ *     sva_status_t WITHOUT launching anything when they are bad.  No exception
+ *     crosses the ABI.  Non-finite inputs give undefined (but memory-safe) results.
+ *   - `device_status` (optional, device int32, zero it before the call): kernels OR
+ *     SVA_DEV_* bits into it instead of trapping (a bad CSR entry is skipped, a
+ *     pipeline wait that ran out gives up and the block exits).
+ */
+#ifndef SVA_H_
+#define SVA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SVA_OK = 0,
+  SVA_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, bad enum            */
+  SVA_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels are built for          */
+  SVA_ERR_WORKSPACE = 3,     /* workspace missing or too small                        */
+  SVA_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (launch, map encode) */
+  SVA_ERR_ALIGNMENT = 5      /* pointer or stride not aligned as required             */
+} sva_status_t;
+
+/* bits a kernel may set in *device_status */
+#define SVA_DEV_BAD_INDEX 1  /* CSR entry outside [0,Nb) or row_ptr not monotone: skipped */
+#define SVA_DEV_TIMEOUT   2  /* a bounded pipeline wait expired; output of that block is undefined */
+
+typedef enum { SVA_BF16 = 0, SVA_FP8_E4M3 = 1 } sva_qk_dtype_t;
+
+typedef struct {
+  int32_t B, H, N, d;        /* d in {64, 128}                                        */
+  int32_t block;             /* tokens per block, 64 or 128; same for queries and keys */
+  int64_t q_stride[3];       /* element strides of b, h, n (d has stride 1)           */
+  int64_t k_stride[3];
+  int64_t v_stride[3];
+  int64_t o_stride[3];
+  float softmax_scale;       /* <= 0 selects 1/sqrt(d)                                */
+  int32_t qk_dtype;          /* SVA_BF16: Q,K bf16.  SVA_FP8_E4M3: Q,K are e4m3 bytes
+                                with one fp32 scale per (b,h,block), [B,H,Nb]          */
+} sva_problem_t;
+
+typedef struct {
+  int32_t mode;              /* 0 = top-k, 1 = cumulative softmax mass >= mass, capped at k */
+  int32_t k;                 /* 1 <= k; values above Nb mean Nb                       */
+  float mass;                /* tau in (0,1]; mode 1 only                             */
+  int32_t win_t, win_s;      /* forced neighbour half-widths on the (frame, strip) block
+                                grid; negative = no forced window                     */
+  int32_t blocks_per_frame;  /* strips per frame; Nb must be a multiple when a window is set */
+} sva_select_t;
+
+/* Capacity (in entries) that col_idx must have for sva_block_select: R * per-row cap,
+ * where the per-row cap is max(min(k,Nb), window size). */
+int64_t sva_select_max_nnz(const sva_problem_t* p, const sva_select_t* s);
+
+/* Bytes of scratch sva_block_select needs (pooled means, per-row staging). 0 on bad input. */
+size_t sva_select_workspace_bytes(const sva_problem_t* p, const sva_select_t* s);
+
+/*
+ * Routing (the paper's "score-based routing" of critical blocks).
+ *   q, k          : Q and K as described by p (bf16, or e4m3 bytes + q_scale/k_scale)
+ *   row_ptr       : out, [R+1] int32, row_ptr[R] = number of kept (row, block) pairs
+ *   col_idx       : out, capacity sva_select_max_nnz entries; rows are packed back to back
+ *   block_scores  : optional out, [B,H,Nb,Nb] fp32, the scaled pooled scores
+ *   workspace     : >= sva_select_workspace_bytes, 256-byte aligned
+ * Pooling is a mean over the VALID tokens of a block; score = softmax_scale*<qbar,kbar>;
+ * order = forced window first, then score descending, ties to the LOWER block index;
+ * mode 0 keeps min(k,Nb) blocks, mode 1 the shortest prefix whose softmax mass (over all
+ * Nb blocks of the row) reaches `mass`, at least one block, at most k; the forced window is
+ * always kept.  Arithmetic is fp32 with a fixed summation order (deterministic).
+ */
+int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* q, const void* k,
+                     const float* q_scale, const float* k_scale, int32_t* row_ptr,
+                     int32_t* col_idx, float* block_scores, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/*
+ * Exact attention over the kept blocks ("critical blocks are computed exactly"):
+ *   o_i = sum_j softmax_j(scale*<q_i,k_j>) v_j,  j over the valid keys of the kept blocks
+ *   lse_i = log sum_j exp(scale*<q_i,k_j>)       (optional, [B,H,N] fp32 contiguous)
+ * O is bf16.  A row with an empty list writes zeros and lse = -inf.
+ * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
+ * (16 for e4m3 Q/K).  Tensor-core kernel: bf16 (or e4m3 x e4m3) MMA, fp32 accumulate.
+ */
+int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                              const float* q_scale, const float* k_scale, const int32_t* row_ptr,
+                              const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
+                              void* stream);
+
+/* The dense fallback: every block kept, no CSR read. */
+int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                       const float* q_scale, const float* k_scale, void* o, float* lse,
+                       int32_t* device_status, void* stream);
+
+/*
+ * Diagnostic twin of sva_block_sparse_attn_fwd: the same contract computed by a plain fp32
+ * CUDA-core kernel (no tensor cores, no TMA).  row_ptr == NULL means dense.  Slow; it exists
+ * so that the tensor-core kernel can be cross-checked on the device.
+ */
+int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const void* k,
+                                   const void* v, const float* q_scale, const float* k_scale,
+                                   const int32_t* row_ptr, const int32_t* col_idx, void* o,
+                                   float* lse, int32_t* device_status, void* stream);
+
+/*
+ * FP8 variant's quantiser: per (b,h,block) absmax a over the valid tokens, scale s = a/448
+ * (s = 1 when a = 0), y = x/s in fp32, round-to-nearest-even saturating cast to OCP e4m3.
+ * q8/k8 use the strides of p (in elements = bytes); scales are [B,H,Nb] fp32.
+ */
+int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q8,
+                        void* k8, float* q_scale, float* k_scale, void* stream);
+
+const char* sva_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SVA_H_ */

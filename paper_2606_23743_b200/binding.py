@@ -1,0 +1,150 @@
+"""Thin ctypes binding over the C ABI declared in include/sva.h.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.  torch is used
+for device memory and streams.  There is no CPU fallback: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsva.so")
+_lib = None
+
+SVA_OK = 0
+SVA_BF16, SVA_FP8_E4M3 = 0, 1
+SVA_DEV_BAD_INDEX, SVA_DEV_TIMEOUT = 1, 2
+
+EXPORTS = [
+    "sva_select_max_nnz", "sva_select_workspace_bytes", "sva_block_select",
+    "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
+    "sva_quantize_qk_fp8", "sva_status_string",
+]
+
+
+class Problem(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("N", C.c_int32), ("d", C.c_int32),
+                ("block", C.c_int32),
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+                ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
+                ("softmax_scale", C.c_float), ("qk_dtype", C.c_int32)]
+
+
+class Select(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("k", C.c_int32), ("mass", C.c_float),
+                ("win_t", C.c_int32), ("win_s", C.c_int32), ("blocks_per_frame", C.c_int32)]
+
+
+class SvaError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+def lib():
+    """Loads libsva.so (built in-tree by paper_2606_23743_b200.build). Raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2606_23743_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(_LIB_PATH)
+        vp = C.c_void_p
+        L.sva_select_max_nnz.restype = C.c_int64
+        L.sva_select_max_nnz.argtypes = [C.POINTER(Problem), C.POINTER(Select)]
+        L.sva_select_workspace_bytes.restype = C.c_size_t
+        L.sva_select_workspace_bytes.argtypes = [C.POINTER(Problem), C.POINTER(Select)]
+        L.sva_block_select.restype = C.c_int
+        L.sva_block_select.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp,
+                                       vp, vp, C.c_size_t, vp]
+        for name in ("sva_block_sparse_attn_fwd", "sva_block_sparse_attn_fwd_simt"):
+            f = getattr(L, name)
+            f.restype = C.c_int
+            f.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sva_dense_attn_fwd.restype = C.c_int
+        L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sva_quantize_qk_fp8.restype = C.c_int
+        L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
+        L.sva_status_string.restype = C.c_char_p
+        L.sva_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().sva_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _strides(t):
+    assert t.dim() == 4 and t.stride(3) == 1, "tensors are [B,H,N,d] with d contiguous"
+    return (C.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+def make_problem(q, k, v, o, N: int, block: int, scale: float = 0.0, fp8: bool = False) -> Problem:
+    """q,k,v,o: [B,H,n_alloc,d] device tensors (d contiguous); N = valid tokens <= n_alloc."""
+    B, H, _, d = q.shape
+    p = Problem()
+    p.B, p.H, p.N, p.d, p.block = B, H, N, d, block
+    p.q_stride, p.k_stride = _strides(q), _strides(k)
+    p.v_stride = _strides(v) if v is not None else _strides(q)
+    p.o_stride = _strides(o) if o is not None else _strides(q)
+    p.softmax_scale = scale
+    p.qk_dtype = SVA_FP8_E4M3 if fp8 else SVA_BF16
+    return p
+
+
+def make_select(mode: int, k: int, mass: float = 1.0, win_t: int = -1, win_s: int = -1,
+                blocks_per_frame: int = 0) -> Select:
+    return Select(mode, k, mass, win_t, win_s, blocks_per_frame)
+
+
+def select_max_nnz(p: Problem, s: Select) -> int:
+    return int(lib().sva_select_max_nnz(C.byref(p), C.byref(s)))
+
+
+def select_workspace_bytes(p: Problem, s: Select) -> int:
+    return int(lib().sva_select_workspace_bytes(C.byref(p), C.byref(s)))
+
+
+def block_select(p: Problem, s: Select, q, k, row_ptr, col_idx, workspace, q_scale=None, k_scale=None,
+                 block_scores=None) -> None:
+    rc = lib().sva_block_select(C.byref(p), C.byref(s), _ptr(q), _ptr(k), _ptr(q_scale), _ptr(k_scale),
+                                _ptr(row_ptr), _ptr(col_idx), _ptr(block_scores), _ptr(workspace),
+                                workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_select")
+
+
+def block_sparse_attn_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, q_scale=None,
+                          k_scale=None, simt: bool = False) -> None:
+    fn = lib().sva_block_sparse_attn_fwd_simt if simt else lib().sva_block_sparse_attn_fwd
+    rc = fn(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale), _ptr(k_scale), _ptr(row_ptr),
+            _ptr(col_idx), _ptr(o), _ptr(lse), _ptr(status), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_sparse_attn_fwd")
+
+
+def dense_attn_fwd(p: Problem, q, k, v, o, lse=None, status=None, q_scale=None, k_scale=None) -> None:
+    rc = lib().sva_dense_attn_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale), _ptr(k_scale),
+                                  _ptr(o), _ptr(lse), _ptr(status), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_dense_attn_fwd")
+
+
+def quantize_qk_fp8(p: Problem, q, k, q8, k8, q_scale, k_scale) -> None:
+    rc = lib().sva_quantize_qk_fp8(C.byref(p), _ptr(q), _ptr(k), _ptr(q8), _ptr(k8), _ptr(q_scale),
+                                   _ptr(k_scale), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_quantize_qk_fp8")

@@ -1,0 +1,164 @@
+// C ABI entry points: host-side validation, then the kernel launchers.
+#include "common.cuh"
+
+namespace sva {
+
+void set_tiles_per_cta(int n);
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_problem(const sva_problem_t* p) {
+  if (!p) return SVA_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->H <= 0 || p->N <= 0) return SVA_ERR_INVALID_ARG;
+  if (p->qk_dtype != SVA_BF16 && p->qk_dtype != SVA_FP8_E4M3) return SVA_ERR_INVALID_ARG;
+  if (p->d != 64 && p->d != 128) return SVA_ERR_UNSUPPORTED;
+  if (p->block != 64 && p->block != 128) return SVA_ERR_UNSUPPORTED;
+  if ((long long)p->B * p->H * ((p->N + p->block - 1) / p->block) > 0x7fffffffLL / 64) return SVA_ERR_UNSUPPORTED;
+  return SVA_OK;
+}
+
+static int check_strides(const int64_t s[3], int mult) {
+  for (int i = 0; i < 3; ++i) {
+    if (s[i] < 0) return SVA_ERR_INVALID_ARG;
+    if (s[i] % mult != 0) return SVA_ERR_ALIGNMENT;
+  }
+  return SVA_OK;
+}
+
+static int validate_select(const Dims& m, const sva_select_t* s) {
+  if (!s) return SVA_ERR_INVALID_ARG;
+  if (s->mode != 0 && s->mode != 1) return SVA_ERR_INVALID_ARG;
+  if (s->k < 1) return SVA_ERR_INVALID_ARG;
+  if (s->mode == 1 && !(s->mass > 0.f && s->mass <= 1.f)) return SVA_ERR_INVALID_ARG;
+  if (s->win_t >= 0 && s->win_s >= 0) {
+    if (s->blocks_per_frame <= 0 || m.Nb % s->blocks_per_frame != 0) return SVA_ERR_INVALID_ARG;
+  }
+  return SVA_OK;
+}
+
+static int validate_attn(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                         const float* qs, const float* ks, const void* o) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q || !k || !v || !o) return SVA_ERR_INVALID_ARG;
+  const bool f8 = p->qk_dtype == SVA_FP8_E4M3;
+  if (f8 && (!qs || !ks)) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, f8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->k_stride, f8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->v_stride, 8))) return rc;
+  if ((rc = check_strides(p->o_stride, 8))) return rc;
+  if (p->q_stride[2] < p->d || p->k_stride[2] < p->d || p->v_stride[2] < p->d || p->o_stride[2] < p->d)
+    return SVA_ERR_INVALID_ARG;
+  return SVA_OK;
+}
+
+// The tensor-core kernel covers 128-token blocks with d = 128; other supported shapes run on
+// the CUDA-core kernel.
+static bool use_sm100(const Dims& m) { return m.block == 128 && m.d == 128; }
+
+}  // namespace sva
+
+using namespace sva;
+
+extern "C" {
+
+int64_t sva_select_max_nnz(const sva_problem_t* p, const sva_select_t* s) {
+  if (validate_problem(p) || !s || s->k < 1) return 0;
+  Dims m = make_dims(p);
+  return (int64_t)m.R * select_row_cap(m, s);
+}
+
+size_t sva_select_workspace_bytes(const sva_problem_t* p, const sva_select_t* s) {
+  if (validate_problem(p) || !s || s->k < 1) return 0;
+  Dims m = make_dims(p);
+  return select_workspace_bytes(m, s);
+}
+
+int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* q, const void* k,
+                     const float* q_scale, const float* k_scale, int32_t* row_ptr,
+                     int32_t* col_idx, float* block_scores, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  Dims m = make_dims(p);
+  if ((rc = validate_select(m, s))) return rc;
+  if (!q || !k || !row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
+  if (m.fp8 && (!q_scale || !k_scale)) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, m.fp8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->k_stride, m.fp8 ? 16 : 8))) return rc;
+  if (!workspace) return SVA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SVA_ERR_ALIGNMENT;
+  return launch_select(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, workspace,
+                       workspace_bytes, (cudaStream_t)stream);
+}
+
+int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                              const float* q_scale, const float* k_scale, const int32_t* row_ptr,
+                              const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
+                              void* stream) {
+  int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
+  if (rc) return rc;
+  if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  if (use_sm100(m))
+    return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
+                             (cudaStream_t)stream);
+  return launch_attn_simt(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
+                          (cudaStream_t)stream);
+}
+
+int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                       const float* q_scale, const float* k_scale, void* o, float* lse,
+                       int32_t* device_status, void* stream) {
+  int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
+  if (rc) return rc;
+  Dims m = make_dims(p);
+  if (use_sm100(m))
+    return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status,
+                             (cudaStream_t)stream);
+  return launch_attn_simt(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status,
+                          (cudaStream_t)stream);
+}
+
+int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const void* k,
+                                   const void* v, const float* q_scale, const float* k_scale,
+                                   const int32_t* row_ptr, const int32_t* col_idx, void* o,
+                                   float* lse, int32_t* device_status, void* stream) {
+  int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
+  if (rc) return rc;
+  if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  return launch_attn_simt(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
+                          (cudaStream_t)stream);
+}
+
+int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q8,
+                        void* k8, float* q_scale, float* k_scale, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q_bf16 || !k_bf16 || !q8 || !k8 || !q_scale || !k_scale) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q_bf16) || !aligned16(k_bf16) || !aligned16(q8) || !aligned16(k8)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, 16))) return rc;
+  if ((rc = check_strides(p->k_stride, 16))) return rc;
+  Dims m = make_dims(p);
+  return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, (cudaStream_t)stream);
+}
+
+const char* sva_status_string(int status) {
+  switch (status) {
+    case SVA_OK: return "ok";
+    case SVA_ERR_INVALID_ARG: return "invalid argument";
+    case SVA_ERR_UNSUPPORTED: return "unsupported shape";
+    case SVA_ERR_WORKSPACE: return "workspace missing or too small";
+    case SVA_ERR_CUDA: return "CUDA call failed";
+    case SVA_ERR_ALIGNMENT: return "pointer or stride misaligned";
+    default: return "unknown status";
+  }
+}
+
+/* bring-up switch (not part of the public header): 1 or 2 query tiles per CTA */
+void sva_debug_set_tiles_per_cta(int n) { set_tiles_per_cta(n); }
+
+}  // extern "C"

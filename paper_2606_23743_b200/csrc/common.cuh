@@ -1,0 +1,60 @@
+// Shared host/device helpers of the sva library (CUDA side only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sva.h"
+
+namespace sva {
+
+struct Dims {
+  int B, H, N, d, block, Nb, R;
+  float scale;
+  bool fp8;
+};
+
+inline Dims make_dims(const sva_problem_t* p) {
+  Dims m;
+  m.B = p->B; m.H = p->H; m.N = p->N; m.d = p->d; m.block = p->block;
+  m.Nb = (p->N + p->block - 1) / p->block;
+  m.R = p->B * p->H * m.Nb;
+  m.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->d);
+  m.fp8 = p->qk_dtype == SVA_FP8_E4M3;
+  return m;
+}
+
+struct Strides { long long b, h, n; };
+inline Strides make_strides(const int64_t s[3]) { return Strides{(long long)s[0], (long long)s[1], (long long)s[2]}; }
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// e4m3 byte -> float (exact)
+__device__ __forceinline__ float e4m3_to_float(uint32_t byte) {
+  __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)byte, __NV_E4M3);
+  return __half2float(__half(h));
+}
+
+// host-side argument checks shared by the entry points
+int validate_problem(const sva_problem_t* p);
+
+// launchers (each returns an sva_status_t)
+int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, const void* q,
+                  const void* k, const float* q_scale, const float* k_scale, int32_t* row_ptr,
+                  int32_t* col_idx, float* block_scores, void* ws, size_t ws_bytes,
+                  cudaStream_t st);
+size_t select_workspace_bytes(const Dims& m, const sva_select_t* s);
+int select_row_cap(const Dims& m, const sva_select_t* s);
+int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
+                    void* k8, float* qs, float* ks, cudaStream_t st);
+int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
+                     const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
+                     const int32_t* col_idx, void* o, float* lse, int32_t* status, cudaStream_t st);
+int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
+                      const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
+                      const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                      cudaStream_t st);
+
+}  // namespace sva
