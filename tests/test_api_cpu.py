@@ -1,0 +1,103 @@
+"""The C-ABI library loads without a GPU, exports what include/sva.h declares, and rejects bad
+arguments on the host before any launch."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2606_23743_b200 import binding as B
+from paper_2606_23743_b200 import build as build_mod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_mod.build()
+    return B.lib()
+
+
+def test_header_symbols_exported(lib):
+    text = open(os.path.join(ROOT, "include", "sva.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = set(re.findall(r"\b(sva_[a-z0-9_]+)\s*\(", text))
+    assert names >= set(B.EXPORTS) and len(names) >= 8
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def _problem(**kw):
+    p = B.Problem()
+    p.B, p.H, p.N, p.d, p.block = 1, 2, 1024, 128, 128
+    for f in ("q_stride", "k_stride", "v_stride", "o_stride"):
+        setattr(p, f, (C.c_int64 * 3)(2 * 1024 * 128, 1024 * 128, 128))
+    p.softmax_scale = 0.0
+    p.qk_dtype = 0
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "ok"
+    assert "workspace" in B.status_string(3)
+    assert "unknown" in B.status_string(99)
+
+
+def test_workspace_and_capacity(lib):
+    p = _problem()
+    s = B.make_select(0, 4)
+    Nb, R = 8, 16
+    assert B.select_max_nnz(p, s) == R * 4
+    pooled = 2 * (2 * Nb * 128 * 4)
+    assert B.select_workspace_bytes(p, s) == pooled                      # fixed-count rows: no staging
+    sm = B.make_select(1, 4, 0.9)
+    assert B.select_workspace_bytes(p, sm) >= pooled + R * 4 * 4 + R * 4  # staged rows + counts
+    sw = B.make_select(0, 4, 1.0, 1, 1, 4)                                # 3x3 window > k
+    assert B.select_max_nnz(p, sw) == R * 8                               # window clipped to Nb = 8
+    assert B.select_max_nnz(p, B.make_select(0, 100)) == R * Nb          # k above Nb means Nb
+    assert B.select_workspace_bytes(_problem(d=100), s) == 0
+
+
+def test_rejects_bad_arguments_before_launch(lib):
+    p = _problem()
+    s = B.make_select(0, 4)
+    one = C.c_void_p(256)      # non-null, aligned, never dereferenced: validation fails first
+    vp = C.c_void_p
+    def sel(p, s, q=one, k=one, rp=one, ci=one, ws=one, wsb=1 << 30):
+        return lib.sva_block_select(C.byref(p), C.byref(s), q, k, None, None, rp, ci, None, ws, wsb, None)
+    assert sel(_problem(d=100), s) == 2
+    assert sel(_problem(block=32), s) == 2
+    assert sel(_problem(N=0), s) == 1
+    assert sel(p, B.make_select(0, 0)) == 1
+    assert sel(p, B.make_select(2, 4)) == 1
+    assert sel(p, B.make_select(1, 4, 0.0)) == 1
+    assert sel(p, B.make_select(0, 4, 1.0, 1, 1, 3)) == 1            # Nb not a multiple of strips/frame
+    assert sel(p, s, q=None) == 1
+    assert sel(p, s, ws=None) == 3
+    assert sel(p, s, wsb=16) == 3
+    assert sel(p, s, q=vp(8)) == 5
+    assert sel(p, s, ws=vp(128)) == 5
+    assert sel(_problem(qk_dtype=1), s) == 1                          # fp8 without scales
+    bad = _problem(); bad.q_stride = (C.c_int64 * 3)(0, 0, 132)
+    assert sel(bad, s) == 5
+
+    def att(p, q=one, k=one, v=one, o=one, rp=one, ci=one):
+        return lib.sva_block_sparse_attn_fwd(C.byref(p), q, k, v, None, None, rp, ci, o, None, None, None)
+    assert att(_problem(d=96)) == 2
+    assert att(p, v=None) == 1
+    assert att(p, rp=None) == 1
+    assert att(p, o=vp(4)) == 5
+    assert att(_problem(qk_dtype=7)) == 1
+    assert lib.sva_dense_attn_fwd(C.byref(p), one, one, None, None, None, one, None, None, None) == 1
+    assert lib.sva_quantize_qk_fp8(C.byref(p), one, one, one, None, one, one, None) == 1
+    bad = _problem(); bad.k_stride = (C.c_int64 * 3)(0, 0, 136)
+    assert lib.sva_quantize_qk_fp8(C.byref(bad), one, one, one, one, one, one, None) == 5
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "_LIB_PATH", "/nonexistent/libsva.so")
+    with pytest.raises(RuntimeError, match="no fallback"):
+        B.lib()

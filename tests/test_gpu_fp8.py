@@ -1,0 +1,56 @@
+"""FP8 (e4m3 Q/K with per-block scales) variant: quantiser bytes against the oracle's, attention
+against the fp64 oracle run on the dequantised Q/K (rel-L2 <= 5e-2)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import _util as U
+from paper_2606_23743_b200 import binding as B
+from paper_2606_23743_b200.workloads import WORKLOADS, shrink
+
+pytestmark = pytest.mark.gpu
+
+
+def _quantize(w, qd, kd):
+    q8 = torch.zeros(qd.shape, dtype=torch.uint8, device="cuda")
+    k8 = torch.zeros(kd.shape, dtype=torch.uint8, device="cuda")
+    qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device="cuda")
+    ks = torch.zeros_like(qs)
+    p = B.make_problem(qd, kd, None, None, w.N, w.block)
+    B.quantize_qk_fp8(p, qd, kd, q8, k8, qs, ks)
+    torch.cuda.synchronize()
+    return q8, k8, qs, ks
+
+
+@pytest.mark.parametrize("name", ["even", "ragged"])
+def test_quantiser_bytes_and_scales(name):
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=2) if name == "ragged" else shrink(WORKLOADS["medium"], H=2, T=2)
+    (q, k, _), (qb, kb, _) = U.host_inputs(w)
+    q8, k8, qs, ks = _quantize(w, U.dev(q), U.dev(k))
+    for bits, g8, gs in ((qb, q8, qs), (kb, k8, ks)):
+        codes, scales = oracle.quantize_e4m3(bits, w.N, w.block)
+        np.testing.assert_array_equal(gs.cpu().numpy(), scales)
+        np.testing.assert_array_equal(g8.cpu().numpy()[:, :, :w.N], codes[:, :, :w.N])
+        assert (g8[:, :, w.N:] == 0).all()
+
+
+@pytest.mark.parametrize("impl", ["tensor", "simt"])
+def test_fp8_select_and_attention(impl):
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=4)          # N = 6240, ragged tail, mass rule
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8, k8, qs, ks = _quantize(w, qd, kd)
+    # the oracle consumes the GPU's codes and scales, dequantised in fp64
+    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    rp, ci, sc = U.gpu_select(w, q8, k8, want_scores=True, q_scale=qs, k_scale=ks, fp8=True)
+    sel, s_ref = U.oracle_select(w, qh, kh)
+    assert np.abs(sc.cpu().numpy() - s_ref).max() < 2e-5
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    assert n_diff <= n_near
+    o, lse, st = U.gpu_attn(w, q8, k8, vd, rp, ci, simt=(impl == "simt"), q_scale=qs, k_scale=ks, fp8=True)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, 10)
+    r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
+    print(f"fp8/{impl}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")

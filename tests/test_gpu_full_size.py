@@ -1,0 +1,61 @@
+"""Full-size configurations in the launch configuration the bench times: selection parity on
+every row, attention parity on sampled rows the oracle computes one by one."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import _util as U
+from paper_2606_23743_b200.workloads import WORKLOADS
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,nrows", [("medium", 16), ("large", 16), ("xl", 12)])
+def test_full_size_select_then_attend(name, nrows):
+    w = WORKLOADS[name]
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w, qd, kd)
+    sel, _ = U.oracle_select(w, qb, kb)
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    print(f"{name}: rows {w.R} nnz {ci.numel()} differing {n_diff} near-tie rows {n_near}")
+    assert n_diff <= n_near
+    o, lse, st = U.gpu_attn(w, qd, kd, vd, rp, ci)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, nrows, seed=w.cfg)
+    r = U.check_attn_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
+    print(f"{name}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
+    # properties that hold at any size: finite outputs inside V's range, rows never written past N
+    of = o[:, :, :w.N].float()
+    assert torch.isfinite(of).all()
+    vmax = vd[:, :, :w.N].float().abs().amax()
+    assert of.abs().amax() <= vmax * 1.01
+    if w.n_alloc > w.N:
+        assert (o[:, :, w.N:] == 7.0).all()
+    if name == "medium":
+        od, lsd, _ = U.gpu_attn(w, qd, kd, vd, None, None, dense=True)
+        U.check_attn_vs_oracle(w, qb, kb, vb, None, None, od, lsd, rows[:4], dense=True)
+
+
+def test_full_size_fp8():
+    from paper_2606_23743_b200 import binding as B
+    w = WORKLOADS["large_fp8"]
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8 = torch.zeros(qd.shape, dtype=torch.uint8, device="cuda"); k8 = torch.zeros_like(q8)
+    qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device="cuda"); ks = torch.zeros_like(qs)
+    p = B.make_problem(qd, kd, None, None, w.N, w.block)
+    B.quantize_qk_fp8(p, qd, kd, q8, k8, qs, ks)
+    torch.cuda.synchronize()
+    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
+    sel, _ = U.oracle_select(w, qh, kh)
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    assert n_diff <= n_near
+    o, lse, st = U.gpu_attn(w, q8, k8, vd, rp, ci, q_scale=qs, k_scale=ks, fp8=True)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, 12, seed=5)
+    r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
+    print(f"large_fp8: differing {n_diff} near {n_near} max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")
