@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the block-sparse video attention hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic Q/K/V: block routing
+(pool -> scores -> select -> CSR) followed by block-sparse attention over the kept blocks.
+`value` is effective TFLOP/s on the selected blocks (4*Bs^2*d FLOP per kept tile) with the
+inputs resident in HBM; `e2e` is the same metric with the step's Q/K/V copied from pinned host
+memory and O copied back inside the timed region.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large] [--impl reference]
+
+With N > 1 (torchrun) every rank is a replica working on its own batch sample: no data-path
+collective, weak scaling, time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2606_23743_b200 import dist as D  # noqa: E402
+from paper_2606_23743_b200.workloads import SEED_BASE, WORKLOADS, bf16_bits, make_qkv  # noqa: E402
+
+METRIC = "block-sparse attn fwd effective TFLOPS (selected blocks)"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the "large" workload,
+# from the ncu capture summarised in profiles/ (None until captured)
+ATTN_TRAFFIC_BYTES = {"large": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            props = torch.cuda.get_device_properties(device_index)
+            handle = None
+            uuid = getattr(props, "uuid", None)
+            if uuid is not None:
+                try:
+                    handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+                except Exception:
+                    handle = None
+            if handle is None:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self._nv, self._h = pynvml, handle
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report no samples rather than fail the bench
+            self._nv, self._h, self.error = None, None, repr(e)
+
+    def _names(self, mask):
+        nv = self._nv
+        table = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+                 "hw_power_brake": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80)}
+        return {k for k, bit in table.items() if mask & bit}
+
+    def _run(self):
+        nv, h = self._nv, self._h
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                self.reasons |= self._names(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def flops_per_tile(w):
+    return 4.0 * w.block * w.block * w.d
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+def oracle_sample(w, qb, kb, vb, n_rows):
+    """Times the oracle, as it stands, on the first n_rows query-block rows of batch 0 (whole
+    heads first): pooling, scores and selection of the heads touched, then attention of those
+    rows.  Returns (seconds, flops, rows)."""
+    import oracle
+    n_rows = max(1, min(n_rows, w.H * w.Nb))
+    heads = -(-n_rows // w.Nb)
+    q1, k1, v1 = qb[:1, :heads], kb[:1, :heads], vb[:1, :heads]
+    t0 = time.perf_counter()
+    sel, _ = oracle.select_from_qk(q1, k1, w.N, w.block, w.scale, w.mode, w.k, w.tau, w.win_t, w.win_s,
+                                   w.blocks_per_frame if w.win_t >= 0 else 0)
+    rows = list(range(n_rows))
+    oracle.attn_rows(q1, k1, v1, w.N, w.block, w.scale, sel.row_ptr, sel.col_idx, rows=rows)
+    dt = time.perf_counter() - t0
+    nnz = int(sel.row_ptr[n_rows] - sel.row_ptr[0])
+    return dt, nnz * flops_per_tile(w), n_rows
+
+
+def cpu_baseline(w, qb, kb, vb, target_s=15.0):
+    import oracle
+    dt, fl, n = oracle_sample(w, qb, kb, vb, 32)
+    per_row = max(dt / max(n, 1), 1e-6)
+    n_rows = int(min(w.H * w.Nb, max(32, target_s / per_row)))
+    dt, fl, n = oracle_sample(w, qb, kb, vb, n_rows)
+    return {"value": fl / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"'{w.name}', batch 0: routing of the first {-(-n // w.Nb)} head(s) and attention of "
+                      f"their first {n} query-block rows; {dt:.1f} s wall",
+            "seconds": dt}
+
+
+def run_reference(args):
+    rank, _, world = D.env_world()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = WORKLOADS[args.workload]
+    from paper_2606_23743_b200.workloads import shrink
+    w1 = shrink(w, B=1, H=min(w.H, 4))
+    q, k, v = make_qkv(w1, SEED_BASE + w.cfg)
+    qb, kb, vb = bf16_bits(q), bf16_bits(k), bf16_bits(v)
+    total = args.steps + args.warmup
+    dt, fl, n = oracle_sample(w1, qb, kb, vb, 16)
+    per_row = max(dt / n, 1e-6)
+    n_rows = int(min(w1.H * w1.Nb, max(4, (150.0 / max(total, 1)) / per_row)))
+    for _ in range(args.warmup):
+        oracle_sample(w1, qb, kb, vb, n_rows)
+    t0 = time.perf_counter()
+    flops = 0.0
+    for _ in range(args.steps):
+        _, fl, n = oracle_sample(w1, qb, kb, vb, n_rows)
+        flops += fl
+    dt = time.perf_counter() - t0
+    value = flops / dt / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "note": "fp64 CPU oracle on host cores; each step is a bounded sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"per step: routing of the first {-(-n // w.Nb)} head(s) + attention of their first {n} query-block rows"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=[k for k in WORKLOADS if not WORKLOADS[k].fp8])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    from paper_2606_23743_b200 import binding as B
+    from paper_2606_23743_b200 import build as build_mod
+    build_mod.build()
+    B.lib()                                       # fail loudly if the CUDA library is missing
+
+    rank, local_rank, world = D.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = WORKLOADS[args.workload]
+    warmup = max(args.warmup, 3)
+
+    qh, kh, vh = (x.pin_memory() for x in make_qkv(w, D.rank_seed(SEED_BASE + w.cfg, rank)))
+    q, k, v = (x.to(dev, non_blocking=True) for x in (qh, kh, vh))
+    o = torch.empty_like(v)
+    oh = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+    p = B.make_problem(q, k, v, o, w.N, w.block)
+    s = B.make_select(w.mode, w.k, w.tau, w.win_t, w.win_s, w.blocks_per_frame if w.win_t >= 0 else 0)
+    ws = torch.empty(max(B.select_workspace_bytes(p, s), 256), dtype=torch.uint8, device=dev)
+    row_ptr = torch.zeros(w.R + 1, dtype=torch.int32, device=dev)
+    col_idx = torch.zeros(B.select_max_nnz(p, s), dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
+    launches_per_step = (4 if variable_rows else 2) + 1
+
+    def step():
+        B.block_select(p, s, q, k, row_ptr, col_idx, ws)
+        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    nnz = int(row_ptr[-1].item())
+    assert int(status.item()) == 0, "device status set during warm-up"
+    step_flops = nnz * flops_per_tile(w)
+
+    # ---- device-resident timing
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sel_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    att_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    D.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0.record()
+    for i in range(args.steps):
+        sel_ev[i][0].record()
+        B.block_select(p, s, q, k, row_ptr, col_idx, ws)
+        sel_ev[i][1].record()
+        att_ev[i][0].record()
+        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status)
+        att_ev[i][1].record()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    D.barrier()
+    total_ms = D.max_over_ranks(ev0.elapsed_time(ev1))
+    ms_per_step = total_ms / args.steps
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in att_ev]))
+    sel_ms = float(np.mean([a.elapsed_time(b) for a, b in sel_ev]))
+    job_flops = D.sum_over_ranks(step_flops)
+    value = job_flops / (ms_per_step * 1e-3) / 1e12
+    assert int(status.item()) == 0, "device status set during the timed region"
+
+    # ---- end to end: pinned host -> device, path, device -> pinned host, every step
+    e2e = None
+    if not args.no_e2e:
+        h2d = sum(x.numel() * x.element_size() for x in (qh, kh, vh))
+        d2h = oh.numel() * oh.element_size()
+        e_steps = max(3, min(args.steps, 10))
+
+        def e2e_step():
+            q.copy_(qh, non_blocking=True); k.copy_(kh, non_blocking=True); v.copy_(vh, non_blocking=True)
+            step()
+            oh.copy_(o, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        D.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e_steps):
+            e2e_step()
+        e1.record()
+        torch.cuda.synchronize()
+        D.barrier()
+        e_ms = D.max_over_ranks(e0.elapsed_time(e1)) / e_steps
+        e2e = {"value": job_flops / (e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": e_steps}
+
+    peaks, peak_kind = load_peaks()
+    peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    achieved = step_flops / (attn_ms * 1e-3) / 1e12
+    sel_bytes = 4.0 * w.B * w.H * w.N * w.d
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
+                   "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
+                   "nnz_tiles": nnz, "parallelism": f"replicas x{world}",
+                   "l2": "inputs (%.0f MB) larger than L2; no flush" % (3 * sel_bytes / 2 / 1e6)},
+        "tokens_per_s": world * w.B * w.N / (ms_per_step * 1e-3),
+        "attention_ms": attn_ms, "select_ms": sel_ms,
+        "attention_tflops": achieved,
+        "select_gbs": sel_bytes / (sel_ms * 1e-3) / 1e9,
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
+                     "kernel": "attn_sm100_kernel", "peak_source": f"{peak_kind} bf16 burst",
+                     "frac_of_nominal_2250": achieved / 2250.0},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            line["cpu_baseline"] = cpu_baseline(w, bf16_bits(qh), bf16_bits(kh), bf16_bits(vh))
+        print(json.dumps(line))
+    D.finalize()
+
+
+if __name__ == "__main__":
+    main()
