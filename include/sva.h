@@ -46,7 +46,8 @@ typedef enum {
   SVA_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels are built for          */
   SVA_ERR_WORKSPACE = 3,     /* workspace missing or too small                        */
   SVA_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (launch, map encode) */
-  SVA_ERR_ALIGNMENT = 5      /* pointer or stride not aligned as required             */
+  SVA_ERR_ALIGNMENT = 5,     /* pointer or stride not aligned as required             */
+  SVA_ERR_SCRATCH_LIMIT = 6  /* sva_block_select_noalloc: problem needs more than the built-in scratch */
 } sva_status_t;
 
 /* bits a kernel may set in *device_status */
@@ -100,6 +101,35 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                      const float* q_scale, const float* k_scale, int32_t* row_ptr,
                      int32_t* col_idx, float* block_scores, void* workspace,
                      size_t workspace_bytes, void* stream);
+
+/*
+ * Routing for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a packaging variant of sva_block_select, same kernels, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin handed only its
+ * input and output buffers by a host runtime, a step that executes inside a region where the
+ * allocator must not be touched, a process whose memory pool is owned by someone else.  Such
+ * a caller has nowhere to get the `workspace` that sva_block_select asks for.
+ *
+ * Here the scratch lives inside the library: a file-scope device array of
+ * SVA_NOALLOC_SCRATCH_BYTES (8 MiB), present on every GPU that loads the library for as long
+ * as the process lives.  The call allocates and frees nothing.  Arguments and results are
+ * those of sva_block_select minus workspace/workspace_bytes.
+ *   - Limit: sva_select_workspace_bytes(p, s) must be <= SVA_NOALLOC_SCRATCH_BYTES, otherwise
+ *     SVA_ERR_SCRATCH_LIMIT is returned and nothing is launched (B*H*Nb*d*8 bytes of pooled
+ *     means dominate: e.g. 24 heads x 256 blocks x d=128 fits, 64 heads x 372 blocks does not).
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents; every value
+ *     a call reads from it is written by that same call first, so nothing needs clearing.
+ *     Two calls that may overlap on the GPU (different streams, no dependency) race on it:
+ *     serialise them.
+ */
+#define SVA_NOALLOC_SCRATCH_BYTES (8u << 20)
+int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, const void* q,
+                             const void* k, const float* q_scale, const float* k_scale,
+                             int32_t* row_ptr, int32_t* col_idx, float* block_scores,
+                             void* stream);
 
 /*
  * Exact attention over the kept blocks ("critical blocks are computed exactly"):

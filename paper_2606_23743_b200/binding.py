@@ -21,8 +21,9 @@ SVA_DEV_BAD_INDEX, SVA_DEV_TIMEOUT = 1, 2
 EXPORTS = [
     "sva_select_max_nnz", "sva_select_workspace_bytes", "sva_block_select",
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
-    "sva_quantize_qk_fp8", "sva_status_string",
+    "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc",
 ]
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 class Problem(C.Structure):
@@ -60,6 +61,9 @@ def lib():
         L.sva_block_select.restype = C.c_int
         L.sva_block_select.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp,
                                        vp, vp, C.c_size_t, vp]
+        L.sva_block_select_noalloc.restype = C.c_int
+        L.sva_block_select_noalloc.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp,
+                                               vp, vp]
         for name in ("sva_block_sparse_attn_fwd", "sva_block_sparse_attn_fwd_simt"):
             f = getattr(L, name)
             f.restype = C.c_int
@@ -125,6 +129,18 @@ def block_select(p: Problem, s: Select, q, k, row_ptr, col_idx, workspace, q_sca
                                 _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_select")
+
+
+def block_select_noalloc(p: Problem, s: Select, q, k, row_ptr, col_idx, q_scale=None, k_scale=None,
+                         block_scores=None) -> None:
+    """sva_block_select for callers that cannot allocate: the scratch is the library's built-in
+    device array (NOALLOC_SCRATCH_BYTES); raises SvaError(status 6) when the problem needs more.
+    Calls share that array, so calls that could overlap on the GPU must be serialised."""
+    rc = lib().sva_block_select_noalloc(C.byref(p), C.byref(s), _ptr(q), _ptr(k), _ptr(q_scale),
+                                        _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(block_scores),
+                                        _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_select_noalloc")
 
 
 def block_sparse_attn_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, q_scale=None,

@@ -94,6 +94,24 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                        workspace_bytes, (cudaStream_t)stream);
 }
 
+/* Same routing, scratch taken from the library's built-in device array: no allocation. */
+int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, const void* q,
+                             const void* k, const float* q_scale, const float* k_scale,
+                             int32_t* row_ptr, int32_t* col_idx, float* block_scores,
+                             void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  Dims m = make_dims(p);
+  if ((rc = validate_select(m, s))) return rc;
+  if (!q || !k || !row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
+  if (m.fp8 && (!q_scale || !k_scale)) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, m.fp8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->k_stride, m.fp8 ? 16 : 8))) return rc;
+  return launch_select_noalloc(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores,
+                               (cudaStream_t)stream);
+}
+
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                               const float* q_scale, const float* k_scale, const int32_t* row_ptr,
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
@@ -154,6 +172,7 @@ const char* sva_status_string(int status) {
     case SVA_ERR_WORKSPACE: return "workspace missing or too small";
     case SVA_ERR_CUDA: return "CUDA call failed";
     case SVA_ERR_ALIGNMENT: return "pointer or stride misaligned";
+    case SVA_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in no-allocation array holds";
     default: return "unknown status";
   }
 }

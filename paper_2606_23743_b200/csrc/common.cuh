@@ -46,6 +46,9 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
                   int32_t* col_idx, float* block_scores, void* ws, size_t ws_bytes,
                   cudaStream_t st);
 size_t select_workspace_bytes(const Dims& m, const sva_select_t* s);
+int launch_select_noalloc(const Dims& m, const sva_problem_t* p, const sva_select_t* s,
+                          const void* q, const void* k, const float* q_scale, const float* k_scale,
+                          int32_t* row_ptr, int32_t* col_idx, float* block_scores, cudaStream_t st);
 int select_row_cap(const Dims& m, const sva_select_t* s);
 int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
                     void* k8, float* qs, float* ks, cudaStream_t st);

@@ -8,6 +8,8 @@
 // block row with the head's pooled K staged through shared memory.  When the per-row count is
 // not a compile-time constant of the call (mass rule, or a window larger than k), rows are
 // staged and kernels 3/4 (scan, compact) build the CSR.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sva {
@@ -357,6 +359,41 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
   if (m.d == 64)
     return launch_select_d<64>(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, ws, st);
   return SVA_ERR_UNSUPPORTED;
+}
+
+// ---------------------------------------------------------------- no-allocation variant
+// Scratch for callers that cannot call cudaMalloc: it lives in the library image, so every
+// GPU that loads the library carries these bytes until the process exits.  In host code the
+// array's name is only a stand-in for the symbol -- not a device address -- so the address
+// is looked up once per device with cudaGetSymbolAddress and that pointer is what the kernels
+// receive.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SVA_NOALLOC_SCRATCH_BYTES];
+
+static constexpr int MAX_DEVICES = 64;
+static std::mutex g_noalloc_mutex;
+static void* g_noalloc_addr[MAX_DEVICES];   // device address of g_noalloc_scratch, per device
+
+int launch_select_noalloc(const Dims& m, const sva_problem_t* p, const sva_select_t* s,
+                          const void* q, const void* k, const float* q_scale, const float* k_scale,
+                          int32_t* row_ptr, int32_t* col_idx, float* block_scores, cudaStream_t st) {
+  if (select_workspace_bytes(m, s) > (size_t)SVA_NOALLOC_SCRATCH_BYTES) return SVA_ERR_SCRATCH_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SVA_ERR_CUDA;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_addr[dev]) {
+      // first call on this device (it is the current one): resolve the symbol
+      void* addr = nullptr;
+      if (cudaGetSymbolAddress(&addr, g_noalloc_scratch) != cudaSuccess || !addr) return SVA_ERR_CUDA;
+      g_noalloc_addr[dev] = addr;
+    }
+    scratch = g_noalloc_addr[dev];
+  }
+  // Nothing in the scratch has to start at zero: pooled means, staged rows and counts are all
+  // written by this call's kernels before they are read.
+  return launch_select(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, scratch,
+                       (size_t)SVA_NOALLOC_SCRATCH_BYTES, st);
 }
 
 }  // namespace sva
