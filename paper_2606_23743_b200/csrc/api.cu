@@ -4,6 +4,9 @@
 namespace sva {
 
 void set_tiles_per_cta(int n);
+void set_exp_emulation(int n);
+void set_prof_buffer(void* p);
+void set_debug_mode(int v);
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -179,5 +182,11 @@ const char* sva_status_string(int status) {
 
 /* bring-up switch (not part of the public header): 1 or 2 query tiles per CTA */
 void sva_debug_set_tiles_per_cta(int n) { set_tiles_per_cta(n); }
+/* tuning switch: 0..3 of every 4 exp2 pairs evaluated by a polynomial on the FMA pipe */
+void sva_debug_set_exp_emulation(int n) { set_exp_emulation(n); }
+/* tuning aid: device buffer of 5*8*8 int64 that CTA 64 fills with a clock64 timeline; NULL = off */
+void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); }
+/* tuning aid: bit0 skips the softmax arithmetic (results are wrong; timing of the MMA side only) */
+void sva_debug_set_mode(int v) { set_debug_mode(v); }
 
 }  // extern "C"

@@ -44,13 +44,26 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok;
 }
-// Bounded wait.  Returns false when the CTA is aborting.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {      // non-blocking
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false when the CTA is aborting.  SLEEP_NS > 0 backs off between polls
+// (for roles whose wake-up latency is not on the critical path) so that the polling does not
+// take issue slots from the softmax warps of the same scheduler.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
@@ -77,26 +90,32 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The MMA warp runs its loop with all lanes (so addresses and descriptors stay warp-uniform)
+// and only the elected lane executes the tcgen05 instruction itself.
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t elected) {
+  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
+               "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+               ::"r"(bar), "r"(elected) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]
 template <bool F8>
-__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc,
+                                          uint32_t elected) {
   if (F8)
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-                 "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
+                 "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
   else
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
+                 "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-               ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc,
+                                          uint32_t elected) {
+  asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
+               "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+               ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
 }
 
 #define SVA_R4(v, i) "=r"(v[i]), "=r"(v[i + 1]), "=r"(v[i + 2]), "=r"(v[i + 3])
@@ -107,6 +126,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : SVA_R4(v, 0), SVA_R4(v, 4), SVA_R4(v, 8), SVA_R4(v, 12), SVA_R4(v, 16), SVA_R4(v, 20),
         SVA_R4(v, 24), SVA_R4(v, 28)
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : SVA_R4(v, 0), SVA_R4(v, 4), SVA_R4(v, 8), SVA_R4(v, 12)
       : "r"(taddr) : "memory");
 }
 #undef SVA_R4
@@ -131,6 +157,39 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+// 2^x for x <= ~8 on the FMA pipe: round-to-nearest split x = n + f, |f| <= 0.5, cubic minimax
+// polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent added
+// to the bit pattern.  Takes and returns a pair so the packed f32x2 instructions are used.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  const float MAGIC = 12582912.0f;                       // 1.5 * 2^23
+  x.x = fmaxf(x.x, -126.0f);
+  x.y = fmaxf(x.y, -126.0f);
+  const float2 t = __fadd2_rn(x, make_float2(MAGIC, MAGIC));
+  const float2 n = __fadd2_rn(t, make_float2(-MAGIC, -MAGIC));
+  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+  float2 p = __ffma2_rn(f, make_float2(0.05517132f, 0.05517132f), make_float2(0.24261054f, 0.24261054f));
+  p = __ffma2_rn(p, f, make_float2(0.69326097f, 0.69326097f));
+  p = __ffma2_rn(p, f, make_float2(0.99992812f, 0.99992812f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return r;
+}
+__device__ __forceinline__ float ex2_poly(float x) {
+  const float MAGIC = 12582912.0f;                       // 1.5 * 2^23
+  x = fmaxf(x, -126.0f);
+  const float t = x + MAGIC;
+  const float f = x - (t - MAGIC);
+  float p = fmaf(f, 0.05517132f, 0.24261054f);
+  p = fmaf(p, f, 0.69326097f);
+  p = fmaf(p, f, 0.99992812f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -161,31 +220,44 @@ struct AttnParams {
   Strides so;
   int H, N, Nb, R;
   float scale_log2;           // softmax_scale * log2(e)
+  long long* prof;            // optional timeline buffer (tuning aid), normally null
+  int debug;                  // tuning aid: bit0 = skip the softmax arithmetic (wrong results)
 };
+
+// Timeline probe: CTA 64 records clock64() for iterations 16..23, [role][j-16][event].
+#define SVA_PROF(role, j, ev)                                                                   \
+  do {                                                                                          \
+    if (prm.prof && blockIdx.x == 64 && (j) >= 16 && (j) < 24)                                  \
+      prm.prof[(((role) * 8) + ((j) - 16)) * 8 + (ev)] = clock64();                             \
+  } while (0)
 
 template <int D, int NT, bool F8>
 struct Cfg {
   static constexpr int QK_ELEM = F8 ? 1 : 2;
   static constexpr int Q_BYTES = BS * D * QK_ELEM;       // one Q (or K) tile
-  static constexpr int V_BYTES = BS * D * 2;
-  static constexpr int STAGE_BYTES = V_BYTES;            // K tiles use a prefix of a stage
-  static constexpr int STAGES = NT == 2 ? (D == 128 ? 5 : 8) : 4;
-  static constexpr int THREADS = NT * 128 + 64;
+  static constexpr int VH_BYTES = (BS / 2) * D * 2;      // half a V tile: 64 keys
+  static constexpr int K_SLOT = BS * D * 2;              // slot size of a K tile (bf16 size also for e4m3)
+  static constexpr int KS = NT == 2 ? 1 : 2;             // K tiles in flight per query tile
+  static constexpr int VS = NT == 2 ? 3 : 6;             // V half-tiles in flight per query tile
+  static constexpr int THREADS = NT * 128 + 128;         // softmax warpgroups + one warpgroup for TMA/MMA
   static constexpr int TMEM_COLS = 512;
   // dynamic shared memory: 1024-aligned tiles first, then the control block
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_RING = OFF_Q + NT * ((Q_BYTES + 1023) / 1024 * 1024);
-  static constexpr int OFF_CTRL = OFF_RING + STAGES * STAGE_BYTES;
-  static constexpr int CTRL_BYTES = 256;
+  static constexpr int Q_SLOT = (Q_BYTES + 1023) / 1024 * 1024;
+  static constexpr int OFF_K = OFF_Q + NT * Q_SLOT;      // K slots of tile t at OFF_K + t*KS*K_SLOT
+  static constexpr int OFF_V = OFF_K + NT * KS * K_SLOT; // V half slots of tile t at OFF_V + t*VS*VH_BYTES
+  static constexpr int OFF_CTRL = OFF_V + NT * VS * VH_BYTES;
+  static constexpr int CTRL_BYTES = 384;
   static constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;   // + alignment slack
 };
 
 // control block layout (bytes from OFF_CTRL):
-//   0   q_full[2]     16  s_full[2]    32  p_full[2]    48  o_done[2]
-//   64  kv_full[8]    128 kv_empty[8]  192 tmem_base    196 abort   200 n_list[2]   208 beg[2]
+//   0   q_full[2]   16 s_full[2]   32 p_full[t] at 32 + 16*t   64 o_done[2]
+//   96 + 128*t : k_full[2] | +16 k_empty[2] | +32 v_full[6] | +80 v_empty[6]
+//   352 tmem_base   356 abort   360 n_list[2]   368 beg[2]   376 issue lock
 
-template <int D, int NT, bool F8>
-__global__ void __launch_bounds__(NT * 128 + 64, 1)
+template <int D, int NT, bool F8, int EMU>
+__global__ void __launch_bounds__(NT * 128 + 128, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams prm) {
   using C = Cfg<D, NT, F8>;
@@ -194,16 +266,16 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   const uint32_t sbase = smem_u32(smem);
   uint8_t* ctrl = smem + C::OFF_CTRL;
   const uint32_t cbase = sbase + C::OFF_CTRL;
-  const uint32_t bar_q_full = cbase + 0, bar_s_full = cbase + 16, bar_p_full = cbase + 32,
-                 bar_o_done = cbase + 48, bar_kv_full = cbase + 64, bar_kv_empty = cbase + 128;
-  volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 192);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 196);
-  volatile int* n_list = reinterpret_cast<volatile int*>(ctrl + 200);
-  volatile int* beg_list = reinterpret_cast<volatile int*>(ctrl + 208);
+  const uint32_t bar_q_full = cbase + 0, bar_s_full = cbase + 16, bar_p_half = cbase + 32,
+                 bar_o_done = cbase + 64, bar_tile = cbase + 96;
+  volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 352);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 356);
+  volatile int* n_list = reinterpret_cast<volatile int*>(ctrl + 360);
+  volatile int* beg_list = reinterpret_cast<volatile int*>(ctrl + 368);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int W_PROD = 4 * NT, W_MMA = 4 * NT + 1;
-  const int row0 = blockIdx.x * NT;                 // first CSR row of this CTA
+  constexpr int W_PROD = 4 * NT, W_MMA = 4 * NT + 2;   // producers: W_PROD + t; MMA issuers: W_MMA + t
+  const int row0 = blockIdx.x * NT;                    // first CSR row of this CTA
   const int Nb = prm.Nb;
   const bool dense = prm.row_ptr == nullptr;
 
@@ -212,14 +284,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int t = 0; t < 2; ++t) {
       mbar_init(bar_q_full + 8 * t, 1);
       mbar_init(bar_s_full + 8 * t, 1);
-      mbar_init(bar_p_full + 8 * t, 128);
+      mbar_init(bar_p_half + 16 * t, 128);
+      mbar_init(bar_p_half + 16 * t + 8, 128);
       mbar_init(bar_o_done + 8 * t, 1);
     }
-    for (int s = 0; s < 8; ++s) {
-      mbar_init(bar_kv_full + 8 * s, 1);
-      mbar_init(bar_kv_empty + 8 * s, 1);
-    }
+    for (int s = 0; s < 32; ++s) mbar_init(bar_tile + 8 * s, 1);      // k/v full and empty, both tiles
     *abort_flag = 0;
+    *reinterpret_cast<volatile int*>(ctrl + 376) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -228,7 +299,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
   if (warp == W_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(cbase + 192), "r"((uint32_t)C::TMEM_COLS) : "memory");
+                 ::"r"(cbase + 352), "r"((uint32_t)C::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // warp 4t validates the CSR row of tile t; a row holding a bad entry is treated as empty
@@ -271,118 +342,164 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   lbeg[0] = beg_list[0];
   lbeg[1] = NT == 2 ? beg_list[1] : 0;
 
-  if (warp == W_PROD) {
-    // ------------------------------------------------------------ producer
-    if (lane == 0) {
-      bool ok = true;
-      for (int t = 0; t < NT; ++t) {
-        if (nl[t] == 0) continue;
+  // Register re-partition: the TMA/MMA warpgroup needs few registers, a softmax thread holds a
+  // whole 128-wide row.  Issued at the top of each branch so the limit is tied to that branch.
+  if (warp >= 4 * NT) {
+    if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
+    if (warp >= W_PROD && warp < W_PROD + NT) {
+      // ---------------------------------------------------------- producer of tile t
+      // lane 0 streams Q and the K tiles, lane 1 the V half-tiles (64 keys each); the two streams
+      // have their own slots and barriers so that V runs a whole block ahead.
+      const int t = warp - W_PROD;
+      const int n = nl[t];
+      const int bh_t = (row0 + t) / Nb;
+      const int hh = bh_t % prm.H, bb = bh_t / prm.H;
+      const uint32_t bt = bar_tile + 128 * t;
+      if (lane == 0 && n > 0) {
         const int I = (row0 + t) % Nb;
-        const int bh_t = (row0 + t) / Nb;
         mbar_expect_tx(bar_q_full + 8 * t, C::Q_BYTES);
-        const uint32_t dst = sbase + C::OFF_Q + t * C::Q_BYTES;
-        if (F8 || D == 64) {
-          tma_load_4d(dst, &tm_q, bar_q_full + 8 * t, 0, I * BS, bh_t % prm.H, bh_t / prm.H);
-        } else {
-          tma_load_4d(dst, &tm_q, bar_q_full + 8 * t, 0, I * BS, bh_t % prm.H, bh_t / prm.H);
-          tma_load_4d(dst + C::Q_BYTES / 2, &tm_q, bar_q_full + 8 * t, 64, I * BS, bh_t % prm.H, bh_t / prm.H);
-        }
-      }
-      int stage = 0;
-      uint32_t phase = 0;
-      auto load_tile = [&](bool is_v, int t, int j) -> bool {
-        if (!mbar_wait(bar_kv_empty + 8 * stage, phase ^ 1u, abort_flag, prm.status)) return false;
-        const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
-        const int bh_t = (row0 + t) / Nb;
-        const int hh = bh_t % prm.H, bb = bh_t / prm.H;
-        const uint32_t dst = sbase + C::OFF_RING + stage * C::STAGE_BYTES;
-        const uint32_t bar = bar_kv_full + 8 * stage;
-        if (is_v) {
-          mbar_expect_tx(bar, C::V_BYTES);
-          tma_load_4d(dst, &tm_v, bar, 0, J * BS, hh, bb);
-          if (D == 128) tma_load_4d(dst + C::V_BYTES / 2, &tm_v, bar, 64, J * BS, hh, bb);
-        } else {
+        const uint32_t qdst = sbase + C::OFF_Q + t * C::Q_SLOT;
+        tma_load_4d(qdst, &tm_q, bar_q_full + 8 * t, 0, I * BS, hh, bb);
+        if (!F8 && D == 128) tma_load_4d(qdst + C::Q_BYTES / 2, &tm_q, bar_q_full + 8 * t, 64, I * BS, hh, bb);
+        int ks = 0;
+        uint32_t kphase = 0;
+        for (int j = 0; j < n; ++j) {
+          if (!mbar_wait(bt + 16 + 8 * ks, kphase ^ 1u, abort_flag, prm.status)) break;
+          const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
+          const uint32_t dst = sbase + C::OFF_K + (t * C::KS + ks) * C::K_SLOT;
+          const uint32_t bar = bt + 8 * ks;
           mbar_expect_tx(bar, C::Q_BYTES);
           tma_load_4d(dst, &tm_k, bar, 0, J * BS, hh, bb);
           if (!F8 && D == 128) tma_load_4d(dst + C::Q_BYTES / 2, &tm_k, bar, 64, J * BS, hh, bb);
+          if (++ks == C::KS) { ks = 0; kphase ^= 1u; }
         }
-        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-        return true;
-      };
-      // tile order must match the MMA warp's consumption order exactly
-      for (int t = 0; t < NT && ok; ++t)
-        if (nl[t] > 0) ok = load_tile(false, t, 0);
-      const int nmax = nl[0] > nl[1] ? nl[0] : nl[1];
-      for (int j = 0; j < nmax && ok; ++j)
-        for (int t = 0; t < NT && ok; ++t) {
-          if (j < nl[t]) ok = load_tile(true, t, j);
-          if (ok && j + 1 < nl[t]) ok = load_tile(false, t, j + 1);
+      } else if (lane == 1 && n > 0) {
+        int vs = 0;
+        uint32_t vphase = 0;
+        for (int i = 0; i < 2 * n; ++i) {
+          if (!mbar_wait<60>(bt + 80 + 8 * vs, vphase ^ 1u, abort_flag, prm.status)) break;
+          const int J = dense ? (i >> 1) : __ldg(prm.col_idx + lbeg[t] + (i >> 1));
+          const uint32_t dst = sbase + C::OFF_V + (t * C::VS + vs) * C::VH_BYTES;
+          const uint32_t bar = bt + 32 + 8 * vs;
+          mbar_expect_tx(bar, C::VH_BYTES);
+          tma_load_4d(dst, &tm_v, bar, 0, J * BS + (i & 1) * (BS / 2), hh, bb);
+          if (D == 128) tma_load_4d(dst + C::VH_BYTES / 2, &tm_v, bar, 64, J * BS + (i & 1) * (BS / 2), hh, bb);
+          if (++vs == C::VS) { vs = 0; vphase ^= 1u; }
         }
-    }
-  } else if (warp == W_MMA) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t IDESC_QK = instr_desc(128, BS, F8 ? 0 : 1, false);
-      constexpr uint32_t IDESC_PV = instr_desc(128, D, 1, true);
-      constexpr int QK_KSTEP_BYTES = 32;                          // 16 bf16 or 32 e4m3
-      constexpr int QK_KSTEPS = D * C::QK_ELEM / QK_KSTEP_BYTES;
-      constexpr int QK_PANEL_BYTES = BS * 128;                    // 128 rows x 128-byte swizzle row
-      bool ok = true;
-      int stage = 0;
-      uint32_t phase = 0;
-      auto advance = [&]() { if (++stage == C::STAGES) { stage = 0; phase ^= 1u; } };
-      auto issue_s = [&](int t, int j) -> bool {
-        if (j == 0 && !mbar_wait(bar_q_full + 8 * t, 0, abort_flag, prm.status)) return false;
-        if (!mbar_wait(bar_kv_full + 8 * stage, phase, abort_flag, prm.status)) return false;
-        tc_fence_after();
-        const uint32_t qa = sbase + C::OFF_Q + t * C::Q_BYTES;
-        const uint32_t ka = sbase + C::OFF_RING + stage * C::STAGE_BYTES;
-        const uint32_t d_tmem = tmem_base + 128 * t;
-#pragma unroll
-        for (int kk = 0; kk < QK_KSTEPS; ++kk) {
-          const uint32_t off = (kk / 4) * QK_PANEL_BYTES + (kk % 4) * QK_KSTEP_BYTES;
-          tc_mma_ss<F8>(d_tmem, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK,
-                        kk > 0 ? 1u : 0u);
-        }
-        tc_commit(bar_kv_empty + 8 * stage);
-        tc_commit(bar_s_full + 8 * t);
-        advance();
-        return true;
-      };
-      auto issue_pv = [&](int t, int j) -> bool {
-        if (!mbar_wait(bar_p_full + 8 * t, (uint32_t)(j & 1), abort_flag, prm.status)) return false;
-        if (!mbar_wait(bar_kv_full + 8 * stage, phase, abort_flag, prm.status)) return false;
-        tc_fence_after();
-        const uint32_t va = sbase + C::OFF_RING + stage * C::STAGE_BYTES;
-        const uint32_t p_tmem = tmem_base + 128 * t;
+      }
+    } else if (warp >= W_MMA && warp < W_MMA + NT) {
+      // ---------------------------------------------------------- MMA issuer of tile t (one lane)
+      // Per block j: P V (two V half-tiles), then S(j+1).  Each issuer blocks only on its own
+      // tile's barriers; a lock taken around every group of MMAs makes the two tiles' groups
+      // reach the tensor pipe one after the other, which keeps the two softmax warpgroups out of
+      // phase (so that one tile's exponentials overlap the other tile's MMAs).
+      const int t = warp - W_MMA;
+      if (lane == 0 && nl[t] > 0) {
+        const uint32_t IDESC_QK = instr_desc(128, BS, F8 ? 0 : 1, false);
+        const uint32_t IDESC_PV = instr_desc(128, D, 1, true);
+        constexpr int QK_KSTEPS = D * C::QK_ELEM / 32;              // 32 bytes of K per MMA
+        const int n = nl[t];
+        int* lock = reinterpret_cast<int*>(ctrl + 376);
+        const uint32_t bt = bar_tile + 128 * t;
+        const uint64_t qd = smem_desc(sbase + C::OFF_Q + t * C::Q_SLOT, 16, 1024);
+        const uint64_t kdesc0 = smem_desc(sbase + C::OFF_K + t * C::KS * C::K_SLOT, 16, 1024);
+        // V half-tile: two 64-wide d panels of 64 keys x 128 bytes, panel stride = half of the slot
+        const uint64_t vdesc0 = smem_desc(sbase + C::OFF_V + t * C::VS * C::VH_BYTES, C::VH_BYTES / 2, 1024);
+        const uint32_t s_tmem = tmem_base + 128 * t;
         const uint32_t o_tmem = tmem_base + 128 * NT + 128 * t;
+        int ks = 0, vs = 0;
+        uint32_t kphase = 0, vphase = 0;
+        auto acquire = [&]() -> bool {
+          if (NT == 1 || (prm.debug & 8)) return true;
+          uint32_t spins = 0;
+          const long long t0 = clock64();
+          while (atomicCAS(lock, 0, 1) != 0) {
+            if ((++spins & 63u) == 0u) {
+              if (*abort_flag) return false;
+              if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                if (prm.status) atomicOr(prm.status, SVA_DEV_TIMEOUT);
+                return false;
+              }
+            }
+          }
+          return true;
+        };
+        auto release = [&]() { if (NT == 2 && !(prm.debug & 8)) atomicExch(lock, 0); };
+        auto issue_s = [&](int j) {                                  // K(j) must be resident
+          const uint64_t kd = kdesc0 + (uint64_t)(ks * (C::K_SLOT >> 4));
 #pragma unroll
-        for (int kk = 0; kk < BS / 16; ++kk)
-          tc_mma_ts(o_tmem, p_tmem + 8 * kk, smem_desc(va + kk * 2048, BS * 128, 1024), IDESC_PV,
-                    (j > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(bar_kv_empty + 8 * stage);
-        if (j == nl[t] - 1) tc_commit(bar_o_done + 8 * t);
-        advance();
-        return true;
-      };
-      for (int t = 0; t < NT && ok; ++t)
-        if (nl[t] > 0) ok = issue_s(t, 0);
-      const int nmax = nl[0] > nl[1] ? nl[0] : nl[1];
-      for (int j = 0; j < nmax && ok; ++j)
-        for (int t = 0; t < NT && ok; ++t) {
-          if (j < nl[t]) ok = issue_pv(t, j);
-          if (ok && j + 1 < nl[t]) ok = issue_s(t, j + 1);
+          for (int kk = 0; kk < QK_KSTEPS; ++kk) {
+            constexpr int PANEL16 = (BS * 128) >> 4;
+            const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+            tc_mma_ss<F8>(s_tmem, qd + off, kd + off, IDESC_QK, kk > 0 ? 1u : 0u, 1u);
+          }
+          tc_commit(bt + 16 + 8 * ks, 1u);
+          tc_commit(bar_s_full + 8 * t, 1u);
+          SVA_PROF(2 + t, j - 1, 5);
+          if (++ks == C::KS) { ks = 0; kphase ^= 1u; }
+        };
+        auto issue_pv_half = [&](int j, int half) {                  // V half-tile vs must be resident
+          const uint64_t vd = vdesc0 + (uint64_t)(vs * (C::VH_BYTES >> 4));
+#pragma unroll
+          for (int kk = 0; kk < BS / 32; ++kk)
+            tc_mma_ts(o_tmem, s_tmem + 8 * (kk + half * (BS / 32)), vd + (uint64_t)(kk * (2048 >> 4)), IDESC_PV,
+                      (j > 0 || half > 0 || kk > 0) ? 1u : 0u, 1u);
+          tc_commit(bt + 80 + 8 * vs, 1u);
+          if (++vs == C::VS) { vs = 0; vphase ^= 1u; }
+        };
+        bool ok = mbar_wait(bar_q_full + 8 * t, 0, abort_flag, prm.status) &&
+                  mbar_wait(bt + 8 * ks, kphase, abort_flag, prm.status);
+        if (ok) {
+          tc_fence_after();
+          ok = acquire();
+          if (ok) { issue_s(0); release(); }
         }
+        for (int j = 0; j < n && ok; ++j) {
+          // One group per block: P V (two V half-tiles) directly followed by S of the next block.
+          // The tensor pipe drains whenever consecutive MMAs change kind (A from shared memory
+          // vs tensor memory, or another instruction descriptor), so kinds are kept together and
+          // the other tile's group never lands in the middle.
+          const bool more = j + 1 < n;
+          int vs2 = vs + 1;
+          uint32_t vphase2 = vphase;
+          if (vs2 == C::VS) { vs2 = 0; vphase2 ^= 1u; }
+          ok = mbar_wait(bar_p_half + 16 * t, (uint32_t)(j & 1), abort_flag, prm.status) &&
+               mbar_wait(bt + 32 + 8 * vs, vphase, abort_flag, prm.status) &&
+               mbar_wait(bt + 32 + 8 * vs2, vphase2, abort_flag, prm.status);
+          if (!ok) break;
+          SVA_PROF(2 + t, j, 1);
+          tc_fence_after();
+          ok = acquire();
+          if (!ok) break;
+          SVA_PROF(2 + t, j, 0);
+          issue_pv_half(j, 0);
+          issue_pv_half(j, 1);
+          if (j == n - 1) tc_commit(bar_o_done + 8 * t, 1u);
+          SVA_PROF(2 + t, j, 2);
+          if (more && !mbar_test(bt + 8 * ks, kphase)) {
+            // K(j+1) has not landed yet: let the other tile use the pipe meanwhile
+            release();
+            ok = mbar_wait(bt + 8 * ks, kphase, abort_flag, prm.status) && acquire();
+            if (!ok) break;
+          }
+          if (more) issue_s(j + 1);
+          release();
+        }
+      }
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
+    // warpgroup t owns tile t; thread <-> query row <-> TMEM lane, all 128 key columns
+    if (NT == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
     const int t = warp >> 2;
     const int r = row0 + t;
     const int n = nl[t];
-    const int row = (warp & 3) * 32 + lane;                  // row of the tile == TMEM lane
+    const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t s_tmem = tmem_base + lane_addr + 128 * t;
     const uint32_t o_tmem = tmem_base + lane_addr + 128 * NT + 128 * t;
+    const bool probe = (threadIdx.x & 127) == 0;
     if (r < prm.R) {
       const int I = r % Nb;
       const int bh_t = r / Nb;
@@ -396,59 +513,79 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       for (int j = 0; j < n; ++j) {
         const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
         if (F8) c = prm.scale_log2 * qs * __ldg(prm.k_scale + (long long)bh_t * Nb + J);
+        const int valid = (J == Nb - 1) ? tail_keys : BS;      // key columns of this block that exist
+        if (probe) SVA_PROF(t, j, 0);
         if (!mbar_wait(bar_s_full + 8 * t, (uint32_t)(j & 1), abort_flag, prm.status)) { ok = false; break; }
+        if (probe) SVA_PROF(t, j, 1);
         tc_fence_after();
+        if (prm.debug & 1) {
+          tc_fence_before();
+          mbar_arrive(bar_p_half + 16 * t);
+          l = 1.f;
+          continue;
+        }
+        // ---- row maximum over the 128 columns (whole row in registers)
         uint32_t sv[128];
         tmem_ld32(s_tmem + 0, sv + 0);
         tmem_ld32(s_tmem + 32, sv + 32);
         tmem_ld32(s_tmem + 64, sv + 64);
         tmem_ld32(s_tmem + 96, sv + 96);
         tc_wait_ld();
-        if (J == Nb - 1 && tail_keys < BS) {
+        if (probe) SVA_PROF(t, j, 2);
+        if (valid < BS) {
 #pragma unroll
           for (int i = 0; i < 128; ++i)
-            if (i >= tail_keys) sv[i] = 0xff800000u;          // -inf
+            if (i >= valid) sv[i] = 0xff800000u;              // keys that do not exist: -inf
         }
-        float mx = -INFINITY;
+        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
-        mx *= c;
+        for (int i = 0; i < 128; i += 8) {
+          mxa = max3(mxa, __uint_as_float(sv[i + 0]), __uint_as_float(sv[i + 1]));
+          mxb = max3(mxb, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+          mxc = max3(mxc, __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
+          mxd = max3(mxd, __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
+        }
+        const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd)) * c;
         // lazy rescale: move the reference maximum only when it would grow by more than 2^8
-        const bool need = mx > m_used + 8.0f;
-        if (__any_sync(0xffffffffu, need)) {
+        if (__any_sync(0xffffffffu, mx > m_used + 8.0f)) {
           const float m_new = fmaxf(m_used, mx);
           const float alpha = ex2(m_used - m_new);            // first block: exp2(-inf) = 0
           l *= alpha;
           m_used = m_new;
           if (j > 0) {
-#pragma unroll
-            for (int cc = 0; cc < D; cc += 32) {
-              uint32_t ov[32];
-              tmem_ld32(o_tmem + cc, ov);
+#pragma unroll 1
+            for (int cc = 0; cc < D; cc += 16) {
+              uint32_t ov[16];
+              tmem_ld16(o_tmem + cc, ov);
               tc_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-              tmem_st32(o_tmem + cc, ov);
+              for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+              tmem_st16(o_tmem + cc, ov);
             }
           }
         }
-        float sum = 0.f;
+        if (probe) SVA_PROF(t, j, 3);
+        // ---- P = 2^(S*c - m_used).  EMU of every 8 elements take a polynomial on the FMA pipe,
+        // the others the MUFU.  Packed bf16 pairs overwrite sv[0..63].
+        const float nm = -m_used;
+        float sum_a = 0.f, sum_b = 0.f;
 #pragma unroll
-        for (int cc = 0; cc < 128; cc += 32) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[cc + 2 * i]), c, -m_used));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[cc + 2 * i + 1]), c, -m_used));
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
-          }
-          tmem_st16(s_tmem + cc / 2, pk);
+        for (int i = 0; i < 128; i += 2) {
+          const float x0 = fmaf(__uint_as_float(sv[i]), c, nm), x1 = fmaf(__uint_as_float(sv[i + 1]), c, nm);
+          const float p0 = ((i & 7) < EMU) ? ex2_poly(x0) : ex2(x0);
+          const float p1 = (((i + 1) & 7) < EMU) ? ex2_poly(x1) : ex2(x1);
+          sum_a += p0;
+          sum_b += p1;
+          sv[i / 2] = pack_bf16(p0, p1);
+          if (i == 62) tmem_st32(s_tmem, sv);
         }
-        l += sum;
+        tmem_st32(s_tmem + 32, sv + 32);
+        l += sum_a + sum_b;
+        if (probe) SVA_PROF(t, j, 4);
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p_full + 8 * t);
+        mbar_arrive(bar_p_half + 16 * t);
+        if (probe) SVA_PROF(t, j, 5);
       }
       // ---- epilogue
       __nv_bfloat16* orow = prm.o + (long long)(bh_t / prm.H) * prm.so.b + (long long)(bh_t % prm.H) * prm.so.h +
@@ -520,7 +657,7 @@ static encode_fn_t get_encode() {
 
 // [B,H,N,d] tensor with element strides s, as a 4-D map (d, N, H, B); box = 128 bytes x 128 rows.
 static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, int H, int N, int d,
-                    const Strides& s) {
+                    const Strides& s, int box_rows) {
   encode_fn_t enc = get_encode();
   if (!enc) return SVA_ERR_CUDA;
   cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
@@ -532,7 +669,7 @@ static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, in
     if (strides[i] % 16 != 0 || strides[i] == 0) return SVA_ERR_ALIGNMENT;
   int inner = 128 / elem_bytes;
   if (inner > d) inner = d;
-  cuuint32_t box[4] = {(cuuint32_t)inner, (cuuint32_t)BS, 1, 1};
+  cuuint32_t box[4] = {(cuuint32_t)inner, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult rc = enc(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
                     const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -542,12 +679,15 @@ static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, in
 }
 
 static int g_tiles_per_cta = 2;   // bring-up switch, see sva_debug_set_tiles_per_cta
+static long long* g_prof = nullptr;   // tuning aid, see sva_debug_set_prof_buffer
+static int g_debug = 0;
+static int g_emu = 2;             // tuning switch: pairs per 4 whose exp2 runs on the FMA pipe
 
-template <int D, int NT, bool F8>
+template <int D, int NT, bool F8, int EMU>
 static int launch_cfg(const Dims& m, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                       const AttnParams& prm, cudaStream_t st) {
   using C = Cfg<D, NT, F8>;
-  auto kern = attn_sm100_kernel<D, NT, F8>;
+  auto kern = attn_sm100_kernel<D, NT, F8, EMU>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
     return SVA_ERR_CUDA;
   const int grid = (m.R + NT - 1) / NT;
@@ -563,23 +703,36 @@ int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, cons
   CUtensorMap tq, tk, tv;
   const int eb = m.fp8 ? 1 : 2;
   int rc;
-  if ((rc = make_map(&tq, q, eb, m.B, m.H, m.N, m.d, make_strides(p->q_stride))) != SVA_OK) return rc;
-  if ((rc = make_map(&tk, k, eb, m.B, m.H, m.N, m.d, make_strides(p->k_stride))) != SVA_OK) return rc;
-  if ((rc = make_map(&tv, v, 2, m.B, m.H, m.N, m.d, make_strides(p->v_stride))) != SVA_OK) return rc;
+  if ((rc = make_map(&tq, q, eb, m.B, m.H, m.N, m.d, make_strides(p->q_stride), BS)) != SVA_OK) return rc;
+  if ((rc = make_map(&tk, k, eb, m.B, m.H, m.N, m.d, make_strides(p->k_stride), BS)) != SVA_OK) return rc;
+  if ((rc = make_map(&tv, v, 2, m.B, m.H, m.N, m.d, make_strides(p->v_stride), BS / 2)) != SVA_OK) return rc;
   AttnParams prm;
   prm.row_ptr = row_ptr; prm.col_idx = col_idx; prm.q_scale = qs; prm.k_scale = ks;
   prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
   prm.so = make_strides(p->o_stride);
   prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
   prm.scale_log2 = m.scale * 1.4426950408889634f;
+  prm.prof = g_prof;
+  prm.debug = g_debug;
   // a CTA's tiles must belong to one head: pair tiles only when Nb is even
   const int nt = (g_tiles_per_cta == 2 && m.Nb % 2 == 0) ? 2 : 1;
-  if (m.fp8) return nt == 2 ? launch_cfg<128, 2, true>(m, tq, tk, tv, prm, st)
-                            : launch_cfg<128, 1, true>(m, tq, tk, tv, prm, st);
-  return nt == 2 ? launch_cfg<128, 2, false>(m, tq, tk, tv, prm, st)
-                 : launch_cfg<128, 1, false>(m, tq, tk, tv, prm, st);
+#define SVA_DISPATCH(NTV, F8V)                                                        \
+  switch (g_emu) {                                                                     \
+    case 0: return launch_cfg<128, NTV, F8V, 0>(m, tq, tk, tv, prm, st);              \
+    case 1: return launch_cfg<128, NTV, F8V, 1>(m, tq, tk, tv, prm, st);              \
+    case 2: return launch_cfg<128, NTV, F8V, 2>(m, tq, tk, tv, prm, st);              \
+    default: return launch_cfg<128, NTV, F8V, 3>(m, tq, tk, tv, prm, st);             \
+  }
+  if (m.fp8) {
+    if (nt == 2) { SVA_DISPATCH(2, true) } else { SVA_DISPATCH(1, true) }
+  }
+  if (nt == 2) { SVA_DISPATCH(2, false) } else { SVA_DISPATCH(1, false) }
+#undef SVA_DISPATCH
 }
 
 void set_tiles_per_cta(int n) { g_tiles_per_cta = n == 1 ? 1 : 2; }
+void set_prof_buffer(void* p) { g_prof = (long long*)p; }
+void set_debug_mode(int v) { g_debug = v; }
+void set_exp_emulation(int n) { g_emu = n < 0 ? 0 : (n > 3 ? 3 : n); }
 
 }  // namespace sva

@@ -77,7 +77,7 @@ pool_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, Stride
   }
 }
 
-static constexpr int SEL_WARPS = 8;     // query-block rows per CTA
+static constexpr int SEL_WARPS = 16;    // query-block rows per CTA, one warp each
 static constexpr int SEL_CHUNK = 32;    // key blocks staged per pass
 
 struct SelParams {
@@ -90,20 +90,32 @@ __device__ __forceinline__ bool in_window(int I, int J, const SelParams& p) {
   return abs(ti - tj) <= p.win_t && abs(si - sj) <= p.win_s;
 }
 
-// dynamic smem: qs[SEL_WARPS][D] | ks[SEL_CHUNK][D] | sc[SEL_WARPS][Nb32]
-template <int D>
+// Order-preserving map float -> uint32 (larger score <=> larger key, every real score maps to a
+// non-zero key); +0 and -0 share a key; NaN maps to 0, which is never selected.
+__device__ __forceinline__ uint32_t score_key(float v) {
+  if (!(v == v)) return 0u;
+  uint32_t u = __float_as_uint(v + 0.0f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_score(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
+}
+
+// One CTA scores and selects SEL_WARPS query-block rows of one head, one warp per row.
+// Lane j of a warp owns the key blocks J = it*32 + j, it < ITEMS, and keeps their scores in
+// registers (as sortable keys); a chunk of 32 pooled keys is staged transposed in shared memory
+// so that lane j reads key j conflict-free while the query values are 128-bit broadcasts.
+// smem: qs[SEL_WARPS][D] | ksT[D][33]
+template <int D, int ITEMS>
 __global__ void __launch_bounds__(SEL_WARPS * 32)
 score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, SelParams p,
                     int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx,
                     int32_t* __restrict__ tmp_idx, int32_t* __restrict__ counts,
                     float* __restrict__ block_scores, int R) {
-  extern __shared__ float smem[];
+  constexpr int KT_LD = SEL_CHUNK + 1;
+  __shared__ __align__(16) float qs[SEL_WARPS * D];
+  __shared__ float ksT[D * KT_LD];
   const int Nb = p.Nb;
-  const int Nb32 = (Nb + 31) & ~31;
-  float* qs = smem;
-  float* ks = qs + SEL_WARPS * D;
-  float* sc = ks + SEL_CHUNK * D;
-
   const int bh = blockIdx.y;
   const int I0 = blockIdx.x * SEL_WARPS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -115,61 +127,69 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
     qs[i] = (I0 + w < Nb) ? qbar[((long long)bh * Nb + I0 + w) * D + (i % D)] : 0.f;
   }
   const float* kb = kbar + (long long)bh * Nb * D;
-  float* my_sc = sc + warp * Nb32;
 
-  for (int c0 = 0; c0 < Nb; c0 += SEL_CHUNK) {
-    __syncthreads();
-    const int nrow = min(SEL_CHUNK, Nb - c0);
-    for (int i = threadIdx.x; i < SEL_CHUNK * D / 4; i += blockDim.x) {
-      int rr = i / (D / 4);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (rr < nrow) v = __ldg(reinterpret_cast<const float4*>(kb + (long long)c0 * D) + i);
-      reinterpret_cast<float4*>(ks)[i] = v;
-    }
-    __syncthreads();
-    // lane j scores key block c0+j; the column index is rotated by the lane so that the 32
-    // lanes touch 32 different banks
-    float acc = 0.f;
-    const float* qrow = qs + warp * D;
-    const float* krow = ks + lane * D;
+  uint32_t key[ITEMS];
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+    key[it] = 0u;
+    if (it * 32 < Nb) {                      // uniform over the CTA
+      __syncthreads();
+      const int J = it * 32 + lane;
+      for (int cc = warp; cc < D / 4; cc += SEL_WARPS) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (J < Nb) v = __ldg(reinterpret_cast<const float4*>(kb + (long long)J * D) + cc);
+        ksT[(4 * cc + 0) * KT_LD + lane] = v.x;
+        ksT[(4 * cc + 1) * KT_LD + lane] = v.y;
+        ksT[(4 * cc + 2) * KT_LD + lane] = v.z;
+        ksT[(4 * cc + 3) * KT_LD + lane] = v.w;
+      }
+      __syncthreads();
+      float a0 = 0.f, a1 = 0.f;
 #pragma unroll 8
-    for (int c = 0; c < D; ++c) {
-      int idx = (c + lane) & (D - 1);
-      acc = fmaf(qrow[idx], krow[idx], acc);
+      for (int c = 0; c < D; c += 4) {
+        const float4 qv = *reinterpret_cast<const float4*>(qs + warp * D + c);
+        a0 = fmaf(qv.x, ksT[(c + 0) * KT_LD + lane], a0);
+        a1 = fmaf(qv.y, ksT[(c + 1) * KT_LD + lane], a1);
+        a0 = fmaf(qv.z, ksT[(c + 2) * KT_LD + lane], a0);
+        a1 = fmaf(qv.w, ksT[(c + 3) * KT_LD + lane], a1);
+      }
+      const float v = (a0 + a1) * p.scale;
+      if (J < Nb) {
+        key[it] = score_key(v);
+        if (block_scores && row_ok) block_scores[((long long)bh * Nb + I) * Nb + J] = v;
+      }
     }
-    acc *= p.scale;
-    int J = c0 + lane;
-    my_sc[J] = (J < Nb) ? acc : -INFINITY;
-    if (block_scores && row_ok && J < Nb) block_scores[((long long)bh * Nb + I) * Nb + J] = acc;
   }
-  __syncwarp();
   if (!row_ok) return;
 
-  // ---- per-row selection, one warp.  Item (it, lane) <-> key block J = it*32 + lane.
-  const int items = Nb32 / 32;
+  // ---- selection
   uint32_t mask = 0;            // bit it set <=> block it*32+lane is kept
   int n = 0;
   float cum = 0.f, mx = 0.f, inv_z = 0.f;
-
   if (p.mode == 1) {
-    float m = -INFINITY;
-    for (int it = 0; it < items; ++it) m = fmaxf(m, my_sc[it * 32 + lane]);
+    uint32_t km = 0u;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    for (int it = 0; it < ITEMS; ++it) km = max(km, key[it]);
+    km = __reduce_max_sync(0xffffffffu, km);
+    mx = key_score(km);
     float z = 0.f;
-    for (int it = 0; it < items; ++it) z += expf(my_sc[it * 32 + lane] - m);   // exp(-inf) = 0
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it)
+      if (key[it]) z += expf(key_score(key[it]) - mx);
 #pragma unroll
     for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-    mx = m; inv_z = 1.0f / z;
+    inv_z = 1.0f / z;
   }
   if (p.use_window) {
     float fm = 0.f;
     int cnt = 0;
-    for (int it = 0; it < items; ++it) {
-      int J = it * 32 + lane;
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+      const int J = it * 32 + lane;
       if (J < Nb && in_window(I, J, p)) {
         mask |= 1u << it; ++cnt;
-        if (p.mode == 1) fm += expf(my_sc[J] - mx) * inv_z;
+        if (p.mode == 1) fm += expf(key_score(key[it]) - mx) * inv_z;
+        key[it] = 0u;                        // no longer a candidate
       }
     }
 #pragma unroll
@@ -183,24 +203,23 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
   while (true) {
     if (n >= kk) break;
     if (p.mode == 1 && n >= 1 && cum >= p.tau) break;
-    float bv = -INFINITY;
-    int bj = 0x7fffffff;
-    for (int it = 0; it < items; ++it) {
-      if (mask >> it & 1u) continue;
-      int J = it * 32 + lane;
-      float v = my_sc[J];
-      if (J < Nb && v == v && (bj == 0x7fffffff || v > bv || (v == bv && J < bj))) { bv = v; bj = J; }
-    }
+    // lane-local best: highest key, lowest item on ties (strict > while scanning upwards)
+    uint32_t bkey = 0u;
+    int bit = 0;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-      if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) { bv = ov; bj = oj; }
+    for (int it = 0; it < ITEMS; ++it)
+      if (key[it] > bkey) { bkey = key[it]; bit = it; }
+    const uint32_t top = __reduce_max_sync(0xffffffffu, bkey);
+    if (top == 0u) break;                     // nothing selectable left
+    const uint32_t win = __reduce_min_sync(0xffffffffu, bkey == top ? (uint32_t)(bit * 32 + lane) : 0x7fffffffu);
+    if ((int)(win & 31u) == lane) {
+      mask |= 1u << (win >> 5);
+#pragma unroll
+      for (int it = 0; it < ITEMS; ++it)
+        if (it == (int)(win >> 5)) key[it] = 0u;
     }
-    if (bj == 0x7fffffff) break;            // nothing selectable left (all NaN)
-    if ((bj & 31) == lane) mask |= 1u << (bj >> 5);
     ++n;
-    if (p.mode == 1) cum += expf(bv - mx) * inv_z;
+    if (p.mode == 1) cum += expf(key_score(top) - mx) * inv_z;
   }
 
   // ---- emit ascending
@@ -217,7 +236,9 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
     if (lane == 0) counts[r] = n;
   }
   int base = 0;
-  for (int it = 0; it < items; ++it) {
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+    if (it * 32 >= Nb) break;
     bool sel = mask >> it & 1u;
     uint32_t bal = __ballot_sync(0xffffffffu, sel);
     if (sel) out[base + __popc(bal & ((1u << lane) - 1u))] = it * 32 + lane;
@@ -334,13 +355,17 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   sp.use_window = (s->win_t >= 0 && s->win_s >= 0 && s->blocks_per_frame > 0) ? 1 : 0;
   sp.win_t = s->win_t; sp.win_s = s->win_s; sp.bpf = sp.use_window ? s->blocks_per_frame : 1;
   sp.cap = cap; sp.fixed_n = fixed_n; sp.scale = m.scale; sp.tau = s->mass;
-  const int Nb32 = (m.Nb + 31) & ~31;
-  size_t smem = (size_t)(SEL_WARPS * D + SEL_CHUNK * D + SEL_WARPS * Nb32) * sizeof(float);
-  if (cudaFuncSetAttribute(score_select_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
-    return SVA_ERR_CUDA;
+  const int items = (m.Nb + 31) / 32;
   dim3 sg((m.Nb + SEL_WARPS - 1) / SEL_WARPS, m.B * m.H);
-  score_select_kernel<D><<<sg, SEL_WARPS * 32, smem, st>>>(qbar, kbar, sp, row_ptr, col_idx, tmp_idx,
-                                                           counts, block_scores, m.R);
+#define SVA_SEL_LAUNCH(IT)                                                                          \
+  score_select_kernel<D, IT><<<sg, SEL_WARPS * 32, 0, st>>>(qbar, kbar, sp, row_ptr, col_idx, tmp_idx, \
+                                                             counts, block_scores, m.R)
+  if (items <= 4) SVA_SEL_LAUNCH(4);
+  else if (items <= 8) SVA_SEL_LAUNCH(8);
+  else if (items <= 12) SVA_SEL_LAUNCH(12);
+  else if (items <= 16) SVA_SEL_LAUNCH(16);
+  else SVA_SEL_LAUNCH(32);
+#undef SVA_SEL_LAUNCH
   if (!fixed_n) {
     scan_kernel<<<1, 1024, 0, st>>>(counts, m.R, row_ptr);
     compact_kernel<<<(m.R * 32 + 255) / 256, 256, 0, st>>>(tmp_idx, counts, row_ptr, cap, m.R, col_idx);
