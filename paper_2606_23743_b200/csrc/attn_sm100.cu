@@ -681,7 +681,7 @@ static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, in
 static int g_tiles_per_cta = 2;   // bring-up switch, see sva_debug_set_tiles_per_cta
 static long long* g_prof = nullptr;   // tuning aid, see sva_debug_set_prof_buffer
 static int g_debug = 0;
-static int g_emu = 2;             // tuning switch: pairs per 4 whose exp2 runs on the FMA pipe
+static int g_emu = 0;             // tuning switch: pairs per 4 whose exp2 runs on the FMA pipe
 
 template <int D, int NT, bool F8, int EMU>
 static int launch_cfg(const Dims& m, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
