@@ -34,8 +34,8 @@ METRIC = "block-sparse attn fwd effective TFLOPS (selected blocks)"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the "large" workload,
-# from the ncu capture summarised in profiles/ (None until captured)
-ATTN_TRAFFIC_BYTES = {"large": None}
+# from the ncu capture summarised in profiles/attn_sm100_kernel_large.md (other workloads: not captured)
+ATTN_TRAFFIC_BYTES = {"large": 790.4e6}
 
 
 def load_peaks():
