@@ -7,6 +7,7 @@ void set_tiles_per_cta(int n);
 void set_exp_emulation(int n);
 void set_prof_buffer(void* p);
 void set_debug_mode(int v);
+int set_wait_limit(long long cycles);
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -188,5 +189,8 @@ void sva_debug_set_exp_emulation(int n) { set_exp_emulation(n); }
 void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); }
 /* tuning aid: bit0 skips the softmax arithmetic (results are wrong; timing of the MMA side only) */
 void sva_debug_set_mode(int v) { set_debug_mode(v); }
+/* test aid: cycles a device-side wait may last before the CTA gives up (<= 0 restores the default);
+   mode bit 16 starves tile 0 of its K tiles so that this limit is reached */
+int sva_debug_set_wait_limit(long long cycles) { return set_wait_limit(cycles); }
 
 }  // extern "C"

@@ -22,6 +22,8 @@ namespace sva {
 
 static constexpr int BS = 128;                 // rows per tile (queries and keys)
 static constexpr long long WAIT_LIMIT_CYCLES = 3000000000LL;
+// cycles a wait may last before the CTA gives up (read only on the slow path of a wait)
+__device__ long long g_wait_limit = WAIT_LIMIT_CYCLES;
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -66,7 +68,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > g_wait_limit) {
         *abort_flag = 1;
         if (status) atomicOr(status, SVA_DEV_TIMEOUT);
         return false;
@@ -364,6 +366,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         int ks = 0;
         uint32_t kphase = 0;
         for (int j = 0; j < n; ++j) {
+          if ((prm.debug & 16) && t == 0 && j >= 1) break;   // test aid: starve the pipeline so that a wait runs out
           if (!mbar_wait(bt + 16 + 8 * ks, kphase ^ 1u, abort_flag, prm.status)) break;
           const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
           const uint32_t dst = sbase + C::OFF_K + (t * C::KS + ks) * C::K_SLOT;
@@ -416,7 +419,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           while (atomicCAS(lock, 0, 1) != 0) {
             if ((++spins & 63u) == 0u) {
               if (*abort_flag) return false;
-              if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+              if (clock64() - t0 > g_wait_limit) {
                 *abort_flag = 1;
                 if (prm.status) atomicOr(prm.status, SVA_DEV_TIMEOUT);
                 return false;
@@ -733,6 +736,10 @@ int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, cons
 void set_tiles_per_cta(int n) { g_tiles_per_cta = n == 1 ? 1 : 2; }
 void set_prof_buffer(void* p) { g_prof = (long long*)p; }
 void set_debug_mode(int v) { g_debug = v; }
+int set_wait_limit(long long cycles) {
+  if (cycles <= 0) cycles = WAIT_LIMIT_CYCLES;
+  return cudaMemcpyToSymbol(g_wait_limit, &cycles, sizeof(cycles)) == cudaSuccess ? 0 : 1;
+}
 void set_exp_emulation(int n) { g_emu = n < 0 ? 0 : (n > 3 ? 3 : n); }
 
 }  // namespace sva

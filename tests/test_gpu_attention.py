@@ -126,3 +126,23 @@ def test_large_logits_need_rescaling():
     rp, ci, _ = U.gpu_select(w, data[0], data[1])
     o, lse, st = U.gpu_attn(w, *data, rp, ci)
     U.check_attn_vs_oracle(w, *bits, rp, ci, o, lse, list(range(w.R)))
+
+
+def test_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Failure detection without faulting the GPU: one tile's K stream is withheld (test switch),
+    the bounded waits expire, the kernel returns with SVA_DEV_TIMEOUT and the next call works."""
+    import ctypes as C
+    w = shrink(WORKLOADS["medium"], H=1, T=2, k=4)        # 16 rows -> 8 CTAs
+    data, bits, rp, ci = _setup(w)
+    L = B.lib()
+    try:
+        assert L.sva_debug_set_wait_limit(C.c_longlong(100_000_000)) == 0     # ~50 ms
+        L.sva_debug_set_mode(16)
+        o, lse, st = U.gpu_attn(w, *data, rp, ci)
+        assert st & B.SVA_DEV_TIMEOUT
+    finally:
+        L.sva_debug_set_mode(0)
+        L.sva_debug_set_wait_limit(C.c_longlong(0))
+    o, lse, st = U.gpu_attn(w, *data, rp, ci)
+    assert st == 0
+    U.check_attn_vs_oracle(w, *bits, rp, ci, o, lse, list(range(w.R)))
