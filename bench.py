@@ -33,9 +33,9 @@ from paper_2606_23743_b200.workloads import SEED_BASE, WORKLOADS, bf16_bits, mak
 METRIC = "block-sparse attn fwd effective TFLOPS (selected blocks)"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the "large" workload,
-# from the ncu capture summarised in profiles/attn_sm100_kernel_large.md (other workloads: not captured)
-ATTN_TRAFFIC_BYTES = {"large": 790.4e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_ts_kernel launch on the "large" workload,
+# from the ncu capture summarised in profiles/attn_ts_kernel_large.md (other workloads: not captured)
+ATTN_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -214,12 +214,13 @@ def main():
     row_ptr = torch.zeros(w.R + 1, dtype=torch.int32, device=dev)
     col_idx = torch.zeros(B.select_max_nnz(p, s), dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    aws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
-    launches_per_step = (4 if variable_rows else 2) + 1
+    launches_per_step = (4 if variable_rows else 2) + 2       # routing kernels + V transpose + attention
 
     def step():
         B.block_select(p, s, q, k, row_ptr, col_idx, ws)
-        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status)
+        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status, workspace=aws)
 
     for _ in range(warmup):
         step()
@@ -242,7 +243,7 @@ def main():
         B.block_select(p, s, q, k, row_ptr, col_idx, ws)
         sel_ev[i][1].record()
         att_ev[i][0].record()
-        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status)
+        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status, workspace=aws)
         att_ev[i][1].record()
     ev1.record()
     torch.cuda.synchronize()
@@ -300,7 +301,10 @@ def main():
         "select_gbs": sel_bytes / (sel_ms * 1e-3) / 1e9,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
-                     "kernel": "attn_sm100_kernel", "peak_source": f"{peak_kind} bf16 burst",
+                     "kernel": "attn_ts_kernel (timed with the V transpose that precedes it in the same call)",
+                     "peak_source": f"{peak_kind} bf16 burst",
+                     "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"])
+                     if "bf16_tflops_sustained" in peaks else None,
                      "frac_of_nominal_2250": achieved / 2250.0},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }

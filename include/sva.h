@@ -22,7 +22,8 @@
  *     unique inside a row.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*), never
  *     synchronise the device and may be issued back to back on one stream.
- *   - The library allocates no device memory; scratch is the caller's `workspace`.
+ *   - The library allocates no device memory; scratch is the caller's `workspace`
+ *     (routing and attention each state their size).
  *   - Every call validates its arguments on the host first and returns a non-zero
  *     sva_status_t WITHOUT launching anything when they are bad.  No exception
  *     crosses the ABI.  Non-finite inputs give undefined (but memory-safe) results.
@@ -138,16 +139,21 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * O is bf16.  A row with an empty list writes zeros and lse = -inf.
  * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
  * (16 for e4m3 Q/K).  Tensor-core kernel: bf16 (or e4m3 x e4m3) MMA, fp32 accumulate.
+ * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The bf16 tensor-core kernel
+ * keeps a tiled, transposed copy of V there (2*B*H*Nb*block*d bytes, rewritten by every call);
+ * the size is 0 -- and the pointer may be NULL -- for the e4m3 variant and for shapes served by
+ * the CUDA-core kernel.
  */
+size_t sva_attn_workspace_bytes(const sva_problem_t* p);
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                               const float* q_scale, const float* k_scale, const int32_t* row_ptr,
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
-                              void* stream);
+                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* The dense fallback: every block kept, no CSR read. */
 int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                        const float* q_scale, const float* k_scale, void* o, float* lse,
-                       int32_t* device_status, void* stream);
+                       int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Diagnostic twin of sva_block_sparse_attn_fwd: the same contract computed by a plain fp32

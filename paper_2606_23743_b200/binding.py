@@ -21,7 +21,7 @@ SVA_DEV_BAD_INDEX, SVA_DEV_TIMEOUT = 1, 2
 EXPORTS = [
     "sva_select_max_nnz", "sva_select_workspace_bytes", "sva_block_select",
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
-    "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc",
+    "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -64,12 +64,15 @@ def lib():
         L.sva_block_select_noalloc.restype = C.c_int
         L.sva_block_select_noalloc.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp,
                                                vp, vp]
-        for name in ("sva_block_sparse_attn_fwd", "sva_block_sparse_attn_fwd_simt"):
-            f = getattr(L, name)
-            f.restype = C.c_int
-            f.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sva_attn_workspace_bytes.restype = C.c_size_t
+        L.sva_attn_workspace_bytes.argtypes = [C.POINTER(Problem)]
+        L.sva_block_sparse_attn_fwd.restype = C.c_int
+        L.sva_block_sparse_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                C.c_size_t, vp]
+        L.sva_block_sparse_attn_fwd_simt.restype = C.c_int
+        L.sva_block_sparse_attn_fwd_simt.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.sva_dense_attn_fwd.restype = C.c_int
-        L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.sva_quantize_qk_fp8.restype = C.c_int
         L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
         L.sva_status_string.restype = C.c_char_p
@@ -143,18 +146,33 @@ def block_select_noalloc(p: Problem, s: Select, q, k, row_ptr, col_idx, q_scale=
         raise SvaError(rc, "sva_block_select_noalloc")
 
 
+def attn_workspace_bytes(p: Problem) -> int:
+    return int(lib().sva_attn_workspace_bytes(C.byref(p)))
+
+
+def _ws_bytes(ws):
+    return ws.numel() * ws.element_size() if ws is not None else 0
+
+
 def block_sparse_attn_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, q_scale=None,
-                          k_scale=None, simt: bool = False) -> None:
-    fn = lib().sva_block_sparse_attn_fwd_simt if simt else lib().sva_block_sparse_attn_fwd
-    rc = fn(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale), _ptr(k_scale), _ptr(row_ptr),
-            _ptr(col_idx), _ptr(o), _ptr(lse), _ptr(status), _stream())
+                          k_scale=None, simt: bool = False, workspace=None) -> None:
+    if simt:
+        rc = lib().sva_block_sparse_attn_fwd_simt(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
+                                                  _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o),
+                                                  _ptr(lse), _ptr(status), _stream())
+    else:
+        rc = lib().sva_block_sparse_attn_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
+                                             _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o), _ptr(lse),
+                                             _ptr(status), _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_fwd")
 
 
-def dense_attn_fwd(p: Problem, q, k, v, o, lse=None, status=None, q_scale=None, k_scale=None) -> None:
+def dense_attn_fwd(p: Problem, q, k, v, o, lse=None, status=None, q_scale=None, k_scale=None,
+                   workspace=None) -> None:
     rc = lib().sva_dense_attn_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale), _ptr(k_scale),
-                                  _ptr(o), _ptr(lse), _ptr(status), _stream())
+                                  _ptr(o), _ptr(lse), _ptr(status), _ptr(workspace), _ws_bytes(workspace),
+                                  _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_dense_attn_fwd")
 

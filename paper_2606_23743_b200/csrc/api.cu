@@ -4,6 +4,9 @@
 namespace sva {
 
 void set_tiles_per_cta(int n);
+void ts_set_prof_buffer(void* p);
+void ts_set_debug_mode(int v);
+int ts_set_wait_limit(long long cycles);
 void set_exp_emulation(int n);
 void set_prof_buffer(void* p);
 void set_debug_mode(int v);
@@ -57,7 +60,8 @@ static int validate_attn(const sva_problem_t* p, const void* q, const void* k, c
   return SVA_OK;
 }
 
-// The tensor-core kernel covers 128-token blocks with d = 128; other supported shapes run on
+// The tensor-core kernels cover 128-token blocks with d = 128 (bf16: the all-TMEM-A kernel, which
+// needs the transposed-V workspace; e4m3 Q/K: the two-tile kernel); other supported shapes run on
 // the CUDA-core kernel.
 static bool use_sm100(const Dims& m) { return m.block == 128 && m.d == 128; }
 
@@ -116,14 +120,25 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
                                (cudaStream_t)stream);
 }
 
+static int g_bf16_kernel = 0;   /* tuning aid: 1 routes bf16 problems to the two-tile SS/TS kernel */
+
+size_t sva_attn_workspace_bytes(const sva_problem_t* p) {
+  if (validate_problem(p)) return 0;
+  Dims m = make_dims(p);
+  return (use_sm100(m) && !m.fp8) ? attn_ts_workspace_bytes(m) : 0;
+}
+
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                               const float* q_scale, const float* k_scale, const int32_t* row_ptr,
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
-                              void* stream) {
+                              void* workspace, size_t workspace_bytes, void* stream) {
   int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
   if (rc) return rc;
   if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
+  if (use_sm100(m) && !m.fp8 && !g_bf16_kernel)
+    return launch_attn_ts(m, p, q, k, v, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
+                          (cudaStream_t)stream);
   if (use_sm100(m))
     return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
                              (cudaStream_t)stream);
@@ -133,10 +148,13 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
 
 int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                        const float* q_scale, const float* k_scale, void* o, float* lse,
-                       int32_t* device_status, void* stream) {
+                       int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
   if (rc) return rc;
   Dims m = make_dims(p);
+  if (use_sm100(m) && !m.fp8 && !g_bf16_kernel)
+    return launch_attn_ts(m, p, q, k, v, nullptr, nullptr, o, lse, device_status, workspace, workspace_bytes,
+                          (cudaStream_t)stream);
   if (use_sm100(m))
     return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status,
                              (cudaStream_t)stream);
@@ -183,14 +201,16 @@ const char* sva_status_string(int status) {
 
 /* bring-up switch (not part of the public header): 1 or 2 query tiles per CTA */
 void sva_debug_set_tiles_per_cta(int n) { set_tiles_per_cta(n); }
+/* tuning aid: 1 sends bf16 problems to the two-tile kernel that otherwise serves e4m3 (A/B timing) */
+void sva_debug_set_bf16_kernel(int v) { g_bf16_kernel = v; }
 /* tuning switch: 0..3 of every 4 exp2 pairs evaluated by a polynomial on the FMA pipe */
 void sva_debug_set_exp_emulation(int n) { set_exp_emulation(n); }
 /* tuning aid: device buffer of 5*8*8 int64 that CTA 64 fills with a clock64 timeline; NULL = off */
-void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); }
+void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); ts_set_prof_buffer(p); }
 /* tuning aid: bit0 skips the softmax arithmetic (results are wrong; timing of the MMA side only) */
-void sva_debug_set_mode(int v) { set_debug_mode(v); }
+void sva_debug_set_mode(int v) { set_debug_mode(v); ts_set_debug_mode(v); }
 /* test aid: cycles a device-side wait may last before the CTA gives up (<= 0 restores the default);
    mode bit 16 starves tile 0 of its K tiles so that this limit is reached */
-int sva_debug_set_wait_limit(long long cycles) { return set_wait_limit(cycles); }
+int sva_debug_set_wait_limit(long long cycles) { return set_wait_limit(cycles) | ts_set_wait_limit(cycles); }
 
 }  // extern "C"

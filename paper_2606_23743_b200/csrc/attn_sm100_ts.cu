@@ -1,0 +1,667 @@
+// Block-sparse / dense attention forward for sm_100a, bf16 path: every MMA of one kind.
+// (Paper: critical blocks "computed exactly"; dense fallback.)
+//
+// The tensor pipe drains (~280 cycles, measured) whenever two consecutive MMAs differ in kind:
+// A operand from shared memory vs tensor memory, or another instruction descriptor.  Here both
+// S = Q K^T and O += P V have the same form -- A from TENSOR memory (Q resp. P, bf16 pairs), B
+// from shared memory, K-major, M = N = 128 -- so the pipe never drains:
+//   * Q is written into TMEM once per row by the softmax threads (straight from global memory);
+//   * V is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed copy
+//     that a small kernel writes into the caller's workspace first.
+// The kernel is persistent: CTA c processes the CSR rows c, c + gridDim.x, ... (one row = one query
+// block of one head, 128 query rows).  All barriers keep running across rows (every role derives the
+// same phase counters from the same row sequence), so the producers run ahead into the next row
+// while the softmax groups finish the current one.
+//   warps 0-3, 4-7  two softmax warpgroups; they take the kept key blocks alternately (even / odd
+//                   position in the row's list); thread <-> query row <-> TMEM lane
+//   warp  8         producer of the K tiles (TMA, one lane)
+//   warp  9         issues the Q K^T MMAs (one lane); owns the TMEM allocation
+//   warp  10        issues the P V MMAs (one lane)
+//   warp  11        producer of the V^T tiles (TMA, one lane)
+// TMEM columns: S of even blocks 0..127, S of odd blocks 128..255, O 256..383, Q 384..447 (bf16
+// pairs), P 448..511 (bf16 pairs).  Because P has columns of its own, an S buffer is free again as
+// soon as its warpgroup has read it into registers: the MMA warp computes S(j+2) while the softmax
+// of block j is still running.  P is single-buffered: block j's P is stored once P V(j-1) has
+// completed, which also staggers the two warpgroups so that one group's exponentials overlap the
+// other group's maximum pass and stores.
+//
+// The two warpgroups share one O accumulator, so they share the reference exponent of every row:
+// the group working on block j takes the reference left by block j-1 (published through shared
+// memory right after that block's row-maximum pass), raises it only when the new row maximum
+// exceeds it by more than 2^LAZY_LOG2, and in that (rare) case rescales its row of O once P V(j-1)
+// has completed.  Row sums are kept per group and merged in the epilogue, where each group
+// normalises its half of O into a swizzled staging panel that one TMA tile store writes out.
+//
+// Every wait is bounded: when one expires the CTA sets SVA_DEV_TIMEOUT, all roles leave their
+// loops, TMEM is released and the kernel returns.  Parity waits never run a whole phase ahead of
+// their barrier (each wait on a barrier is preceded by a wait on its previous phase).
+#include "tc_ptx.cuh"
+
+namespace sva {
+
+struct TsParams {
+  const __nv_bfloat16* q;
+  Strides sq;
+  const int32_t* row_ptr;     // null = dense
+  const int32_t* col_idx;
+  __nv_bfloat16* o;
+  float* lse;
+  int32_t* status;
+  Strides so;
+  int H, N, Nb, R;
+  float scale_log2;           // softmax_scale * log2(e)
+  long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
+  int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
+                              // bit4: starve the pipeline so that a wait runs out (test aid)
+};
+
+namespace ts {
+constexpr int D = 128;
+constexpr int TILE = BS * D * 2;            // one bf16 tile: 32 KB
+constexpr int KS = 2;                       // K tiles in flight
+constexpr int VS = 3;                       // V^T tiles in flight
+constexpr int THREADS = 384;
+constexpr int OFF_K = 0;
+constexpr int OFF_V = OFF_K + KS * TILE;
+constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][128 B] panels (one per softmax group)
+constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
+constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4;   // barriers, reference exponents, row sums (two rows)
+constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;      // + alignment slack
+constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
+// The reference exponent of a row is raised only when a block's maximum exceeds it by more than this
+// many powers of two.  P then reaches at most 2^32 and a row sum 2^32 * N: far inside fp32 (and bf16
+// has fp32's exponent range), while raises -- each one a pass over the row's O accumulator -- become rare.
+constexpr float LAZY_LOG2 = 32.0f;
+}  // namespace ts
+
+// control block (bytes from OFF_CTRL):
+//   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
+//   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
+//   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
+
+// Kept-block list of CSR row r: count and start.  A corrupt row_ptr pair gives an empty row; every
+// role calls this with the same inputs and so reaches the same answer.
+__device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int& beg) {
+  if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return; }
+  beg = __ldg(prm.row_ptr + r);
+  n = __ldg(prm.row_ptr + r + 1) - beg;
+  if (n < 0 || n > prm.Nb || beg < 0) n = 0;
+}
+// Key block of list entry j; an out-of-range entry is replaced by block 0 (the producer reports it).
+__device__ __forceinline__ int list_block(const TsParams& prm, int beg, int j) {
+  if (prm.row_ptr == nullptr) return j;
+  const int J = __ldg(prm.col_idx + beg + j);
+  return (J < 0 || J >= prm.Nb) ? 0 : J;
+}
+
+// Persistent kernel: CTA c processes the CSR rows c, c + gridDim.x, ...  All barriers keep running
+// across rows (every role derives the same phase counters from the same row sequence), so the
+// producers and the S issuer run ahead into the next row while the softmax groups finish the
+// current one, and a row's epilogue overlaps the next row's first MMAs.
+__global__ void __launch_bounds__(384, 1)
+attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
+               const __grid_constant__ CUtensorMap tm_o, const TsParams prm) {
+  using namespace ts;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  uint8_t* ctrl = smem + OFF_CTRL;
+  const uint32_t cb = sbase + OFF_CTRL;
+  const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
+                 bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
+                 bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
+                 bar_ost = cb + 224;
+  volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
+  volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
+  volatile float* lx = reinterpret_cast<volatile float*>(ctrl + 1280);      // [2][2][128]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int Nb = prm.Nb;
+
+  // ---------------------------------------------------------------- set-up
+  const long long t_cta0 = prm.prof ? clock64() : 0;
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q_ready, 256);
+    mbar_init(bar_o_free, 256);
+    mbar_init(bar_xch, 256);
+    for (int w = 0; w < 2; ++w) {
+      mbar_init(bar_s_full + 8 * w, 1);
+      mbar_init(bar_p_full + 8 * w, 128);
+      mbar_init(bar_pv_done + 8 * w, 1);
+      mbar_init(bar_ref + 8 * w, 128);
+      mbar_init(bar_s_free + 8 * w, 128);
+      mbar_init(bar_ost + 8 * w, 128);
+    }
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(bar_k_full + 8 * s, 1);
+      mbar_init(bar_k_empty + 8 * s, 1);
+      mbar_init(bar_v_full + 8 * s, 1);
+      mbar_init(bar_v_empty + 8 * s, 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 8 && lane == 0) prefetch_tmap(&tm_k);
+  if (warp == 11 && lane == 0) prefetch_tmap(&tm_vt);
+  if (warp == 0 && lane == 0) prefetch_tmap(&tm_o);
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(cb + 216), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_p;
+  constexpr uint32_t IDESC = instr_desc(128, 128, 1, false);   // bf16 x bf16 -> fp32, A and B K-major
+  constexpr int PANEL16 = (BS * 128) >> 4;                      // one 128-row x 128-byte panel
+
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
+    if (warp == 8) {
+      // ---------------------------------------------------------- K producer (one lane)
+      if (lane == 0) {
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
+          int n, beg;
+          row_list(prm, r, n, beg);
+          const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          for (int j = 0; j < n; ++j) {
+            if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
+            if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+            int J = j;
+            if (prm.row_ptr) {
+              J = __ldg(prm.col_idx + beg + j);
+              if (J < 0 || J >= Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
+            }
+            const uint32_t dst = sbase + OFF_K + s * TILE;
+            mbar_expect_tx(bar_k_full + 8 * s, TILE);
+            tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);
+            tma_load_4d(dst + TILE / 2, &tm_k, bar_k_full + 8 * s, 64, J * BS, hh, bb);
+            if (++s == KS) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    } else if (warp == 11) {
+      // ---------------------------------------------------------- V^T producer (one lane)
+      // tile J of head (b,h): 128 d-rows x 128 keys, contiguous 32 KB, two 64-key panels
+      if (lane == 0) {
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
+          int n, beg;
+          row_list(prm, r, n, beg);
+          const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          for (int j = 0; j < n; ++j) {
+            if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+            const int J = list_block(prm, beg, j);
+            const uint32_t dst = sbase + OFF_V + s * TILE;
+            mbar_expect_tx(bar_v_full + 8 * s, TILE);
+            tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, J * BS, hh, bb);
+            tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, J * BS, hh, bb);
+            if (++s == VS) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    } else if (warp == 9) {
+      // ---------------------------------------------------------- S issuer (one lane)
+      // per row: S(0), S(1), then S(j) into the buffer of S(j-2) as soon as that block's softmax
+      // has read it; the first S of a row also needs the row's Q in TMEM
+      if (lane == 0) {
+        const uint64_t kd0 = smem_desc(sbase + OFF_K, 16, 1024);
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t cs[2] = {0, 0};            // S tiles issued so far into buffer w
+        uint32_t rows_done = 0;             // non-empty rows started so far
+        bool ok = true;
+        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
+          int n, beg;
+          row_list(prm, r, n, beg);
+          if (n == 0) continue;
+          ok = mbar_wait(bar_q_ready, rows_done & 1u, abort_flag, prm.status);
+          ++rows_done;
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            if (cs[w] > 0) {
+              ok = mbar_wait(bar_s_free + 8 * w, (cs[w] - 1u) & 1u, abort_flag, prm.status);
+              if (!ok) break;
+            }
+            ok = mbar_wait(bar_k_full + 8 * s, ph, abort_flag, prm.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t kd = kd0 + (uint64_t)(s * (TILE >> 4));
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+              tc_mma_ts(tmem_base + 128 * w, tmem_base + COL_Q + 8 * kk, kd + off, IDESC, kk > 0 ? 1u : 0u, 1u);
+            }
+            tc_commit(bar_k_empty + 8 * s, 1u);
+            tc_commit(bar_s_full + 8 * w, 1u);
+            ++cs[w];
+            if (++s == KS) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    } else {
+      // ---------------------------------------------------------- P V issuer (one lane)
+      if (lane == 0) {
+        const uint64_t vd0 = smem_desc(sbase + OFF_V, 16, 1024);
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t cp[2] = {0, 0};            // P V groups issued so far for parity w
+        uint32_t rows_done = 0;
+        bool ok = true;
+        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
+          int n, beg;
+          row_list(prm, r, n, beg);
+          if (n == 0) continue;
+          // the first P V of a row overwrites O: the previous row's O must have been read
+          if (rows_done > 0) ok = mbar_wait(bar_o_free, (rows_done - 1u) & 1u, abort_flag, prm.status);
+          ++rows_done;
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            const uint64_t vd = vd0 + (uint64_t)(s * (TILE >> 4));
+            ok = mbar_wait(bar_p_full + 8 * w, cp[w] & 1u, abort_flag, prm.status) &&
+                 mbar_wait(bar_v_full + 8 * s, ph, abort_flag, prm.status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < BS / 16; ++kk) {
+              const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+              tc_mma_ts(tmem_base + COL_O, tmem_base + COL_P + 8 * kk, vd + off, IDESC, (j > 0 || kk > 0) ? 1u : 0u, 1u);
+            }
+            tc_commit(bar_v_empty + 8 * s, 1u);
+            tc_commit(bar_pv_done + 8 * w, 1u);
+            if (!ok) break;
+            ++cp[w];
+            if (++s == VS) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+    const int w = warp >> 2;                                 // this group takes blocks j = w, w+2, ... of a row
+    const int row = (warp & 3) * 32 + lane;                  // query row of the tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t s_tmem = tmem_base + lane_addr + 128 * w;
+    const uint32_t o_tmem = tmem_base + lane_addr + COL_O;
+    const uint32_t p_tmem = tmem_base + lane_addr + COL_P;
+    const uint32_t q_tmem = tmem_base + lane_addr + COL_Q + 32 * w;
+    const int tail_keys = prm.N - (Nb - 1) * BS;             // valid keys of the last block
+    const float c = prm.scale_log2;
+    uint32_t cnt[2] = {0, 0};      // blocks of parity 0 / 1 completed in earlier rows (barrier phase bases)
+    uint32_t rows_done = 0;        // non-empty rows finished
+    bool ok = true;
+
+    // this group's half (d columns 64w..64w+63) of a row's Q: global -> registers -> TMEM
+    auto load_q = [&](int r, uint32_t* qv) {
+#pragma unroll
+      for (int e = 0; e < 32; ++e) qv[e] = 0u;
+      if (r >= prm.R) return;
+      const int bh = r / Nb, qi = (r % Nb) * BS + row;
+      if (qi >= prm.N) return;
+      const uint4* src = reinterpret_cast<const uint4*>(prm.q + (long long)(bh / prm.H) * prm.sq.b +
+                                                        (long long)(bh % prm.H) * prm.sq.h + (long long)qi * prm.sq.n + 64 * w);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint4 u = __ldg(src + e);
+        qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
+      }
+    };
+    auto next_row = [&](int r) {                              // next non-empty row of this CTA (or >= R)
+      for (r += gridDim.x; r < prm.R; r += gridDim.x) {
+        int n, beg;
+        row_list(prm, r, n, beg);
+        if (n > 0) return r;
+      }
+      return prm.R;
+    };
+    auto store_q = [&](const uint32_t* qv) {
+      tmem_st32(q_tmem, qv);
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_q_ready);
+    };
+
+    // first non-empty row: its Q goes in right away
+    int r_first = (int)blockIdx.x - (int)gridDim.x;
+    r_first = next_row(r_first);
+    {
+      uint32_t qv[32];
+      load_q(r_first, qv);
+      if (r_first < prm.R) store_q(qv);
+    }
+
+    // The list of the row after this one (count, start, first entry of this group) is loaded one row
+    // ahead, so that no global-memory latency sits between two rows.
+    int n_c = 0, beg_c = 0, J_c = 0;
+    if ((int)blockIdx.x < prm.R) {
+      row_list(prm, blockIdx.x, n_c, beg_c);
+      if (w < n_c) J_c = list_block(prm, beg_c, w);
+    }
+    for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
+      const int n = n_c, lbeg = beg_c;
+      int J = J_c;
+      const int r_c = r + gridDim.x;
+      n_c = 0;
+      if (r_c < prm.R) row_list(prm, r_c, n_c, beg_c);                // consumed in this row's last block
+      const int I = r % Nb, bh = r / Nb;
+      const int hh = bh % prm.H, bb = bh / prm.H;
+      const int qi = I * BS + row;
+      __nv_bfloat16* orow = prm.o + (long long)bb * prm.so.b + (long long)hh * prm.so.h + (long long)qi * prm.so.n;
+      if (n == 0) {
+        if (qi < prm.N) {
+#pragma unroll
+          for (int cc = 0; cc < D / 2; cc += 8) *reinterpret_cast<uint4*>(orow + (D / 2) * w + cc) = make_uint4(0, 0, 0, 0);
+          if (prm.lse && w == 0) prm.lse[(long long)bh * prm.N + qi] = -INFINITY;
+        }
+        if (w < n_c) J_c = list_block(prm, beg_c, w);
+        continue;
+      }
+      const int wl = (n - 1) & 1;                                     // group that takes the row's last block
+      const uint32_t last = cnt[wl] + (uint32_t)((n - 1) >> 1);       // phase index of that block
+      float m_mine = -INFINITY;      // reference exponent my partial row sum is relative to
+      float l = 0.f;                 // partial row sum over this group's blocks
+      for (int j = w; j < n; j += 2) {
+        const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
+        const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
+        const int valid = (J == Nb - 1) ? tail_keys : BS;
+        if (j + 2 < n) J = list_block(prm, lbeg, j + 2);               // one block ahead
+        if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t sv[128];
+        tmem_ld32(s_tmem + 0, sv + 0);
+        tmem_ld32(s_tmem + 32, sv + 32);
+        tmem_ld32(s_tmem + 64, sv + 64);
+        tmem_ld32(s_tmem + 96, sv + 96);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
+        if (valid < BS) {
+#pragma unroll
+          for (int e = 0; e < 128; ++e)
+            if (e >= valid) sv[e] = 0xff800000u;              // keys that do not exist: -inf
+        }
+        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 128; e += 8) {
+          mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+          mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+          mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
+          mxd = max3(mxd, __uint_as_float(sv[e + 6]), __uint_as_float(sv[e + 7]));
+        }
+        const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd)) * c;
+        // reference exponent left by block j-1 (other group)
+        float m_prev = -INFINITY;
+        if (j > 0) {
+          if (!mbar_wait(bar_ref + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          m_prev = ref[(w ^ 1) * 128 + row];
+        }
+        // lazy rule: raise the reference only when the row maximum outgrows it by more than 2^LAZY_LOG2
+        const float m_new = (mx > m_prev + LAZY_LOG2) ? mx : m_prev;
+        ref[w * 128 + row] = m_new;
+        mbar_arrive(bar_ref + 8 * w);
+        if (m_new != m_mine) { l *= ex2(m_mine - m_new); m_mine = m_new; }      // first block: 0 * 2^-inf
+        bool pv_waited = false;
+        if (j > 0 && __any_sync(0xffffffffu, m_new != m_prev)) {
+          // rescale this row of O once P V(j-1) has completed (O is then quiescent: P V(j) waits for us)
+          if (!mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          pv_waited = true;
+          tc_fence_after();
+          const float alpha = ex2(m_prev - m_new);
+#pragma unroll 1
+          for (int cc = 0; cc < D; cc += 16) {
+            uint32_t ov[16];
+            tmem_ld16(o_tmem + cc, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+            tmem_st16(o_tmem + cc, ov);
+          }
+          tc_wait_st();
+        }
+        // P = 2^(S*c - m); the packed bf16 pairs overwrite sv[0..63]
+        const float nm = -m_new;
+        float sum_a = 0.f, sum_b = 0.f;
+        if (!(prm.debug & 1)) {
+#pragma unroll
+          for (int e = 0; e < 128; e += 2) {
+            const float x0 = fmaf(__uint_as_float(sv[e]), c, nm), x1 = fmaf(__uint_as_float(sv[e + 1]), c, nm);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            sum_a += p0;
+            sum_b += p1;
+            sv[e / 2] = pack_bf16(p0, p1);
+          }
+        }
+        l += sum_a + sum_b;
+        // the P columns are free once P V(j-1) has completed (block 0: the previous row's last P V
+        // was waited for in that row's epilogue)
+        if (j > 0 && !pv_waited &&
+            !mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st32(p_tmem, sv);
+        tmem_st32(p_tmem + 32, sv + 32);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p_full + 8 * w);
+      }
+      if (!ok) break;
+      // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
+      // normalise and store (each group half of d)
+      const int r_next = (n_c > 0 || r_c >= prm.R) ? r_c : next_row(r_c);   // next non-empty row of this CTA
+      if (w < n_c) J_c = list_block(prm, beg_c, w);
+      uint32_t qn[32];
+      load_q(r_next, qn);                                             // in flight during the waits below
+      if (!mbar_wait(bar_ref + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+      const float m_fin = ref[wl * 128 + row];
+      if (m_mine != m_fin) { l *= ex2(m_mine - m_fin); m_mine = m_fin; }        // l = 0 for a group without blocks
+      volatile float* lxr = lx + (rows_done & 1u) * 256;
+      lxr[w * 128 + row] = l;
+      if ((threadIdx.x & 127) == 0) bulk_wait_read0();                // the previous row's store has read the staging panel
+      mbar_arrive(bar_xch);
+      if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
+      // both groups have seen all their S tiles: no MMA reads Q any more
+      if (r_next < prm.R) store_q(qn);
+      if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+      tc_fence_after();
+      const float lt = l + lxr[(w ^ 1) * 128 + row];
+      const float inv = 1.0f / lt;
+      {
+        uint32_t ov[64];
+        tmem_ld32(o_tmem + (D / 2) * w, ov);
+        tmem_ld32(o_tmem + (D / 2) * w + 32, ov + 32);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_o_free);                                      // the next row may overwrite O
+        // normalised bf16 row -> this group's staging panel (128-byte swizzle), then one tile store;
+        // rows beyond N are clipped by the tensor map
+        uint8_t* stg = smem + OFF_O + w * (TILE / 2) + row * 128;
+#pragma unroll
+        for (int e = 0; e < 64; e += 8) {
+          uint4 v4;
+          v4.x = pack_bf16(__uint_as_float(ov[e + 0]) * inv, __uint_as_float(ov[e + 1]) * inv);
+          v4.y = pack_bf16(__uint_as_float(ov[e + 2]) * inv, __uint_as_float(ov[e + 3]) * inv);
+          v4.z = pack_bf16(__uint_as_float(ov[e + 4]) * inv, __uint_as_float(ov[e + 5]) * inv);
+          v4.w = pack_bf16(__uint_as_float(ov[e + 6]) * inv, __uint_as_float(ov[e + 7]) * inv);
+          *reinterpret_cast<uint4*>(stg + (((e >> 3) ^ (row & 7)) << 4)) = v4;
+        }
+        fence_async_smem();
+        mbar_arrive(bar_ost + 8 * w);
+        if ((threadIdx.x & 127) == 0) {
+          // (a wait that runs out has raised the abort flag; the other threads leave at their next wait)
+          if (mbar_wait(bar_ost + 8 * w, rows_done & 1u, abort_flag, prm.status)) {
+            tma_store_4d(&tm_o, sbase + OFF_O + w * (TILE / 2), (D / 2) * w, I * BS, hh, bb);
+            bulk_commit();
+          }
+        }
+        if (qi < prm.N && prm.lse && w == 0) prm.lse[(long long)bh * prm.N + qi] = (m_fin + log2f(lt)) * 0.6931471805599453f;
+      }
+      cnt[0] += (uint32_t)((n + 1) >> 1);
+      cnt[1] += (uint32_t)(n >> 1);
+      ++rows_done;
+    }
+    if ((threadIdx.x & 127) == 0) bulk_wait0();                       // my output stores have completed
+  }
+
+  // ---------------------------------------------------------------- tear-down
+  if (prm.prof && threadIdx.x == 0)
+    atomicMax(reinterpret_cast<unsigned long long*>(prm.prof + 319), (unsigned long long)(clock64() - t_cta0));
+  if (*abort_flag) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ V^T
+// V [B,H,N,d] (strided) -> tiled transposed copy: for every (b,h) and key block J one contiguous
+// 32 KB tile [d = 128 rows][128 keys], keys >= N zero.  A tile is then one contiguous TMA box pair,
+// exactly like a K tile.
+__global__ void __launch_bounds__(256)
+transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
+                   int Nb, int d) {
+  __shared__ __nv_bfloat16 tile[64][66];            // [d][key], padded
+  const int n0 = blockIdx.x * 64, d0 = blockIdx.y * 64, bh = blockIdx.z;
+  const int b = bh / H, h = bh % H;
+  const __nv_bfloat16* src = v + (long long)b * sv.b + (long long)h * sv.h;
+  {
+    const int c8 = threadIdx.x & 7;                 // 8 d-values (16 bytes)
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int key = (threadIdx.x >> 3) + 32 * pass;
+      uint4 u = make_uint4(0, 0, 0, 0);
+      if (n0 + key < N) u = __ldg(reinterpret_cast<const uint4*>(src + (long long)(n0 + key) * sv.n + d0) + c8);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&u);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) tile[c8 * 8 + q][key] = e[q];
+    }
+  }
+  __syncthreads();
+  {
+    const int k8 = threadIdx.x & 7;                 // 8 keys (16 bytes)
+    const int J = n0 / BS, kin = (n0 % BS) + k8 * 8;
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int dd = (threadIdx.x >> 3) + 32 * pass;
+      __align__(16) __nv_bfloat16 e[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) e[q] = tile[dd][k8 * 8 + q];
+      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * d + d0 + dd) * BS + kin) = *reinterpret_cast<uint4*>(e);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                CUtensorMapFloatOOBfill);
+
+static encode_fn_t get_encode_ts() {
+  static encode_fn_t fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<encode_fn_t>(p);
+  }
+  return fn;
+}
+
+// bf16 4-D map (inner, rows, H, B) with byte strides; box = 64 x 128 (128 bytes x 128 rows), 128-byte swizzle.
+static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuuint64_t rows, int H, int B,
+                       cuuint64_t row_stride, cuuint64_t h_stride, cuuint64_t b_stride) {
+  encode_fn_t enc = get_encode_ts();
+  if (!enc) return SVA_ERR_CUDA;
+  cuuint64_t dims[4] = {inner, rows, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {row_stride, h_stride, b_stride};
+  // a size-1 dimension may carry any stride; give it a legal one
+  if (H == 1) strides[1] = strides[0] * rows;
+  if (B == 1) strides[2] = strides[1] * (cuuint64_t)H;
+  for (int i = 0; i < 3; ++i)
+    if (strides[i] % 16 != 0 || strides[i] == 0) return SVA_ERR_ALIGNMENT;
+  cuuint32_t box[4] = {64, (cuuint32_t)BS, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult rc = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? SVA_OK : SVA_ERR_CUDA;
+}
+
+static long long* g_prof_ts = nullptr;
+static int g_debug_ts = 0;
+
+static int launch_ts(const Dims& m, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                     const TsParams& prm,
+                     cudaStream_t st) {
+  auto kern = attn_ts_kernel;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
+    return SVA_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return SVA_ERR_CUDA;
+  const int grid = m.R < sms ? m.R : sms;          // persistent: one CTA per SM, rows round-robin
+  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, prm);
+  return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
+}
+
+size_t attn_ts_workspace_bytes(const Dims& m) {
+  return (size_t)m.B * m.H * m.Nb * BS * m.d * 2;        // one transposed V tile per (b, h, key block)
+}
+
+int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
+                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                   void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (m.block != BS || m.d != 128 || m.fp8) return SVA_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < attn_ts_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
+  const Strides sk = make_strides(p->k_stride), sv = make_strides(p->v_stride);
+  const Strides so = make_strides(p->o_stride);
+  CUtensorMap tk, tv, to;
+  int rc;
+  if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2)) != SVA_OK)
+    return rc;
+  if ((rc = make_map_ts(&tk, k, m.d, m.N, m.H, m.B, (cuuint64_t)sk.n * 2, (cuuint64_t)sk.h * 2, (cuuint64_t)sk.b * 2)) != SVA_OK)
+    return rc;
+  // transposed V: per (b,h) a [Nb*128 rows][128 keys] matrix, tile J = rows J*128 .. J*128+127
+  const cuuint64_t vrows = (cuuint64_t)m.Nb * m.d;
+  if ((rc = make_map_ts(&tv, ws, BS, vrows, m.H, m.B, (cuuint64_t)BS * 2, vrows * BS * 2, vrows * BS * 2 * m.H)) != SVA_OK)
+    return rc;
+  dim3 tg(m.Nb * 2, m.d / 64, m.B * m.H);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d);
+  TsParams prm;
+  prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
+  prm.row_ptr = row_ptr; prm.col_idx = col_idx;
+  prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
+  prm.so = make_strides(p->o_stride);
+  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
+  prm.scale_log2 = m.scale * 1.4426950408889634f;
+  prm.prof = g_prof_ts;
+  prm.debug = g_debug_ts;
+  return launch_ts(m, tk, tv, to, prm, st);
+}
+
+void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }
+void ts_set_debug_mode(int v) { g_debug_ts = v; }
+int ts_set_wait_limit(long long cycles) {
+  if (cycles <= 0) cycles = WAIT_LIMIT_CYCLES;
+  return cudaMemcpyToSymbol(g_wait_limit, &cycles, sizeof(cycles)) == cudaSuccess ? 0 : 1;
+}
+
+}  // namespace sva

@@ -60,4 +60,9 @@ int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, cons
                       const int32_t* col_idx, void* o, float* lse, int32_t* status,
                       cudaStream_t st);
 
+int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
+                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                   void* ws, size_t ws_bytes, cudaStream_t st);
+size_t attn_ts_workspace_bytes(const Dims& m);
+
 }  // namespace sva

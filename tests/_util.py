@@ -69,11 +69,12 @@ def gpu_attn(w: Workload, q, k, v, row_ptr, col_idx, N=None, simt=False, dense=F
     lse = torch.full((q.shape[0], q.shape[1], N), 7.0, dtype=torch.float32, device="cuda") if want_lse else None
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(q, k, v, o, N, w.block, 0.0, fp8)
+    ws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device="cuda")
     if dense and not simt:
-        B.dense_attn_fwd(p, q, k, v, o, lse, status, q_scale, k_scale)
+        B.dense_attn_fwd(p, q, k, v, o, lse, status, q_scale, k_scale, workspace=ws)
     else:
         B.block_sparse_attn_fwd(p, q, k, v, None if dense else row_ptr, None if dense else col_idx, o, lse,
-                                status, q_scale, k_scale, simt=simt)
+                                status, q_scale, k_scale, simt=simt, workspace=ws)
     torch.cuda.synchronize()
     return o, lse, int(status.item())
 

@@ -84,13 +84,17 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert sel(bad, s) == 5
 
     def att(p, q=one, k=one, v=one, o=one, rp=one, ci=one):
-        return lib.sva_block_sparse_attn_fwd(C.byref(p), q, k, v, None, None, rp, ci, o, None, None, None)
+        return lib.sva_block_sparse_attn_fwd(C.byref(p), q, k, v, None, None, rp, ci, o, None, None, None, 0, None)
     assert att(_problem(d=96)) == 2
     assert att(p, v=None) == 1
     assert att(p, rp=None) == 1
     assert att(p, o=vp(4)) == 5
     assert att(_problem(qk_dtype=7)) == 1
-    assert lib.sva_dense_attn_fwd(C.byref(p), one, one, None, None, None, one, None, None, None) == 1
+    assert lib.sva_dense_attn_fwd(C.byref(p), one, one, None, None, None, one, None, None, None, 0, None) == 1
+    assert B.attn_workspace_bytes(p) == 1 * 2 * 8 * 128 * 128 * 2       # transposed V tiles
+    assert B.attn_workspace_bytes(_problem(block=64)) == 0               # CUDA-core kernel needs none
+    assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 0             # e4m3 variant needs none
+    assert att(p) == 3                                                   # bf16 tensor-core path without workspace
     assert lib.sva_quantize_qk_fp8(C.byref(p), one, one, one, None, one, one, None) == 1
     bad = _problem(); bad.k_stride = (C.c_int64 * 3)(0, 0, 136)
     assert lib.sva_quantize_qk_fp8(C.byref(bad), one, one, one, one, one, one, None) == 5
