@@ -376,6 +376,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (j + 2 < n) J = list_block(prm, lbeg, j + 2);               // one block ahead
         if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
         tc_fence_after();
+        if (valid < BS) {
+          // ragged last key block: keys that do not exist become -inf in TMEM before S is read (a short
+          // rolled loop -- this keeps 128 compare/select pairs out of the hot instruction stream)
+#pragma unroll 1
+          for (int e = valid; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+          tc_wait_st();
+        }
         uint32_t sv[128];
         tmem_ld32(s_tmem + 0, sv + 0);
         tmem_ld32(s_tmem + 32, sv + 32);
@@ -384,11 +391,6 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
-        if (valid < BS) {
-#pragma unroll
-          for (int e = 0; e < 128; ++e)
-            if (e >= valid) sv[e] = 0xff800000u;              // keys that do not exist: -inf
-        }
         float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 128; e += 8) {

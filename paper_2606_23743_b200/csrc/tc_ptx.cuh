@@ -147,6 +147,9 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
       ::SVA_I4(v, 0), SVA_I4(v, 4), SVA_I4(v, 8), SVA_I4(v, 12), SVA_I4(v, 16), SVA_I4(v, 20),
         SVA_I4(v, 24), SVA_I4(v, 28), "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t v) {       // one column of this warp's 32 lanes
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(v) : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
