@@ -431,18 +431,23 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         // P = 2^(S*c - m); the packed bf16 pairs overwrite sv[0..63]
         const float nm = -m_new;
-        float sum_a = 0.f, sum_b = 0.f;
+        const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
+        uint64_t sum2 = pack2(0.f, 0.f);
         if (!(prm.debug & 1)) {
 #pragma unroll
           for (int e = 0; e < 128; e += 2) {
-            const float x0 = fmaf(__uint_as_float(sv[e]), c, nm), x1 = fmaf(__uint_as_float(sv[e + 1]), c, nm);
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, nm2), x0, x1);
             const float p0 = ex2(x0), p1 = ex2(x1);
-            sum_a += p0;
-            sum_b += p1;
+            sum2 = add2(sum2, pack2(p0, p1));
             sv[e / 2] = pack_bf16(p0, p1);
           }
         }
-        l += sum_a + sum_b;
+        {
+          float sum_a, sum_b;
+          unpack2(sum2, sum_a, sum_b);
+          l += sum_a + sum_b;
+        }
         // the P columns are free once P V(j-1) has completed (block 0: the previous row's last P V
         // was waited for in that row's epilogue)
         if (j > 0 && !pv_waited &&

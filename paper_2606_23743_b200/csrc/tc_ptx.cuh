@@ -47,12 +47,13 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {  
   return ok;
 }
 // Bounded wait.  Returns false when the CTA is aborting.  SLEEP_NS > 0 backs off between polls
-// (for roles whose wake-up latency is not on the critical path) so that the polling does not
-// take issue slots from the softmax warps of the same scheduler.
+// (for roles whose wake-up latency is not on the critical path).  The first poll is marked as the
+// likely exit so that the polling loop is laid out away from the hot instruction stream
+// (instruction fetch is a measurable cost in these kernels).
 template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (__builtin_expect(mbar_try_wait(bar, parity) != 0u, 1)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
@@ -162,6 +163,25 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// two fp32 lanes in one instruction (sm_100): d = a * b + c, d = a + b
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float y;
