@@ -334,6 +334,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           l = 1.f;
           continue;
         }
+        if (valid < BS) {
+          // ragged last key block: keys that do not exist become -inf in TMEM before S is read (a short
+          // rolled loop -- this keeps 128 compare/select pairs out of the hot instruction stream)
+#pragma unroll 1
+          for (int i = valid; i < BS; ++i) tmem_st1(s_tmem + i, 0xff800000u);
+          tc_wait_st();
+        }
         // ---- row maximum over the 128 columns (whole row in registers)
         uint32_t sv[128];
         tmem_ld32(s_tmem + 0, sv + 0);
@@ -342,11 +349,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tmem_ld32(s_tmem + 96, sv + 96);
         tc_wait_ld();
         if (probe) SVA_PROF(t, j, 2);
-        if (valid < BS) {
-#pragma unroll
-          for (int i = 0; i < 128; ++i)
-            if (i >= valid) sv[i] = 0xff800000u;              // keys that do not exist: -inf
-        }
         float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 128; i += 8) {
