@@ -28,8 +28,8 @@
  *     sva_status_t WITHOUT launching anything when they are bad.  No exception
  *     crosses the ABI.  Non-finite inputs give undefined (but memory-safe) results.
  *   - `device_status` (optional, device int32, zero it before the call): kernels OR
- *     SVA_DEV_* bits into it instead of trapping (a bad CSR entry is skipped, a
- *     pipeline wait that ran out gives up and the block exits).
+ *     SVA_DEV_* bits into it instead of trapping (a bad CSR entry is never used as an
+ *     address, a pipeline wait that ran out gives up and the block exits).
  */
 #ifndef SVA_H_
 #define SVA_H_
@@ -52,7 +52,9 @@ typedef enum {
 } sva_status_t;
 
 /* bits a kernel may set in *device_status */
-#define SVA_DEV_BAD_INDEX 1  /* CSR entry outside [0,Nb) or row_ptr not monotone: skipped */
+#define SVA_DEV_BAD_INDEX 1  /* CSR entry outside [0,Nb) or row_ptr not monotone: never dereferenced (the entry is
+                                skipped, replaced by block 0 or its row treated as empty, depending on the kernel);
+                                the affected rows' output is not meaningful */
 #define SVA_DEV_TIMEOUT   2  /* a bounded pipeline wait expired; output of that block is undefined */
 
 typedef enum { SVA_BF16 = 0, SVA_FP8_E4M3 = 1 } sva_qk_dtype_t;
