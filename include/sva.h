@@ -142,7 +142,8 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
  * (16 for e4m3 Q/K).  Tensor-core kernel: bf16 (or e4m3 x e4m3) MMA, fp32 accumulate.
  * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The bf16 tensor-core kernel
- * keeps a tiled, transposed copy of V there (2*B*H*Nb*block*d bytes, rewritten by every call);
+ * keeps a tiled, transposed copy of V (2*B*H*Nb*block*d bytes) and its row counter there, both
+ * rewritten by every call (so two calls that may overlap on the GPU need a workspace each);
  * the size is 0 -- and the pointer may be NULL -- for the e4m3 variant and for shapes served by
  * the CUDA-core kernel.
  */

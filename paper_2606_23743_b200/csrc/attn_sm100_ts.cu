@@ -50,6 +50,7 @@ struct TsParams {
   Strides so;
   int H, N, Nb, R;
   float scale_log2;           // softmax_scale * log2(e)
+  int32_t* next_row;          // device counter (starts at 0): the next CSR row to hand out
   long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
   int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
                               // bit4: starve the pipeline so that a wait runs out (test aid)
@@ -61,11 +62,12 @@ constexpr int TILE = BS * D * 2;            // one bf16 tile: 32 KB
 constexpr int KS = 2;                       // K tiles in flight
 constexpr int VS = 3;                       // V^T tiles in flight
 constexpr int THREADS = 384;
+constexpr int QD = 4;                       // depth of the row queue
 constexpr int OFF_K = 0;
 constexpr int OFF_V = OFF_K + KS * TILE;
 constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][128 B] panels (one per softmax group)
 constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
-constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4;   // barriers, reference exponents, row sums (two rows)
+constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers, reference exponents, row sums (two rows), row queue
 constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;      // + alignment slack
 constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
 // The reference exponent of a row is raised only when a block's maximum exceeds it by more than this
@@ -78,6 +80,7 @@ constexpr float LAZY_LOG2 = 32.0f;
 //   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
 //   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
 //   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
+//   3328 row queue: QD entries {row, count, start, first entry | second entry << 16} | 3392 rq_full[QD] | 3424 rq_empty[QD]
 
 // Kept-block list of CSR row r: count and start.  A corrupt row_ptr pair gives an empty row; every
 // role calls this with the same inputs and so reaches the same answer.
@@ -94,10 +97,12 @@ __device__ __forceinline__ int list_block(const TsParams& prm, int beg, int j) {
   return (J < 0 || J >= prm.Nb) ? 0 : J;
 }
 
-// Persistent kernel: CTA c processes the CSR rows c, c + gridDim.x, ...  All barriers keep running
-// across rows (every role derives the same phase counters from the same row sequence), so the
-// producers and the S issuer run ahead into the next row while the softmax groups finish the
-// current one, and a row's epilogue overlaps the next row's first MMAs.
+// Persistent kernel.  Rows are handed out in their natural order from one device-wide counter (so the
+// CTAs work on neighbouring rows at any time -- their K/V tiles share the L2 -- and rows of unequal
+// length balance by themselves): the K producer, which runs furthest ahead, draws the next row,
+// zero-fills it if its list is empty, and otherwise publishes {row, count, start, first two entries}
+// in a small shared-memory queue that every other role reads in the same order.  All barriers keep running across rows, so the producers and the S
+// issuer run ahead into the next row while the softmax groups finish the current one.
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const TsParams prm) {
@@ -110,11 +115,12 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
                  bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
                  bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
-                 bar_ost = cb + 224;
+                 bar_ost = cb + 224, bar_rq_full = cb + 3392, bar_rq_empty = cb + 3424;
   volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
   volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
   volatile float* lx = reinterpret_cast<volatile float*>(ctrl + 1280);      // [2][2][128]
+  volatile int* rowq = reinterpret_cast<volatile int*>(ctrl + 3328);        // [QD][4]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int Nb = prm.Nb;
@@ -139,6 +145,10 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_init(bar_v_full + 8 * s, 1);
       mbar_init(bar_v_empty + 8 * s, 1);
     }
+    for (int i = 0; i < QD; ++i) {
+      mbar_init(bar_rq_full + 8 * i, 1);
+      mbar_init(bar_rq_empty + 8 * i, 11);       // 3 producer / issuer lanes + one lane of each softmax warp
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -158,6 +168,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   constexpr uint32_t IDESC = instr_desc(128, 128, 1, false);   // bf16 x bf16 -> fp32, A and B K-major
   constexpr int PANEL16 = (BS * 128) >> 4;                      // one 128-row x 128-byte panel
 
+  // Entry i of the row sequence (the same for every role): false when a wait ran out.  r >= R ends the
+  // sequence.  `arrive` tells whether this thread signs the entry off (one thread per consumer).
+  auto fetch_row = [&](uint32_t i, int& r, int& n, int& beg, int& jj, bool arrive) -> bool {
+    const uint32_t slot = i % QD;
+    if (!mbar_wait(bar_rq_full + 8 * slot, (i / QD) & 1u, abort_flag, prm.status)) return false;
+    r = rowq[4 * slot];
+    n = rowq[4 * slot + 1];
+    beg = rowq[4 * slot + 2];
+    jj = rowq[4 * slot + 3];
+    if (warp < 8) __syncwarp();                  // softmax warps: every lane has read the entry before lane 0 signs
+    if (arrive) mbar_arrive(bar_rq_empty + 8 * slot);
+    return true;
+  };
+
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
     if (warp == 8) {
@@ -166,9 +190,36 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
-          int n, beg;
-          row_list(prm, r, n, beg);
+        for (uint32_t i = 0; ok; ++i) {
+          // ---- row scheduling: draw the next row with a non-empty list and publish it
+          const uint32_t slot = i % QD;
+          if (i >= QD && !mbar_wait(bar_rq_empty + 8 * slot, (i / QD - 1u) & 1u, abort_flag, prm.status)) break;
+          int r, n = 0, beg = 0;
+          for (;;) {
+            r = atomicAdd(prm.next_row, 1);
+            if (r >= prm.R) break;
+            row_list(prm, r, n, beg);
+            if (n > 0) break;
+            // nothing kept (or a corrupt row_ptr pair): zeros and lse = -inf; rare, so this one lane does it
+            const int I = r % Nb, bh0 = r / Nb;
+            for (int t = 0; t < BS; ++t) {
+              const int qi = I * BS + t;
+              if (qi >= prm.N) break;
+              __nv_bfloat16* orow = prm.o + (long long)(bh0 / prm.H) * prm.so.b + (long long)(bh0 % prm.H) * prm.so.h +
+                                    (long long)qi * prm.so.n;
+              for (int cc = 0; cc < D; cc += 8) *reinterpret_cast<uint4*>(orow + cc) = make_uint4(0, 0, 0, 0);
+              if (prm.lse) prm.lse[(long long)bh0 * prm.N + qi] = -INFINITY;
+            }
+          }
+          int jj = 0;
+          if (r < prm.R) jj = list_block(prm, beg, 0) | ((n > 1 ? list_block(prm, beg, 1) : 0) << 16);
+          rowq[4 * slot] = r;
+          rowq[4 * slot + 1] = n;
+          rowq[4 * slot + 2] = beg;
+          rowq[4 * slot + 3] = jj;
+          mbar_arrive(bar_rq_full + 8 * slot);
+          if (r >= prm.R) break;
+          // ---- K tiles of the row
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
           for (int j = 0; j < n; ++j) {
             if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
@@ -193,9 +244,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
-          int n, beg;
-          row_list(prm, r, n, beg);
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg, jj;
+          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
           for (int j = 0; j < n; ++j) {
             if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
@@ -217,14 +268,11 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int s = 0;
         uint32_t ph = 0;
         uint32_t cs[2] = {0, 0};            // S tiles issued so far into buffer w
-        uint32_t rows_done = 0;             // non-empty rows started so far
         bool ok = true;
-        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
-          int n, beg;
-          row_list(prm, r, n, beg);
-          if (n == 0) continue;
-          ok = mbar_wait(bar_q_ready, rows_done & 1u, abort_flag, prm.status);
-          ++rows_done;
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg, jj;
+          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
+          ok = mbar_wait(bar_q_ready, i & 1u, abort_flag, prm.status);
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
             if (cs[w] > 0) {
@@ -254,15 +302,12 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int s = 0;
         uint32_t ph = 0;
         uint32_t cp[2] = {0, 0};            // P V groups issued so far for parity w
-        uint32_t rows_done = 0;
         bool ok = true;
-        for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
-          int n, beg;
-          row_list(prm, r, n, beg);
-          if (n == 0) continue;
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg, jj;
+          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
           // the first P V of a row overwrites O: the previous row's O must have been read
-          if (rows_done > 0) ok = mbar_wait(bar_o_free, (rows_done - 1u) & 1u, abort_flag, prm.status);
-          ++rows_done;
+          if (i > 0) ok = mbar_wait(bar_o_free, (i - 1u) & 1u, abort_flag, prm.status);
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
             const uint64_t vd = vd0 + (uint64_t)(s * (TILE >> 4));
@@ -315,14 +360,6 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
       }
     };
-    auto next_row = [&](int r) {                              // next non-empty row of this CTA (or >= R)
-      for (r += gridDim.x; r < prm.R; r += gridDim.x) {
-        int n, beg;
-        row_list(prm, r, n, beg);
-        if (n > 0) return r;
-      }
-      return prm.R;
-    };
     auto store_q = [&](const uint32_t* qv) {
       tmem_st32(q_tmem, qv);
       tc_wait_st();
@@ -330,41 +367,24 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_arrive(bar_q_ready);
     };
 
-    // first non-empty row: its Q goes in right away
-    int r_first = (int)blockIdx.x - (int)gridDim.x;
-    r_first = next_row(r_first);
-    {
+    // The row sequence comes from the queue the K producer fills.  The entry after the current one is
+    // read in the epilogue (the producer has published it by then: it runs about two blocks ahead),
+    // so the next row's Q and first list entries are at hand when the row changes.
+    const bool signs = lane == 0;                             // one lane per warp signs queue entries off
+    int r_c = prm.R, n_c = 0, beg_c = 0, jj_c = 0;
+    if (!fetch_row(0, r_c, n_c, beg_c, jj_c, signs)) ok = false;
+    if (ok && r_c < prm.R) {
+      // first row: its Q goes in right away
       uint32_t qv[32];
-      load_q(r_first, qv);
-      if (r_first < prm.R) store_q(qv);
+      load_q(r_c, qv);
+      store_q(qv);
     }
-
-    // The list of the row after this one (count, start, first entry of this group) is loaded one row
-    // ahead, so that no global-memory latency sits between two rows.
-    int n_c = 0, beg_c = 0, J_c = 0;
-    if ((int)blockIdx.x < prm.R) {
-      row_list(prm, blockIdx.x, n_c, beg_c);
-      if (w < n_c) J_c = list_block(prm, beg_c, w);
-    }
-    for (int r = blockIdx.x; r < prm.R && ok; r += gridDim.x) {
-      const int n = n_c, lbeg = beg_c;
-      int J = J_c;
-      const int r_c = r + gridDim.x;
-      n_c = 0;
-      if (r_c < prm.R) row_list(prm, r_c, n_c, beg_c);                // consumed in this row's last block
+    for (; ok && r_c < prm.R; ++rows_done) {
+      const int r = r_c, n = n_c, lbeg = beg_c;
+      int J = (w == 0) ? (jj_c & 0xffff) : (jj_c >> 16);              // my first block of the row
       const int I = r % Nb, bh = r / Nb;
       const int hh = bh % prm.H, bb = bh / prm.H;
       const int qi = I * BS + row;
-      __nv_bfloat16* orow = prm.o + (long long)bb * prm.so.b + (long long)hh * prm.so.h + (long long)qi * prm.so.n;
-      if (n == 0) {
-        if (qi < prm.N) {
-#pragma unroll
-          for (int cc = 0; cc < D / 2; cc += 8) *reinterpret_cast<uint4*>(orow + (D / 2) * w + cc) = make_uint4(0, 0, 0, 0);
-          if (prm.lse && w == 0) prm.lse[(long long)bh * prm.N + qi] = -INFINITY;
-        }
-        if (w < n_c) J_c = list_block(prm, beg_c, w);
-        continue;
-      }
       const int wl = (n - 1) & 1;                                     // group that takes the row's last block
       const uint32_t last = cnt[wl] + (uint32_t)((n - 1) >> 1);       // phase index of that block
       float m_mine = -INFINITY;      // reference exponent my partial row sum is relative to
@@ -462,8 +482,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (!ok) break;
       // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
       // normalise and store (each group half of d)
-      const int r_next = (n_c > 0 || r_c >= prm.R) ? r_c : next_row(r_c);   // next non-empty row of this CTA
-      if (w < n_c) J_c = list_block(prm, beg_c, w);
+      if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, jj_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
+      const int r_next = r_c;                                         // (the queue holds non-empty rows only)
       uint32_t qn[32];
       load_q(r_next, qn);                                             // in flight during the waits below
       if (!mbar_wait(bar_ref + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
@@ -512,7 +532,6 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
       cnt[0] += (uint32_t)((n + 1) >> 1);
       cnt[1] += (uint32_t)(n >> 1);
-      ++rows_done;
     }
     if ((threadIdx.x & 127) == 0) bulk_wait0();                       // my output stores have completed
   }
@@ -539,7 +558,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // exactly like a K tile.
 __global__ void __launch_bounds__(256)
 transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
-                   int Nb, int d) {
+                   int Nb, int d, int32_t* __restrict__ row_counter) {
+  // the attention kernel that follows draws its rows from this counter
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *row_counter = 0;
   __shared__ __nv_bfloat16 tile[64][66];            // [d][key], padded
   const int n0 = blockIdx.x * 64, d0 = blockIdx.y * 64, bh = blockIdx.z;
   const int b = bh / H, h = bh % H;
@@ -629,7 +650,8 @@ static int launch_ts(const Dims& m, const CUtensorMap& tk, const CUtensorMap& tv
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {
-  return (size_t)m.B * m.H * m.Nb * BS * m.d * 2;        // one transposed V tile per (b, h, key block)
+  // one transposed V tile per (b, h, key block), then the row counter of the scheduler
+  return (size_t)m.B * m.H * m.Nb * BS * m.d * 2 + 256;
 }
 
 int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
@@ -651,7 +673,8 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
   if ((rc = make_map_ts(&tv, ws, BS, vrows, m.H, m.B, (cuuint64_t)BS * 2, vrows * BS * 2, vrows * BS * 2 * m.H)) != SVA_OK)
     return rc;
   dim3 tg(m.Nb * 2, m.d / 64, m.B * m.H);
-  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d);
+  int32_t* row_counter = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + (size_t)m.B * m.H * m.Nb * BS * m.d * 2);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, row_counter);
   TsParams prm;
   prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
   prm.row_ptr = row_ptr; prm.col_idx = col_idx;
@@ -659,6 +682,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
   prm.so = make_strides(p->o_stride);
   prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
   prm.scale_log2 = m.scale * 1.4426950408889634f;
+  prm.next_row = row_counter;
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
   return launch_ts(m, tk, tv, to, prm, st);

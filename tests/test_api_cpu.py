@@ -91,7 +91,7 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert att(p, o=vp(4)) == 5
     assert att(_problem(qk_dtype=7)) == 1
     assert lib.sva_dense_attn_fwd(C.byref(p), one, one, None, None, None, one, None, None, None, 0, None) == 1
-    assert B.attn_workspace_bytes(p) == 1 * 2 * 8 * 128 * 128 * 2       # transposed V tiles
+    assert B.attn_workspace_bytes(p) == 1 * 2 * 8 * 128 * 128 * 2 + 256  # transposed V tiles + row counter
     assert B.attn_workspace_bytes(_problem(block=64)) == 0               # CUDA-core kernel needs none
     assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 0             # e4m3 variant needs none
     assert att(p) == 3                                                   # bf16 tensor-core path without workspace
