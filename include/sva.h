@@ -159,6 +159,25 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The bf16 tensor-core path in two steps, for callers that can prepare V early -- on another stream
+ * while routing runs (routing never reads V), or because the producer of V can be made to write
+ * the prepared layout itself.  sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
+ * and key block one contiguous tile [d][block keys], keys >= N zero) and resets the row counter in
+ * `workspace`; sva_block_sparse_attn_fwd_prepared then runs the attention kernel alone (row_ptr ==
+ * NULL means dense).  One prepare per attention call (the attention call uses the counter up), and
+ * the caller orders the two (same stream, or an event).  Together they do exactly what
+ * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call.  SVA_ERR_UNSUPPORTED for problems
+ * the bf16 tensor-core kernel does not serve (e4m3 Q/K, block or d other than 128): use the one-call
+ * entry points there.
+ */
+int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, size_t workspace_bytes,
+                       void* stream);
+int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k,
+                                       const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                       int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                       void* stream);
+
+/*
  * Diagnostic twin of sva_block_sparse_attn_fwd: the same contract computed by a plain fp32
  * CUDA-core kernel (no tensor cores, no TMA).  row_ptr == NULL means dense.  Slow; it exists
  * so that the tensor-core kernel can be cross-checked on the device.

@@ -22,6 +22,7 @@ EXPORTS = [
     "sva_select_max_nnz", "sva_select_workspace_bytes", "sva_block_select",
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
+    "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -73,6 +74,10 @@ def lib():
         L.sva_block_sparse_attn_fwd_simt.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.sva_dense_attn_fwd.restype = C.c_int
         L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_attn_prepare_v.restype = C.c_int
+        L.sva_attn_prepare_v.argtypes = [C.POINTER(Problem), vp, vp, C.c_size_t, vp]
+        L.sva_block_sparse_attn_fwd_prepared.restype = C.c_int
+        L.sva_block_sparse_attn_fwd_prepared.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.sva_quantize_qk_fp8.restype = C.c_int
         L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
         L.sva_status_string.restype = C.c_char_p
@@ -175,6 +180,23 @@ def dense_attn_fwd(p: Problem, q, k, v, o, lse=None, status=None, q_scale=None, 
                                   _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_dense_attn_fwd")
+
+
+def attn_prepare_v(p: Problem, v, workspace) -> None:
+    """First half of the bf16 tensor-core path: V -> tiled transposed copy in `workspace` (on the current stream)."""
+    rc = lib().sva_attn_prepare_v(C.byref(p), _ptr(v), _ptr(workspace), _ws_bytes(workspace), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_attn_prepare_v")
+
+
+def block_sparse_attn_fwd_prepared(p: Problem, q, k, row_ptr, col_idx, o, lse=None, status=None,
+                                   workspace=None) -> None:
+    """Second half: the attention kernel alone on a workspace that attn_prepare_v filled (row_ptr None = dense)."""
+    rc = lib().sva_block_sparse_attn_fwd_prepared(C.byref(p), _ptr(q), _ptr(k), _ptr(row_ptr), _ptr(col_idx),
+                                                  _ptr(o), _ptr(lse), _ptr(status), _ptr(workspace),
+                                                  _ws_bytes(workspace), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_sparse_attn_fwd_prepared")
 
 
 def quantize_qk_fp8(p: Problem, q, k, q8, k8, q_scale, k_scale) -> None:

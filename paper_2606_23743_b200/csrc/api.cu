@@ -162,6 +162,33 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
                           (cudaStream_t)stream);
 }
 
+int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, size_t workspace_bytes,
+                       void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!v) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(v)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->v_stride, 8))) return rc;
+  if (p->v_stride[2] < p->d) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  if (!use_sm100(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  return launch_prepare_v_ts(m, p, v, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k,
+                                       const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                       int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  // (q stands in for v in the shared checks: the prepared call takes no V pointer; the v strides of p are still checked)
+  int rc = validate_attn(p, q, k, q, nullptr, nullptr, o);
+  if (rc) return rc;
+  if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  if (!use_sm100(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  return launch_attn_ts(m, p, q, k, nullptr, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
+                        (cudaStream_t)stream);
+}
+
 int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const void* k,
                                    const void* v, const float* q_scale, const float* k_scale,
                                    const int32_t* row_ptr, const int32_t* col_idx, void* o,

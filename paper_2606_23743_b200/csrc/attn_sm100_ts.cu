@@ -654,16 +654,37 @@ size_t attn_ts_workspace_bytes(const Dims& m) {
   return (size_t)m.B * m.H * m.Nb * BS * m.d * 2 + 256;
 }
 
-int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
-                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                   void* ws, size_t ws_bytes, cudaStream_t st) {
+static int check_ts_workspace(const Dims& m, const void* ws, size_t ws_bytes) {
   if (m.block != BS || m.d != 128 || m.fp8) return SVA_ERR_UNSUPPORTED;
   if (!ws || ws_bytes < attn_ts_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
-  const Strides sk = make_strides(p->k_stride), sv = make_strides(p->v_stride);
+  return SVA_OK;
+}
+static int32_t* ts_row_counter(const Dims& m, void* ws) {
+  return reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + (size_t)m.B * m.H * m.Nb * BS * m.d * 2);
+}
+
+// V -> tiled transposed copy in the workspace, row counter of the scheduler = 0.
+int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
+                        cudaStream_t st) {
+  int rc = check_ts_workspace(m, ws, ws_bytes);
+  if (rc) return rc;
+  const Strides sv = make_strides(p->v_stride);
+  dim3 tg(m.Nb * 2, m.d / 64, m.B * m.H);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d,
+                                         ts_row_counter(m, ws));
+  return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
+}
+
+// v == nullptr: the workspace has been prepared by launch_prepare_v_ts (once per attention call).
+int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
+                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                   void* ws, size_t ws_bytes, cudaStream_t st) {
+  int rc = check_ts_workspace(m, ws, ws_bytes);
+  if (rc) return rc;
+  const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
   CUtensorMap tk, tv, to;
-  int rc;
   if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2)) != SVA_OK)
     return rc;
   if ((rc = make_map_ts(&tk, k, m.d, m.N, m.H, m.B, (cuuint64_t)sk.n * 2, (cuuint64_t)sk.h * 2, (cuuint64_t)sk.b * 2)) != SVA_OK)
@@ -672,9 +693,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
   const cuuint64_t vrows = (cuuint64_t)m.Nb * m.d;
   if ((rc = make_map_ts(&tv, ws, BS, vrows, m.H, m.B, (cuuint64_t)BS * 2, vrows * BS * 2, vrows * BS * 2 * m.H)) != SVA_OK)
     return rc;
-  dim3 tg(m.Nb * 2, m.d / 64, m.B * m.H);
-  int32_t* row_counter = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + (size_t)m.B * m.H * m.Nb * BS * m.d * 2);
-  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, row_counter);
+  if (v && (rc = launch_prepare_v_ts(m, p, v, ws, ws_bytes, st)) != SVA_OK) return rc;
   TsParams prm;
   prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
   prm.row_ptr = row_ptr; prm.col_idx = col_idx;
@@ -682,7 +701,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
   prm.so = make_strides(p->o_stride);
   prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
   prm.scale_log2 = m.scale * 1.4426950408889634f;
-  prm.next_row = row_counter;
+  prm.next_row = ts_row_counter(m, ws);
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
   return launch_ts(m, tk, tv, to, prm, st);

@@ -92,6 +92,20 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert att(_problem(qk_dtype=7)) == 1
     assert lib.sva_dense_attn_fwd(C.byref(p), one, one, None, None, None, one, None, None, None, 0, None) == 1
     assert B.attn_workspace_bytes(p) == 1 * 2 * 8 * 128 * 128 * 2 + 256  # transposed V tiles + row counter
+    # the two-step form of the bf16 tensor-core path
+    prep = lambda pp, v=one, ws=one, nb=1 << 30: lib.sva_attn_prepare_v(C.byref(pp), v, ws, nb, None)
+    assert prep(p, v=None) == 1
+    assert prep(p, ws=None) == 3
+    assert prep(p, nb=16) == 3
+    assert prep(p, ws=vp(4096 + 16)) == 5
+    assert prep(_problem(qk_dtype=1)) == 2                                # e4m3 Q/K: one-call entry points only
+    assert prep(_problem(block=64)) == 2
+    att2 = lambda pp, q=one, rp=one, ci=one, ws=None: lib.sva_block_sparse_attn_fwd_prepared(
+        C.byref(pp), q, one, rp, ci, one, None, None, ws, 0, None)
+    assert att2(p, q=None) == 1
+    assert att2(p, ci=None) == 1
+    assert att2(p) == 3                                                   # no workspace
+    assert att2(_problem(qk_dtype=1)) in (1, 2)
     assert B.attn_workspace_bytes(_problem(block=64)) == 0               # CUDA-core kernel needs none
     assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 0             # e4m3 variant needs none
     assert att(p) == 3                                                   # bf16 tensor-core path without workspace

@@ -78,6 +78,33 @@ def test_repeatable_bytes():
         assert torch.equal(od, o2) and torch.equal(ld, l2)
 
 
+def test_two_step_form_matches_the_one_call_form():
+    """V prepared on a second stream, then the attention kernel alone: same bytes as the one-call entry
+    points (sparse and dense), and the workspace can be prepared again for the next call."""
+    w, _ = CASES["mass_ragged_rows"]
+    (qd, kd, vd), bits, rp, ci = _setup(w)
+    o1, l1, st1 = U.gpu_attn(w, qd, kd, vd, rp, ci)
+    od, ld, _ = U.gpu_attn(w, qd, kd, vd, None, None, dense=True)
+    o2 = torch.full_like(o1, 3.0); l2 = torch.full_like(l1, 3.0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p = B.make_problem(qd, kd, vd, o2, w.N, w.block)
+    ws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    for sparse in (True, False, True):
+        ready = torch.cuda.Event()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            B.attn_prepare_v(p, vd, ws)
+            ready.record()
+        torch.cuda.current_stream().wait_event(ready)
+        B.block_sparse_attn_fwd_prepared(p, qd, kd, rp if sparse else None, ci if sparse else None, o2, l2, status,
+                                         workspace=ws)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref_o, ref_l = (o1, l1) if sparse else (od, ld)
+        assert torch.equal(o2[:, :, :w.N], ref_o[:, :, :w.N]) and torch.equal(l2, ref_l)   # rows >= N are never written
+
+
 def test_empty_rows_and_bad_indices_are_reported_not_trapped():
     w = shrink(WORKLOADS["medium"], H=1, T=2, k=2)       # Nb = 16
     data, bits, rp, ci = _setup(w)
