@@ -35,7 +35,7 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_ts_kernel launch on the "large" workload,
 # from the ncu capture summarised in profiles/attn_ts_kernel_large.md (other workloads: not captured)
-ATTN_TRAFFIC_BYTES = {"large": 794.4e6}
+ATTN_TRAFFIC_BYTES = {"large": 796.0e6}
 
 
 def load_peaks():
