@@ -7,7 +7,6 @@ void set_tiles_per_cta(int n);
 void ts_set_prof_buffer(void* p);
 void ts_set_debug_mode(int v);
 int ts_set_wait_limit(long long cycles);
-void set_exp_emulation(int n);
 void set_prof_buffer(void* p);
 void set_debug_mode(int v);
 int set_wait_limit(long long cycles);
@@ -230,8 +229,6 @@ const char* sva_status_string(int status) {
 void sva_debug_set_tiles_per_cta(int n) { set_tiles_per_cta(n); }
 /* tuning aid: 1 sends bf16 problems to the two-tile kernel that otherwise serves e4m3 (A/B timing) */
 void sva_debug_set_bf16_kernel(int v) { g_bf16_kernel = v; }
-/* tuning switch: 0..3 of every 4 exp2 pairs evaluated by a polynomial on the FMA pipe */
-void sva_debug_set_exp_emulation(int n) { set_exp_emulation(n); }
 /* tuning aid: device buffer of 5*8*8 int64 that CTA 64 fills with a clock64 timeline; NULL = off */
 void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); ts_set_prof_buffer(p); }
 /* tuning aid: bit0 skips the softmax arithmetic (results are wrong; timing of the MMA side only) */

@@ -65,7 +65,7 @@ struct Cfg {
 //   96 + 128*t : k_full[2] | +16 k_empty[2] | +32 v_full[6] | +80 v_empty[6]
 //   352 tmem_base   356 abort   360 n_list[2]   368 beg[2]   376 issue lock
 
-template <int D, int NT, bool F8, int EMU>
+template <int D, int NT, bool F8>
 __global__ void __launch_bounds__(NT * 128 + 128, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams prm) {
@@ -377,15 +377,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           }
         }
         if (probe) SVA_PROF(t, j, 3);
-        // ---- P = 2^(S*c - m_used).  EMU of every 8 elements take a polynomial on the FMA pipe,
-        // the others the MUFU.  Packed bf16 pairs overwrite sv[0..63].
+        // ---- P = 2^(S*c - m_used); the packed bf16 pairs overwrite sv[0..63]
         const float nm = -m_used;
         float sum_a = 0.f, sum_b = 0.f;
 #pragma unroll
         for (int i = 0; i < 128; i += 2) {
           const float x0 = fmaf(__uint_as_float(sv[i]), c, nm), x1 = fmaf(__uint_as_float(sv[i + 1]), c, nm);
-          const float p0 = ((i & 7) < EMU) ? ex2_poly(x0) : ex2(x0);
-          const float p1 = (((i + 1) & 7) < EMU) ? ex2_poly(x1) : ex2(x1);
+          const float p0 = ex2(x0), p1 = ex2(x1);
           sum_a += p0;
           sum_b += p1;
           sv[i / 2] = pack_bf16(p0, p1);
@@ -493,13 +491,12 @@ static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, in
 static int g_tiles_per_cta = 2;   // bring-up switch, see sva_debug_set_tiles_per_cta
 static long long* g_prof = nullptr;   // tuning aid, see sva_debug_set_prof_buffer
 static int g_debug = 0;
-static int g_emu = 0;             // tuning switch: pairs per 4 whose exp2 runs on the FMA pipe
 
-template <int D, int NT, bool F8, int EMU>
+template <int D, int NT, bool F8>
 static int launch_cfg(const Dims& m, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                       const AttnParams& prm, cudaStream_t st) {
   using C = Cfg<D, NT, F8>;
-  auto kern = attn_sm100_kernel<D, NT, F8, EMU>;
+  auto kern = attn_sm100_kernel<D, NT, F8>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
     return SVA_ERR_CUDA;
   const int grid = (m.R + NT - 1) / NT;
@@ -528,18 +525,8 @@ int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, cons
   prm.debug = g_debug;
   // a CTA's tiles must belong to one head: pair tiles only when Nb is even
   const int nt = (g_tiles_per_cta == 2 && m.Nb % 2 == 0) ? 2 : 1;
-#define SVA_DISPATCH(NTV, F8V)                                                        \
-  switch (g_emu) {                                                                     \
-    case 0: return launch_cfg<128, NTV, F8V, 0>(m, tq, tk, tv, prm, st);              \
-    case 1: return launch_cfg<128, NTV, F8V, 1>(m, tq, tk, tv, prm, st);              \
-    case 2: return launch_cfg<128, NTV, F8V, 2>(m, tq, tk, tv, prm, st);              \
-    default: return launch_cfg<128, NTV, F8V, 3>(m, tq, tk, tv, prm, st);             \
-  }
-  if (m.fp8) {
-    if (nt == 2) { SVA_DISPATCH(2, true) } else { SVA_DISPATCH(1, true) }
-  }
-  if (nt == 2) { SVA_DISPATCH(2, false) } else { SVA_DISPATCH(1, false) }
-#undef SVA_DISPATCH
+  if (m.fp8) return nt == 2 ? launch_cfg<128, 2, true>(m, tq, tk, tv, prm, st) : launch_cfg<128, 1, true>(m, tq, tk, tv, prm, st);
+  return nt == 2 ? launch_cfg<128, 2, false>(m, tq, tk, tv, prm, st) : launch_cfg<128, 1, false>(m, tq, tk, tv, prm, st);
 }
 
 void set_tiles_per_cta(int n) { g_tiles_per_cta = n == 1 ? 1 : 2; }
@@ -549,6 +536,5 @@ int set_wait_limit(long long cycles) {
   if (cycles <= 0) cycles = WAIT_LIMIT_CYCLES;
   return cudaMemcpyToSymbol(g_wait_limit, &cycles, sizeof(cycles)) == cudaSuccess ? 0 : 1;
 }
-void set_exp_emulation(int n) { g_emu = n < 0 ? 0 : (n > 3 ? 3 : n); }
 
 }  // namespace sva

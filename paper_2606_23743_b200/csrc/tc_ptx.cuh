@@ -189,33 +189,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return y;
 }
 // 2^x for x <= ~8 on the FMA pipe: round-to-nearest split x = n + f, |f| <= 0.5, cubic minimax
-// polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent added
-// to the bit pattern.  Takes and returns a pair so the packed f32x2 instructions are used.
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-  const float MAGIC = 12582912.0f;                       // 1.5 * 2^23
-  x.x = fmaxf(x.x, -126.0f);
-  x.y = fmaxf(x.y, -126.0f);
-  const float2 t = __fadd2_rn(x, make_float2(MAGIC, MAGIC));
-  const float2 n = __fadd2_rn(t, make_float2(-MAGIC, -MAGIC));
-  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-  float2 p = __ffma2_rn(f, make_float2(0.05517132f, 0.05517132f), make_float2(0.24261054f, 0.24261054f));
-  p = __ffma2_rn(p, f, make_float2(0.69326097f, 0.69326097f));
-  p = __ffma2_rn(p, f, make_float2(0.99992812f, 0.99992812f));
-  float2 r;
-  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
-  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
-  return r;
-}
-__device__ __forceinline__ float ex2_poly(float x) {
-  const float MAGIC = 12582912.0f;                       // 1.5 * 2^23
-  x = fmaxf(x, -126.0f);
-  const float t = x + MAGIC;
-  const float f = x - (t - MAGIC);
-  float p = fmaf(f, 0.05517132f, 0.24261054f);
-  p = fmaf(p, f, 0.69326097f);
-  p = fmaf(p, f, 0.99992812f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

@@ -127,6 +127,35 @@ def test_empty_rows_and_bad_indices_are_reported_not_trapped():
         U.check_attn_vs_oracle(w, *bits, rp, ci, o, lse, [0, 4, 6, 15])
 
 
+def test_runs_of_empty_rows_and_no_rows_at_all():
+    """The row scheduler finishes rows with an empty list itself: runs of them (between, before and
+    after rows with work) and a CSR without any entry must give zeros / -inf and no hang."""
+    w = shrink(WORKLOADS["medium"], H=2, T=2, k=3)       # Nb = 16, R = 32
+    data, bits, rp, ci = _setup(w)
+    rp_h, ci_h = rp.cpu().clone(), ci.cpu().clone()
+    keep = [5, 6, 20]                                    # every other row loses its list
+    cnt = rp_h[1:] - rp_h[:-1]
+    new_cnt = torch.zeros_like(cnt)
+    for r in keep:
+        new_cnt[r] = cnt[r]
+    rp2 = torch.zeros_like(rp_h); rp2[1:] = torch.cumsum(new_cnt, 0)
+    ci2 = torch.cat([ci_h[rp_h[r]: rp_h[r + 1]] for r in keep])
+    o_ref, lse_ref, _ = U.gpu_attn(w, *data, rp, ci)
+    o, lse, st = U.gpu_attn(w, *data, rp2.cuda(), ci2.cuda())
+    assert st == 0
+    for r in range(w.R):
+        bh, I = divmod(r, w.Nb)
+        sl = (bh // w.H, bh % w.H, slice(I * w.block, min((I + 1) * w.block, w.N)))
+        if r in keep:
+            assert torch.equal(o[sl], o_ref[sl]) and torch.equal(lse[sl], lse_ref[sl])
+        else:
+            assert (o[sl] == 0).all() and torch.isinf(lse[sl]).all() and (lse[sl] < 0).all()
+    # no entry at all
+    rp0 = torch.zeros_like(rp)
+    o, lse, st = U.gpu_attn(w, *data, rp0, ci)
+    assert st == 0 and (o[:, :, :w.N] == 0).all() and torch.isinf(lse).all()
+
+
 def test_strided_qkv_and_output():
     w = shrink(WORKLOADS["medium"], H=2, T=2)
     (q, k, v), bits = U.host_inputs(w)
