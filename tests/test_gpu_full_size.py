@@ -33,6 +33,22 @@ def test_full_size_select_then_attend(name, nrows):
     assert of.abs().amax() <= vmax * 1.01
     if w.n_alloc > w.N:
         assert (o[:, :, w.N:] == 7.0).all()
+    if name == "large":
+        # the launch configuration bench.py times: V prepared on a second stream, then the kernel alone
+        from paper_2606_23743_b200 import binding as B
+        o2 = torch.full_like(o, 7.0); lse2 = torch.full_like(lse, 7.0)
+        st2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+        p = B.make_problem(qd, kd, vd, o2, w.N, w.block)
+        aws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        side, ready = torch.cuda.Stream(), torch.cuda.Event()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            B.attn_prepare_v(p, vd, aws)
+            ready.record()
+        torch.cuda.current_stream().wait_event(ready)
+        B.block_sparse_attn_fwd_prepared(p, qd, kd, rp, ci, o2, lse2, st2, workspace=aws)
+        torch.cuda.synchronize()
+        assert int(st2.item()) == 0 and torch.equal(o2, o) and torch.equal(lse2, lse)
     if name == "medium":
         od, lsd, _ = U.gpu_attn(w, qd, kd, vd, None, None, dense=True)
         U.check_attn_vs_oracle(w, qb, kb, vb, None, None, od, lsd, rows[:4], dense=True)
