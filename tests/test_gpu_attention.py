@@ -27,6 +27,10 @@ CASES = {
     "window": (shrink(WORKLOADS["xl"], B=2, H=2, T=5), 12),
     "single_block": (shrink(WORKLOADS["medium"], H=1, T=1, Hg=8, Wg=16, k=1), None),   # N = 128
     "short_tail_only": (shrink(WORKLOADS["medium"], H=2, T=1, Hg=5, Wg=20, k=1), None),  # N = 100 < block
+    "block64_d128": (shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=8), 10),          # CUDA-core kernel
+    "block128_d64": (shrink(WORKLOADS["tiny"], H=2, T=4, block=128, k=3), None),         # CUDA-core kernel
+    "many_rows_few_blocks": (shrink(WORKLOADS["medium"], H=6, T=8, k=2), 12),            # R = 384 > 148 CTAs, 2 blocks per row
+    "one_block_rows": (shrink(WORKLOADS["medium"], H=3, T=4, k=1), 10),                  # odd row length 1: only one group has work
 }
 
 
