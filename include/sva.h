@@ -140,10 +140,13 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  *   lse_i = log sum_j exp(scale*<q_i,k_j>)       (optional, [B,H,N] fp32 contiguous)
  * O is bf16.  A row with an empty list writes zeros and lse = -inf.
  * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
- * (16 for e4m3 Q/K).  Tensor-core kernel: bf16 (or e4m3 x e4m3) MMA, fp32 accumulate.
+ * (16 for e4m3 Q/K).  Tensor-core kernels (bf16 or e4m3 x e4m3 MMA, fp32 accumulate) serve d = 128:
+ * bf16 Q/K with 128- or 64-token blocks, e4m3 Q/K with 128-token blocks; other supported shapes run
+ * on a CUDA-core kernel.
  * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The bf16 tensor-core kernel
- * keeps a tiled, transposed copy of V (2*B*H*Nb*block*d bytes) and its row counter there, both
- * rewritten by every call (so two calls that may overlap on the GPU need a workspace each);
+ * keeps a tiled, transposed copy of V (2*B*H*Nb*block*d bytes), its row counter and, for 64-token
+ * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
+ * GPU need a workspace each);
  * the size is 0 -- and the pointer may be NULL -- for the e4m3 variant and for shapes served by
  * the CUDA-core kernel.
  */
@@ -167,8 +170,8 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
  * NULL means dense).  One prepare per attention call (the attention call uses the counter up), and
  * the caller orders the two (same stream, or an event).  Together they do exactly what
  * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call.  SVA_ERR_UNSUPPORTED for problems
- * the bf16 tensor-core kernel does not serve (e4m3 Q/K, block or d other than 128): use the one-call
- * entry points there.
+ * the bf16 tensor-core kernel does not serve (e4m3 Q/K, d other than 128) and for the dense form with
+ * 64-token blocks: use the one-call entry points there.
  */
 int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, size_t workspace_bytes,
                        void* stream);

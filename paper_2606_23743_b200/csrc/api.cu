@@ -59,9 +59,9 @@ static int validate_attn(const sva_problem_t* p, const void* q, const void* k, c
   return SVA_OK;
 }
 
-// The tensor-core kernels cover 128-token blocks with d = 128 (bf16: the all-TMEM-A kernel, which
-// needs the transposed-V workspace; e4m3 Q/K: the two-tile kernel); other supported shapes run on
-// the CUDA-core kernel.
+// Tensor-core kernels: bf16 with d = 128 and 128- or 64-token blocks runs on the all-TMEM-A kernel
+// (attn_ts_serves; it needs the transposed-V workspace), e4m3 Q/K with 128-token blocks and d = 128 on
+// the two-tile kernel (use_sm100); other supported shapes run on the CUDA-core kernel.
 static bool use_sm100(const Dims& m) { return m.block == 128 && m.d == 128; }
 
 }  // namespace sva
@@ -124,7 +124,7 @@ static int g_bf16_kernel = 0;   /* tuning aid: 1 routes bf16 problems to the two
 size_t sva_attn_workspace_bytes(const sva_problem_t* p) {
   if (validate_problem(p)) return 0;
   Dims m = make_dims(p);
-  return (use_sm100(m) && !m.fp8) ? attn_ts_workspace_bytes(m) : 0;
+  return attn_ts_workspace_bytes(m);
 }
 
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
@@ -135,7 +135,7 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
   if (rc) return rc;
   if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (use_sm100(m) && !m.fp8 && !g_bf16_kernel)
+  if (attn_ts_serves(m) && !(g_bf16_kernel && use_sm100(m)))
     return launch_attn_ts(m, p, q, k, v, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
                           (cudaStream_t)stream);
   if (use_sm100(m))
@@ -151,7 +151,7 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
   int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
   if (rc) return rc;
   Dims m = make_dims(p);
-  if (use_sm100(m) && !m.fp8 && !g_bf16_kernel)
+  if (attn_ts_serves(m) && !(g_bf16_kernel && use_sm100(m)))
     return launch_attn_ts(m, p, q, k, v, nullptr, nullptr, o, lse, device_status, workspace, workspace_bytes,
                           (cudaStream_t)stream);
   if (use_sm100(m))
@@ -170,7 +170,7 @@ int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, s
   if ((rc = check_strides(p->v_stride, 8))) return rc;
   if (p->v_stride[2] < p->d) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!use_sm100(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
   return launch_prepare_v_ts(m, p, v, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
@@ -183,7 +183,7 @@ int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, co
   if (rc) return rc;
   if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!use_sm100(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
   return launch_attn_ts(m, p, q, k, nullptr, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
                         (cudaStream_t)stream);
 }

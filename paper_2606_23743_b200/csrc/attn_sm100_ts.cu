@@ -32,6 +32,14 @@
 // has completed.  Row sums are kept per group and merged in the epilogue, where each group
 // normalises its half of O into a swizzled staging panel that one TMA tile store writes out.
 //
+// 64-token blocks (template switch): the MMA tile stays 128 x 128, so one row of work is two adjacent
+// query blocks (A, B) and one tile two key blocks out of the ascending union of A's and B's lists
+// (pair_lists_kernel builds the tile lists).  The K / V^T producers fetch the two halves of a tile
+// from two key blocks; the softmax excludes, per query block, the half it does not keep -- with -inf
+// as the additive constant of the exponentials' FMA, at no cost -- and masks a ragged tail per half.
+// The price is the part of the union one of the two query blocks does not keep (adjacent query
+// blocks share most of their lists).
+//
 // Every wait is bounded: when one expires the CTA sets SVA_DEV_TIMEOUT, all roles leave their
 // loops, TMEM is released and the kernel returns.  Parity waits never run a whole phase ahead of
 // their barrier (each wait on a barrier is preceded by a wait on its previous phase).
@@ -48,7 +56,11 @@ struct TsParams {
   float* lse;
   int32_t* status;
   Strides so;
-  int H, N, Nb, R;
+  int H, N, Nb, R;            // Nb: key blocks per head; R: rows handed out (128-query tiles)
+  int Nt;                     // 128-query tiles per head (= Nb for 128-token blocks, ceil(Nb/2) for 64-token blocks)
+  const int32_t* tile_cnt;    // 64-token blocks only: per tile row, number of 128-key tiles ...
+  const int32_t* tile_beg;    // ... and where its descriptors start
+  const uint32_t* tile_desc;  // two 16-bit halves {key block (14 bits), kept by query block A, kept by B}
   float scale_log2;           // softmax_scale * log2(e)
   int32_t* next_row;          // device counter (starts at 0): the next CSR row to hand out
   long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
@@ -80,21 +92,28 @@ constexpr float LAZY_LOG2 = 32.0f;
 //   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
 //   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
 //   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
-//   3328 row queue: QD entries {row, count, start, first entry | second entry << 16} | 3392 rq_full[QD] | 3424 rq_empty[QD]
+//   3328 row queue: QD entries {row, count, start, first entry, second entry, -, -, -} | 3456 rq_full[QD] | 3488 rq_empty[QD]
 
-// Kept-block list of CSR row r: count and start.  A corrupt row_ptr pair gives an empty row; every
-// role calls this with the same inputs and so reaches the same answer.
+// Work list of row r (a 128-query tile): count and start.  128-token blocks: the CSR row itself (a corrupt
+// row_ptr pair gives an empty row).  64-token blocks: the tile row's list of 128-key tiles that
+// pair_lists_kernel built from the two CSR rows of the tile.  Every role calls this with the same
+// inputs and so reaches the same answer.
+template <bool B64>
 __device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int& beg) {
+  if (B64) { n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r); return; }
   if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return; }
   beg = __ldg(prm.row_ptr + r);
   n = __ldg(prm.row_ptr + r + 1) - beg;
   if (n < 0 || n > prm.Nb || beg < 0) n = 0;
 }
-// Key block of list entry j; an out-of-range entry is replaced by block 0 (the producer reports it).
-__device__ __forceinline__ int list_block(const TsParams& prm, int beg, int j) {
-  if (prm.row_ptr == nullptr) return j;
+// Entry j of a work list.  128-token blocks: the key block (an out-of-range entry is replaced by block 0;
+// the producer reports it).  64-token blocks: the tile descriptor.
+template <bool B64>
+__device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j) {
+  if (B64) return __ldg(prm.tile_desc + beg + j);
+  if (prm.row_ptr == nullptr) return (uint32_t)j;
   const int J = __ldg(prm.col_idx + beg + j);
-  return (J < 0 || J >= prm.Nb) ? 0 : J;
+  return (J < 0 || J >= prm.Nb) ? 0u : (uint32_t)J;
 }
 
 // Persistent kernel.  Rows are handed out in their natural order from one device-wide counter (so the
@@ -103,6 +122,7 @@ __device__ __forceinline__ int list_block(const TsParams& prm, int beg, int j) {
 // zero-fills it if its list is empty, and otherwise publishes {row, count, start, first two entries}
 // in a small shared-memory queue that every other role reads in the same order.  All barriers keep running across rows, so the producers and the S
 // issuer run ahead into the next row while the softmax groups finish the current one.
+template <bool B64>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const TsParams prm) {
@@ -115,15 +135,16 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
                  bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
                  bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
-                 bar_ost = cb + 224, bar_rq_full = cb + 3392, bar_rq_empty = cb + 3424;
+                 bar_ost = cb + 224, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
   volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
   volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
   volatile float* lx = reinterpret_cast<volatile float*>(ctrl + 1280);      // [2][2][128]
-  volatile int* rowq = reinterpret_cast<volatile int*>(ctrl + 3328);        // [QD][4]
+  volatile int* rowq = reinterpret_cast<volatile int*>(ctrl + 3328);        // [QD][8]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int Nb = prm.Nb;
+  const int Nb = prm.Nt;             // row index arithmetic: rows per head
+  constexpr int KB = B64 ? 64 : BS;  // tokens per key block
 
   // ---------------------------------------------------------------- set-up
   const long long t_cta0 = prm.prof ? clock64() : 0;
@@ -170,13 +191,14 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   // Entry i of the row sequence (the same for every role): false when a wait ran out.  r >= R ends the
   // sequence.  `arrive` tells whether this thread signs the entry off (one thread per consumer).
-  auto fetch_row = [&](uint32_t i, int& r, int& n, int& beg, int& jj, bool arrive) -> bool {
+  auto fetch_row = [&](uint32_t i, int& r, int& n, int& beg, uint32_t& e0, uint32_t& e1, bool arrive) -> bool {
     const uint32_t slot = i % QD;
     if (!mbar_wait(bar_rq_full + 8 * slot, (i / QD) & 1u, abort_flag, prm.status)) return false;
-    r = rowq[4 * slot];
-    n = rowq[4 * slot + 1];
-    beg = rowq[4 * slot + 2];
-    jj = rowq[4 * slot + 3];
+    r = rowq[8 * slot];
+    n = rowq[8 * slot + 1];
+    beg = rowq[8 * slot + 2];
+    e0 = (uint32_t)rowq[8 * slot + 3];
+    e1 = (uint32_t)rowq[8 * slot + 4];
     if (warp < 8) __syncwarp();                  // softmax warps: every lane has read the entry before lane 0 signs
     if (arrive) mbar_arrive(bar_rq_empty + 8 * slot);
     return true;
@@ -198,7 +220,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (;;) {
             r = atomicAdd(prm.next_row, 1);
             if (r >= prm.R) break;
-            row_list(prm, r, n, beg);
+            row_list<B64>(prm, r, n, beg);
             if (n > 0) break;
             // nothing kept (or a corrupt row_ptr pair): zeros and lse = -inf; rare, so this one lane does it
             const int I = r % Nb, bh0 = r / Nb;
@@ -211,12 +233,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (prm.lse) prm.lse[(long long)bh0 * prm.N + qi] = -INFINITY;
             }
           }
-          int jj = 0;
-          if (r < prm.R) jj = list_block(prm, beg, 0) | ((n > 1 ? list_block(prm, beg, 1) : 0) << 16);
-          rowq[4 * slot] = r;
-          rowq[4 * slot + 1] = n;
-          rowq[4 * slot + 2] = beg;
-          rowq[4 * slot + 3] = jj;
+          uint32_t e0 = 0u, e1 = 0u;
+          if (r < prm.R) { e0 = list_block<B64>(prm, beg, 0); if (n > 1) e1 = list_block<B64>(prm, beg, 1); }
+          rowq[8 * slot] = r;
+          rowq[8 * slot + 1] = n;
+          rowq[8 * slot + 2] = beg;
+          rowq[8 * slot + 3] = (int)e0;
+          rowq[8 * slot + 4] = (int)e1;
           mbar_arrive(bar_rq_full + 8 * slot);
           if (r >= prm.R) break;
           // ---- K tiles of the row
@@ -224,15 +247,26 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (int j = 0; j < n; ++j) {
             if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
             if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-            int J = j;
-            if (prm.row_ptr) {
-              J = __ldg(prm.col_idx + beg + j);
-              if (J < 0 || J >= Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
-            }
             const uint32_t dst = sbase + OFF_K + s * TILE;
             mbar_expect_tx(bar_k_full + 8 * s, TILE);
-            tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);
-            tma_load_4d(dst + TILE / 2, &tm_k, bar_k_full + 8 * s, 64, J * BS, hh, bb);
+            if (B64) {
+              // two 64-key blocks side by side: rows 0..63 and 64..127 of both d-panels
+              const uint32_t dsc = __ldg(prm.tile_desc + beg + j);
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const int J = (int)((dsc >> (16 * h)) & 0x3fffu);
+                tma_load_4d(dst + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 0, J * KB, hh, bb);
+                tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 64, J * KB, hh, bb);
+              }
+            } else {
+              int J = j;
+              if (prm.row_ptr) {
+                J = __ldg(prm.col_idx + beg + j);
+                if (J < 0 || J >= prm.Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
+              }
+              tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_k, bar_k_full + 8 * s, 64, J * BS, hh, bb);
+            }
             if (++s == KS) { s = 0; ph ^= 1u; }
           }
         }
@@ -245,16 +279,23 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         uint32_t ph = 0;
         bool ok = true;
         for (uint32_t i = 0; ok; ++i) {
-          int r, n, beg, jj;
-          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
           for (int j = 0; j < n; ++j) {
             if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-            const int J = list_block(prm, beg, j);
+            const uint32_t e = list_block<B64>(prm, beg, j);
             const uint32_t dst = sbase + OFF_V + s * TILE;
             mbar_expect_tx(bar_v_full + 8 * s, TILE);
-            tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, J * BS, hh, bb);
-            tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, J * BS, hh, bb);
+            if (B64) {
+              // each 64-key panel of the tile is one key block's transposed V: [128 d rows][64 keys]
+              tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)(e & 0x3fffu) * D, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 0, (int)((e >> 16) & 0x3fffu) * D, hh, bb);
+            } else {
+              tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)e * BS, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, (int)e * BS, hh, bb);
+            }
             if (++s == VS) { s = 0; ph ^= 1u; }
           }
         }
@@ -270,8 +311,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         uint32_t cs[2] = {0, 0};            // S tiles issued so far into buffer w
         bool ok = true;
         for (uint32_t i = 0; ok; ++i) {
-          int r, n, beg, jj;
-          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
           ok = mbar_wait(bar_q_ready, i & 1u, abort_flag, prm.status);
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
@@ -304,8 +346,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         uint32_t cp[2] = {0, 0};            // P V groups issued so far for parity w
         bool ok = true;
         for (uint32_t i = 0; ok; ++i) {
-          int r, n, beg, jj;
-          if (!fetch_row(i, r, n, beg, jj, true) || r >= prm.R) break;
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
           // the first P V of a row overwrites O: the previous row's O must have been read
           if (i > 0) ok = mbar_wait(bar_o_free, (i - 1u) & 1u, abort_flag, prm.status);
           for (int j = 0; j < n && ok; ++j) {
@@ -339,7 +382,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t o_tmem = tmem_base + lane_addr + COL_O;
     const uint32_t p_tmem = tmem_base + lane_addr + COL_P;
     const uint32_t q_tmem = tmem_base + lane_addr + COL_Q + 32 * w;
-    const int tail_keys = prm.N - (Nb - 1) * BS;             // valid keys of the last block
+    const int tail_keys = prm.N - (prm.Nb - 1) * KB;         // valid keys of the last key block
+    const int qh = row >> 6;                                 // 64-token blocks: which query block of the tile I am in
     const float c = prm.scale_log2;
     uint32_t cnt[2] = {0, 0};      // blocks of parity 0 / 1 completed in earlier rows (barrier phase bases)
     uint32_t rows_done = 0;        // non-empty rows finished
@@ -371,8 +415,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // read in the epilogue (the producer has published it by then: it runs about two blocks ahead),
     // so the next row's Q and first list entries are at hand when the row changes.
     const bool signs = lane == 0;                             // one lane per warp signs queue entries off
-    int r_c = prm.R, n_c = 0, beg_c = 0, jj_c = 0;
-    if (!fetch_row(0, r_c, n_c, beg_c, jj_c, signs)) ok = false;
+    int r_c = prm.R, n_c = 0, beg_c = 0;
+    uint32_t e0_c = 0u, e1_c = 0u;
+    if (!fetch_row(0, r_c, n_c, beg_c, e0_c, e1_c, signs)) ok = false;
     if (ok && r_c < prm.R) {
       // first row: its Q goes in right away
       uint32_t qv[32];
@@ -381,7 +426,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
     for (; ok && r_c < prm.R; ++rows_done) {
       const int r = r_c, n = n_c, lbeg = beg_c;
-      int J = (w == 0) ? (jj_c & 0xffff) : (jj_c >> 16);              // my first block of the row
+      uint32_t J = (w == 0) ? e0_c : e1_c;                           // my first list entry of the row
       const int I = r % Nb, bh = r / Nb;
       const int hh = bh % prm.H, bb = bh / prm.H;
       const int qi = I * BS + row;
@@ -392,15 +437,33 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int j = w; j < n; j += 2) {
         const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
         const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
-        const int valid = (J == Nb - 1) ? tail_keys : BS;
-        if (j + 2 < n) J = list_block(prm, lbeg, j + 2);               // one block ahead
+        // valid keys of the tile's two 64-key halves (64-token blocks: a half whose key block this
+        // thread's query block does not keep counts as 0; uniform over a warp)
+        int v0, v1;
+        if (B64) {
+          const int u0 = (int)(J & 0x3fffu), u1 = (int)((J >> 16) & 0x3fffu);
+          v0 = ((J >> (14 + qh)) & 1u) ? (u0 == prm.Nb - 1 ? tail_keys : 64) : 0;
+          v1 = ((J >> (30 + qh)) & 1u) ? (u1 == prm.Nb - 1 ? tail_keys : 64) : 0;
+        } else {
+          const int valid = ((int)J == prm.Nb - 1) ? tail_keys : BS;
+          v0 = valid < 64 ? valid : 64;
+          v1 = valid - v0;
+        }
+        if (j + 2 < n) J = list_block<B64>(prm, lbeg, j + 2);          // one entry ahead
         if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
         tc_fence_after();
-        if (valid < BS) {
-          // ragged last key block: keys that do not exist become -inf in TMEM before S is read (a short
-          // rolled loop -- this keeps 128 compare/select pairs out of the hot instruction stream)
+        if (v0 + v1 < BS) {
+          // Keys that do not exist (ragged last key block) become -inf in TMEM before S is read: a short
+          // rolled loop, which keeps 128 compare/select pairs out of the hot instruction stream.  A half
+          // that is not kept at all (64-token blocks) is left alone here: it is excluded below.
+          if (!B64 || v0 > 0) {
 #pragma unroll 1
-          for (int e = valid; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+            for (int e = v0; e < 64; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+          }
+          if (!B64 || v1 > 0) {
+#pragma unroll 1
+            for (int e = 64 + v1; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+          }
           tc_wait_st();
         }
         uint32_t sv[128];
@@ -411,15 +474,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
-        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;   // a, b: keys 0..63; c, d: keys 64..127
 #pragma unroll
-        for (int e = 0; e < 128; e += 8) {
+        for (int e = 0; e < 64; e += 4) {
           mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
           mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
-          mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
-          mxd = max3(mxd, __uint_as_float(sv[e + 6]), __uint_as_float(sv[e + 7]));
+          mxc = max3(mxc, __uint_as_float(sv[e + 64]), __uint_as_float(sv[e + 65]));
+          mxd = max3(mxd, __uint_as_float(sv[e + 66]), __uint_as_float(sv[e + 67]));
         }
-        const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd)) * c;
+        float mx0 = fmaxf(mxa, mxb), mx1 = fmaxf(mxc, mxd);
+        if (B64) {                                           // a half this query block does not keep has no say
+          if (v0 == 0) mx0 = -INFINITY;
+          if (v1 == 0) mx1 = -INFINITY;
+        }
+        const float mx = fmaxf(mx0, mx1) * c;
         // reference exponent left by block j-1 (other group)
         float m_prev = -INFINITY;
         if (j > 0) {
@@ -450,14 +518,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           tc_wait_st();
         }
         // P = 2^(S*c - m); the packed bf16 pairs overwrite sv[0..63]
-        const float nm = -m_new;
-        const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
+        // (64-token blocks: -inf instead of -m for a half that is not kept, or while the row has seen no
+        // kept key yet, makes those P exactly 0 at no cost)
+        float nm = -m_new, nmh1 = -m_new;
+        if (B64) {
+          if (m_new == -INFINITY || v0 == 0) nm = -INFINITY;
+          if (m_new == -INFINITY || v1 == 0) nmh1 = -INFINITY;
+        }
+        const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm), nm2h1 = B64 ? pack2(nmh1, nmh1) : nm2;
         uint64_t sum2 = pack2(0.f, 0.f);
         if (!(prm.debug & 1)) {
 #pragma unroll
           for (int e = 0; e < 128; e += 2) {
             float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, nm2), x0, x1);
+            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, e < 64 ? nm2 : nm2h1), x0, x1);
             const float p0 = ex2(x0), p1 = ex2(x1);
             sum2 = add2(sum2, pack2(p0, p1));
             sv[e / 2] = pack_bf16(p0, p1);
@@ -482,7 +556,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (!ok) break;
       // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
       // normalise and store (each group half of d)
-      if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, jj_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
+      if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
       const int r_next = r_c;                                         // (the queue holds non-empty rows only)
       uint32_t qn[32];
       load_q(r_next, qn);                                             // in flight during the waits below
@@ -499,7 +573,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
       tc_fence_after();
       const float lt = l + lxr[(w ^ 1) * 128 + row];
-      const float inv = 1.0f / lt;
+      // (64-token blocks: a query block with an empty list beside one with work has lt = 0 -> zeros, lse = -inf)
+      const float inv = (!B64 || lt > 0.f) ? 1.0f / lt : 0.f;
       {
         uint32_t ov[64];
         tmem_ld32(o_tmem + (D / 2) * w, ov);
@@ -553,12 +628,12 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 }
 
 // ------------------------------------------------------------------ V^T
-// V [B,H,N,d] (strided) -> tiled transposed copy: for every (b,h) and key block J one contiguous
-// 32 KB tile [d = 128 rows][128 keys], keys >= N zero.  A tile is then one contiguous TMA box pair,
-// exactly like a K tile.
+// V [B,H,N,d] (strided) -> tiled transposed copy: for every (b,h) and key block J (kb = 128 or 64
+// keys) one contiguous tile [d = 128 rows][kb keys], keys >= N zero.  A 128-key tile is then one
+// contiguous TMA box pair, exactly like a K tile; a 64-key tile is one box (one panel of a tile).
 __global__ void __launch_bounds__(256)
 transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
-                   int Nb, int d, int32_t* __restrict__ row_counter) {
+                   int Nb, int d, int kb, int32_t* __restrict__ row_counter) {
   // the attention kernel that follows draws its rows from this counter
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *row_counter = 0;
   __shared__ __nv_bfloat16 tile[64][66];            // [d][key], padded
@@ -580,15 +655,80 @@ transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat1
   __syncthreads();
   {
     const int k8 = threadIdx.x & 7;                 // 8 keys (16 bytes)
-    const int J = n0 / BS, kin = (n0 % BS) + k8 * 8;
+    const int J = n0 / kb, kin = (n0 % kb) + k8 * 8;
 #pragma unroll
     for (int pass = 0; pass < 2; ++pass) {
       const int dd = (threadIdx.x >> 3) + 32 * pass;
       __align__(16) __nv_bfloat16 e[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) e[q] = tile[dd][k8 * 8 + q];
-      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * d + d0 + dd) * BS + kin) = *reinterpret_cast<uint4*>(e);
+      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * d + d0 + dd) * kb + kin) = *reinterpret_cast<uint4*>(e);
     }
+  }
+}
+
+// ------------------------------------------------------------------ 64-token blocks: tile lists
+// The MMA tile is 128 x 128, so with 64-token blocks one tile row is two adjacent query blocks (A, B)
+// and one tile two key blocks.  Per tile row this kernel merges the two CSR rows into the ascending
+// union of their key blocks, pairs the union up into tiles and notes for every key block which of the
+// two query blocks keeps it (the softmax excludes the other).  One warp per tile row: membership
+// bitmaps in shared memory, then every lane enumerates the bits of its word.  Entries are 16 bits
+// {key block (14), kept by A, kept by B}; tile j of the row is the 32-bit word at start + j.  The
+// start needs no scan: ceil((entries before the tile row + its index) / 2) leaves room for every earlier
+// row's ceil(|union| / 2) tiles.
+constexpr int PAIR_WARPS = 8;
+__global__ void __launch_bounds__(PAIR_WARPS * 32)
+pair_lists_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, int Nb, int Nt, int R2,
+                  int32_t* __restrict__ tile_cnt, int32_t* __restrict__ tile_beg, uint32_t* __restrict__ tile_desc,
+                  long long cap, int32_t* __restrict__ status) {
+  __shared__ uint32_t bm[PAIR_WARPS][2][32];
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * PAIR_WARPS + w;
+  if (t >= R2) return;
+  const int bh = t / Nt, I2 = t % Nt;
+  const int rA = bh * Nb + 2 * I2;
+  const bool hasB = 2 * I2 + 1 < Nb;
+  bm[w][0][lane] = 0u;
+  bm[w][1][lane] = 0u;
+  __syncwarp();
+  const int begA = __ldg(row_ptr + rA), endA = __ldg(row_ptr + rA + 1);
+  const int endB = hasB ? __ldg(row_ptr + rA + 2) : endA;
+  const bool bad = begA < 0 || endA < begA || endB < endA || endA - begA > Nb || endB - endA > Nb;
+  bool bad_idx = false;
+  if (!bad) {
+    for (int e = begA + lane; e < endB; e += 32) {
+      const int J = __ldg(col_idx + e);
+      if (J < 0 || J >= Nb) { bad_idx = true; continue; }
+      atomicOr(&bm[w][e < endA ? 0 : 1][J >> 5], 1u << (J & 31));
+    }
+  }
+  if ((bad || bad_idx) && status) atomicOr(status, SVA_DEV_BAD_INDEX);
+  __syncwarp();
+  const uint32_t a = bm[w][0][lane], b = bm[w][1][lane];
+  uint32_t u = a | b;
+  int incl = __popc(u);
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
+  }
+  const int total = __shfl_sync(0xffffffffu, incl, 31);
+  long long start = ((long long)(bad ? 0 : begA) + t + 1) / 2;
+  int ntile = (total + 1) / 2;
+  if (start + ntile > cap) { ntile = 0; if (lane == 0 && status) atomicOr(status, SVA_DEV_BAD_INDEX); }
+  if (ntile > 0) {
+    uint16_t* ent = reinterpret_cast<uint16_t*>(tile_desc) + 2 * start;
+    int p = incl - __popc(u);
+    while (u) {
+      const int bit = __ffs(u) - 1;
+      u &= u - 1;
+      ent[p++] = (uint16_t)((lane * 32 + bit) | (((a >> bit) & 1u) << 14) | (((b >> bit) & 1u) << 15));
+    }
+    if (lane == 0 && (total & 1)) ent[total] = 0;          // odd union: the last tile's second half is nobody's
+  }
+  if (lane == 0) {
+    tile_cnt[t] = ntile;
+    tile_beg[t] = (int32_t)start;
   }
 }
 
@@ -611,9 +751,9 @@ static encode_fn_t get_encode_ts() {
   return fn;
 }
 
-// bf16 4-D map (inner, rows, H, B) with byte strides; box = 64 x 128 (128 bytes x 128 rows), 128-byte swizzle.
+// bf16 4-D map (inner, rows, H, B) with byte strides; box = 64 x box_rows (128 bytes per row), 128-byte swizzle.
 static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuuint64_t rows, int H, int B,
-                       cuuint64_t row_stride, cuuint64_t h_stride, cuuint64_t b_stride) {
+                       cuuint64_t row_stride, cuuint64_t h_stride, cuuint64_t b_stride, int box_rows) {
   encode_fn_t enc = get_encode_ts();
   if (!enc) return SVA_ERR_CUDA;
   cuuint64_t dims[4] = {inner, rows, (cuuint64_t)H, (cuuint64_t)B};
@@ -623,7 +763,7 @@ static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuui
   if (B == 1) strides[2] = strides[1] * (cuuint64_t)H;
   for (int i = 0; i < 3; ++i)
     if (strides[i] % 16 != 0 || strides[i] == 0) return SVA_ERR_ALIGNMENT;
-  cuuint32_t box[4] = {64, (cuuint32_t)BS, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult rc = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -634,34 +774,65 @@ static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuui
 static long long* g_prof_ts = nullptr;
 static int g_debug_ts = 0;
 
-static int launch_ts(const Dims& m, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                     const TsParams& prm,
-                     cudaStream_t st) {
-  auto kern = attn_ts_kernel;
+template <bool B64>
+static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                     const TsParams& prm, cudaStream_t st) {
+  auto kern = attn_ts_kernel<B64>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
     return SVA_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return SVA_ERR_CUDA;
-  const int grid = m.R < sms ? m.R : sms;          // persistent: one CTA per SM, rows round-robin
+  const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
   kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
+// Workspace layout: transposed V tiles | row counter (256 bytes) | 64-token blocks only: tile_cnt[R2],
+// tile_beg[R2], tile_desc[cap] with R2 = B*H*ceil(Nb/2) tile rows and cap the bound for a dense CSR.
+struct TsLayout {
+  size_t vt_bytes, counter_off, cnt_off, beg_off, desc_off, total;
+  long long cap;
+  int R2, Nt;
+};
+static TsLayout ts_layout(const Dims& m) {
+  TsLayout L;
+  L.vt_bytes = (size_t)m.B * m.H * m.Nb * m.block * m.d * 2;
+  L.counter_off = L.vt_bytes;
+  L.Nt = m.block == 64 ? (m.Nb + 1) / 2 : m.Nb;
+  L.R2 = m.B * m.H * L.Nt;
+  L.cnt_off = L.beg_off = L.desc_off = L.counter_off + 256;
+  L.cap = 0;
+  L.total = L.counter_off + 256;
+  if (m.block == 64) {
+    L.beg_off = L.cnt_off + (((size_t)L.R2 * 4 + 255) & ~(size_t)255);
+    L.desc_off = L.beg_off + (((size_t)L.R2 * 4 + 255) & ~(size_t)255);
+    L.cap = ((long long)m.R * m.Nb + L.R2) / 2 + 2;
+    L.total = L.desc_off + (((size_t)L.cap * 4 + 255) & ~(size_t)255);
+  }
+  return L;
+}
+
+bool attn_ts_serves(const Dims& m) { return (m.block == BS || m.block == 64) && m.d == 128 && !m.fp8 && m.Nb <= 16383; }
+
 size_t attn_ts_workspace_bytes(const Dims& m) {
-  // one transposed V tile per (b, h, key block), then the row counter of the scheduler
-  return (size_t)m.B * m.H * m.Nb * BS * m.d * 2 + 256;
+  if (!attn_ts_serves(m)) return 0;
+  size_t bytes = ts_layout(m).total;
+  if (m.block == 64) {                      // the dense entry point runs 64-token blocks as 128-token blocks
+    Dims d = m;
+    d.block = BS; d.Nb = (m.N + BS - 1) / BS; d.R = m.B * m.H * d.Nb;
+    const size_t b2 = ts_layout(d).total;
+    if (b2 > bytes) bytes = b2;
+  }
+  return bytes;
 }
 
 static int check_ts_workspace(const Dims& m, const void* ws, size_t ws_bytes) {
-  if (m.block != BS || m.d != 128 || m.fp8) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
   if (!ws || ws_bytes < attn_ts_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
   return SVA_OK;
-}
-static int32_t* ts_row_counter(const Dims& m, void* ws) {
-  return reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + (size_t)m.B * m.H * m.Nb * BS * m.d * 2);
 }
 
 // V -> tiled transposed copy in the workspace, row counter of the scheduler = 0.
@@ -669,42 +840,73 @@ int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, vo
                         cudaStream_t st) {
   int rc = check_ts_workspace(m, ws, ws_bytes);
   if (rc) return rc;
+  const TsLayout L = ts_layout(m);
   const Strides sv = make_strides(p->v_stride);
-  dim3 tg(m.Nb * 2, m.d / 64, m.B * m.H);
-  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d,
-                                         ts_row_counter(m, ws));
+  dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
+                                         reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + L.counter_off));
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
 // v == nullptr: the workspace has been prepared by launch_prepare_v_ts (once per attention call).
-int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
+int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st) {
-  int rc = check_ts_workspace(m, ws, ws_bytes);
+  int rc = check_ts_workspace(m_in, ws, ws_bytes);
   if (rc) return rc;
+  // dense attention does not depend on the block size: 64-token blocks run as 128-token blocks
+  Dims m = m_in;
+  if (m.block == 64 && row_ptr == nullptr) {
+    m.block = BS;
+    m.Nb = (m.N + BS - 1) / BS;
+    m.R = m.B * m.H * m.Nb;
+  }
+  const bool b64 = m.block == 64;
+  const TsLayout L = ts_layout(m);
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
   CUtensorMap tk, tv, to;
-  if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2)) != SVA_OK)
+  if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2, BS)) != SVA_OK)
     return rc;
-  if ((rc = make_map_ts(&tk, k, m.d, m.N, m.H, m.B, (cuuint64_t)sk.n * 2, (cuuint64_t)sk.h * 2, (cuuint64_t)sk.b * 2)) != SVA_OK)
+  if ((rc = make_map_ts(&tk, k, m.d, m.N, m.H, m.B, (cuuint64_t)sk.n * 2, (cuuint64_t)sk.h * 2, (cuuint64_t)sk.b * 2, m.block)) != SVA_OK)
     return rc;
-  // transposed V: per (b,h) a [Nb*128 rows][128 keys] matrix, tile J = rows J*128 .. J*128+127
+  // transposed V: per (b,h) a [Nb*128 rows][block keys] matrix, key block J = rows J*128 .. J*128+127
   const cuuint64_t vrows = (cuuint64_t)m.Nb * m.d;
-  if ((rc = make_map_ts(&tv, ws, BS, vrows, m.H, m.B, (cuuint64_t)BS * 2, vrows * BS * 2, vrows * BS * 2 * m.H)) != SVA_OK)
+  if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
+                        vrows * m.block * 2 * m.H, BS)) != SVA_OK)
     return rc;
-  if (v && (rc = launch_prepare_v_ts(m, p, v, ws, ws_bytes, st)) != SVA_OK) return rc;
+  if (v) {
+    // (the transposed copy is laid out for the block size of this launch)
+    const Strides sv = make_strides(p->v_stride);
+    dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+    transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
+                                           reinterpret_cast<int32_t*>(wsb + L.counter_off));
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+  } else if (m.block != m_in.block) {
+    return SVA_ERR_UNSUPPORTED;     // a workspace prepared for 64-token blocks cannot serve the dense path
+  }
   TsParams prm;
   prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
   prm.row_ptr = row_ptr; prm.col_idx = col_idx;
   prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
   prm.so = make_strides(p->o_stride);
-  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
+  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.Nt = L.Nt; prm.R = L.R2;
+  prm.tile_cnt = reinterpret_cast<const int32_t*>(wsb + L.cnt_off);
+  prm.tile_beg = reinterpret_cast<const int32_t*>(wsb + L.beg_off);
+  prm.tile_desc = reinterpret_cast<const uint32_t*>(wsb + L.desc_off);
   prm.scale_log2 = m.scale * 1.4426950408889634f;
-  prm.next_row = ts_row_counter(m, ws);
+  prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
-  return launch_ts(m, tk, tv, to, prm, st);
+  if (b64) {
+    pair_lists_kernel<<<(L.R2 + PAIR_WARPS - 1) / PAIR_WARPS, PAIR_WARPS * 32, 0, st>>>(
+        row_ptr, col_idx, m.Nb, L.Nt, L.R2, reinterpret_cast<int32_t*>(wsb + L.cnt_off),
+        reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+    return launch_ts<true>(L.R2, tk, tv, to, prm, st);
+  }
+  return launch_ts<false>(L.R2, tk, tv, to, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }

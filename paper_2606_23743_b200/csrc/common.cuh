@@ -64,6 +64,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st);
 size_t attn_ts_workspace_bytes(const Dims& m);
+bool attn_ts_serves(const Dims& m);    // bf16, d = 128, 128- or 64-token blocks
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
                         cudaStream_t st);
 

@@ -75,6 +75,10 @@ WORKLOADS = {
                    win_t=1, win_s=1, sigma_w=0.5, qk_mult=1.5),
     "large_fp8": Workload("large_fp8", 5, B=1, H=24, d=128, T=21, Hg=30, Wg=52, block=128, mode=1,
                           k=40, tau=0.9, sigma_w=0.5, fp8=True),
+    # paper-shaped second workload (its deployment preset: 64-token blocks, d = 128, about 10 % of the key
+    # blocks kept); same tokens as "large", not a benchmark configuration
+    "large_b64": Workload("large_b64", 7, B=1, H=24, d=128, T=21, Hg=30, Wg=52, block=64, mode=0, k=51,
+                          sigma_w=0.5),
     # test-only variant of "large": stronger offsets so that the mass rule yields ragged rows
     "large_ragged": Workload("large_ragged", 6, B=1, H=24, d=128, T=21, Hg=30, Wg=52, block=128,
                              mode=1, k=40, tau=0.9, sigma_f=0.65, sigma_w=0.65),

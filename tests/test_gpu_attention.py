@@ -27,7 +27,13 @@ CASES = {
     "window": (shrink(WORKLOADS["xl"], B=2, H=2, T=5), 12),
     "single_block": (shrink(WORKLOADS["medium"], H=1, T=1, Hg=8, Wg=16, k=1), None),   # N = 128
     "short_tail_only": (shrink(WORKLOADS["medium"], H=2, T=1, Hg=5, Wg=20, k=1), None),  # N = 100 < block
-    "block64_d128": (shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=8), 10),          # CUDA-core kernel
+    # 64-token blocks with d = 128 run on the tensor-core kernel too (two query blocks and two key blocks per tile)
+    "block64_d128": (shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=8), 10),
+    "b64_ragged_tail": (shrink(WORKLOADS["medium"], H=3, T=2, Hg=30, Wg=31, block=64, k=7), None),    # N = 1860: 30 blocks, 4-key tail
+    "b64_odd_nb": (shrink(WORKLOADS["medium"], H=2, T=1, Hg=30, Wg=30, block=64, k=4), None),       # N = 900: 15 blocks
+    "b64_mass_ragged_rows": (shrink(WORKLOADS["large_ragged"], H=2, T=8, block=64, k=60), 14),
+    "b64_k1": (shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=1), 12),
+    "b64_single_block": (shrink(WORKLOADS["medium"], H=1, T=1, Hg=5, Wg=8, block=64, k=1), None),   # N = 40 < block
     "block128_d64": (shrink(WORKLOADS["tiny"], H=2, T=4, block=128, k=3), None),         # CUDA-core kernel
     "many_rows_few_blocks": (shrink(WORKLOADS["medium"], H=6, T=8, k=2), 12),            # R = 384 > 148 CTAs, 2 blocks per row
     "one_block_rows": (shrink(WORKLOADS["medium"], H=3, T=4, k=1), 10),                  # odd row length 1: only one group has work
@@ -49,7 +55,7 @@ def test_sparse_attention_matches_oracle(name, impl):
         assert (o[:, :, w.N:] == 7.0).all()
 
 
-@pytest.mark.parametrize("name", ["ragged_tail", "medium_h4"])
+@pytest.mark.parametrize("name", ["ragged_tail", "medium_h4", "b64_ragged_tail", "b64_odd_nb"])
 def test_dense_equals_keep_all_and_oracle(name):
     w, _ = CASES[name]
     data, bits, _, _ = _setup(w)
@@ -82,10 +88,11 @@ def test_repeatable_bytes():
         assert torch.equal(od, o2) and torch.equal(ld, l2)
 
 
-def test_two_step_form_matches_the_one_call_form():
+@pytest.mark.parametrize("name", ["mass_ragged_rows", "b64_mass_ragged_rows"])
+def test_two_step_form_matches_the_one_call_form(name):
     """V prepared on a second stream, then the attention kernel alone: same bytes as the one-call entry
-    points (sparse and dense), and the workspace can be prepared again for the next call."""
-    w, _ = CASES["mass_ragged_rows"]
+    points (sparse and, for 128-token blocks, dense), and the workspace can be prepared again for the next call."""
+    w, _ = CASES[name]
     (qd, kd, vd), bits, rp, ci = _setup(w)
     o1, l1, st1 = U.gpu_attn(w, qd, kd, vd, rp, ci)
     od, ld, _ = U.gpu_attn(w, qd, kd, vd, None, None, dense=True)
@@ -94,7 +101,7 @@ def test_two_step_form_matches_the_one_call_form():
     p = B.make_problem(qd, kd, vd, o2, w.N, w.block)
     ws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
     side = torch.cuda.Stream()
-    for sparse in (True, False, True):
+    for sparse in ((True, False, True) if w.block == 128 else (True, True)):
         ready = torch.cuda.Event()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -129,6 +136,33 @@ def test_empty_rows_and_bad_indices_are_reported_not_trapped():
         o, lse, st = U.gpu_attn(w, *data, rp, ci3.cuda(), simt=simt)
         assert st & B.SVA_DEV_BAD_INDEX
         U.check_attn_vs_oracle(w, *bits, rp, ci, o, lse, [0, 4, 6, 15])
+
+
+def test_block64_tile_with_one_empty_query_block():
+    """64-token blocks: a tile row whose two query blocks keep different key blocks, down to one of them
+    keeping nothing, against the CUDA-core kernel and the oracle."""
+    w = shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=6)      # Nb = 32
+    data, bits, rp, ci = _setup(w)
+    rp_h, ci_h = rp.cpu().clone(), ci.cpu().clone()
+    cnt = (rp_h[1:] - rp_h[:-1]).clone()
+    keep = torch.ones_like(cnt, dtype=torch.bool)
+    keep[1::4] = False            # query block B of every other tile row keeps nothing
+    keep[6] = False; keep[7] = False   # a whole tile row without work
+    keep[8] = False               # query block A empty, B not
+    new_cnt = cnt * keep
+    rp2 = torch.zeros_like(rp_h); rp2[1:] = torch.cumsum(new_cnt, 0)
+    ci2 = torch.cat([ci_h[rp_h[r]: rp_h[r + 1]] for r in range(w.R) if keep[r]])
+    o, lse, st = U.gpu_attn(w, *data, rp2.cuda(), ci2.cuda())
+    o_s, lse_s, st_s = U.gpu_attn(w, *data, rp2.cuda(), ci2.cuda(), simt=True)
+    assert st == 0 and st_s == 0
+    for r in range(w.R):
+        bh, I = divmod(r, w.Nb)
+        sl = (bh // w.H, bh % w.H, slice(I * w.block, min((I + 1) * w.block, w.N)))
+        if not keep[r]:
+            assert (o[sl] == 0).all() and torch.isinf(lse[sl]).all() and (lse[sl] < 0).all()
+    rows = [r for r in range(w.R) if keep[r]][:24]
+    U.check_attn_vs_oracle(w, *bits, rp2, ci2, o, lse, rows)
+    assert (o.float() - o_s.float()).abs().max() < 2e-2
 
 
 def test_runs_of_empty_rows_and_no_rows_at_all():

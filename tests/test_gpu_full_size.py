@@ -11,7 +11,7 @@ from paper_2606_23743_b200.workloads import WORKLOADS
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,nrows", [("medium", 16), ("large", 16), ("xl", 12)])
+@pytest.mark.parametrize("name,nrows", [("medium", 16), ("large", 16), ("xl", 12), ("large_b64", 16)])
 def test_full_size_select_then_attend(name, nrows):
     w = WORKLOADS[name]
     (q, k, v), (qb, kb, vb) = U.host_inputs(w)
