@@ -445,24 +445,28 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           v0 = ((J >> (14 + qh)) & 1u) ? (u0 == prm.Nb - 1 ? tail_keys : 64) : 0;
           v1 = ((J >> (30 + qh)) & 1u) ? (u1 == prm.Nb - 1 ? tail_keys : 64) : 0;
         } else {
-          const int valid = ((int)J == prm.Nb - 1) ? tail_keys : BS;
-          v0 = valid < 64 ? valid : 64;
-          v1 = valid - v0;
+          v0 = ((int)J == prm.Nb - 1) ? tail_keys : BS;      // 128-token blocks: all valid keys counted in v0
+          v1 = 0;
         }
         if (j + 2 < n) J = list_block<B64>(prm, lbeg, j + 2);          // one entry ahead
         if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
         tc_fence_after();
-        if (v0 + v1 < BS) {
+        if (B64 ? (v0 + v1 < BS) : (v0 < BS)) {
           // Keys that do not exist (ragged last key block) become -inf in TMEM before S is read: a short
           // rolled loop, which keeps 128 compare/select pairs out of the hot instruction stream.  A half
           // that is not kept at all (64-token blocks) is left alone here: it is excluded below.
-          if (!B64 || v0 > 0) {
+          if (B64) {
+            if (v0 > 0) {
 #pragma unroll 1
-            for (int e = v0; e < 64; ++e) tmem_st1(s_tmem + e, 0xff800000u);
-          }
-          if (!B64 || v1 > 0) {
+              for (int e = v0; e < 64; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+            }
+            if (v1 > 0) {
 #pragma unroll 1
-            for (int e = 64 + v1; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+              for (int e = 64 + v1; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+            }
+          } else {
+#pragma unroll 1
+            for (int e = v0; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
           }
           tc_wait_st();
         }
@@ -474,18 +478,28 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
-        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;   // a, b: keys 0..63; c, d: keys 64..127
+        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+        float mx0, mx1;
+        if (B64) {                                           // a, b: keys 0..63; c, d: keys 64..127
 #pragma unroll
-        for (int e = 0; e < 64; e += 4) {
-          mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
-          mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
-          mxc = max3(mxc, __uint_as_float(sv[e + 64]), __uint_as_float(sv[e + 65]));
-          mxd = max3(mxd, __uint_as_float(sv[e + 66]), __uint_as_float(sv[e + 67]));
-        }
-        float mx0 = fmaxf(mxa, mxb), mx1 = fmaxf(mxc, mxd);
-        if (B64) {                                           // a half this query block does not keep has no say
-          if (v0 == 0) mx0 = -INFINITY;
-          if (v1 == 0) mx1 = -INFINITY;
+          for (int e = 0; e < 64; e += 4) {
+            mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+            mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+            mxc = max3(mxc, __uint_as_float(sv[e + 64]), __uint_as_float(sv[e + 65]));
+            mxd = max3(mxd, __uint_as_float(sv[e + 66]), __uint_as_float(sv[e + 67]));
+          }
+          mx0 = v0 > 0 ? fmaxf(mxa, mxb) : -INFINITY;        // a half this query block does not keep has no say
+          mx1 = v1 > 0 ? fmaxf(mxc, mxd) : -INFINITY;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 128; e += 8) {
+            mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+            mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+            mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
+            mxd = max3(mxd, __uint_as_float(sv[e + 6]), __uint_as_float(sv[e + 7]));
+          }
+          mx0 = fmaxf(mxa, mxb);
+          mx1 = fmaxf(mxc, mxd);
         }
         const float mx = fmaxf(mx0, mx1) * c;
         // reference exponent left by block j-1 (other group)
