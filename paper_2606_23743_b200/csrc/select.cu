@@ -77,7 +77,7 @@ pool_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, Stride
   }
 }
 
-static constexpr int SEL_WARPS = 16;    // query-block rows per CTA, one warp each
+static constexpr int SEL_ROWS = 16;     // query-block rows per CTA
 static constexpr int SEL_CHUNK = 32;    // key blocks staged per pass
 
 struct SelParams {
@@ -101,71 +101,28 @@ __device__ __forceinline__ float key_score(uint32_t key) {
   return __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
 }
 
-// One CTA scores and selects SEL_WARPS query-block rows of one head, one warp per row.
-// Lane j of a warp owns the key blocks J = it*32 + j, it < ITEMS, and keeps their scores in
-// registers (as sortable keys); a chunk of 32 pooled keys is staged transposed in shared memory
-// so that lane j reads key j conflict-free while the query values are 128-bit broadcasts.
-// smem: qs[SEL_WARPS][D] | ksT[D][33]
-template <int D, int ITEMS>
-__global__ void __launch_bounds__(SEL_WARPS * 32)
-score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, SelParams p,
-                    int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx,
-                    int32_t* __restrict__ tmp_idx, int32_t* __restrict__ counts,
-                    float* __restrict__ block_scores, int R) {
-  constexpr int KT_LD = SEL_CHUNK + 1;
-  __shared__ __align__(16) float qs[SEL_WARPS * D];
-  __shared__ float ksT[D * KT_LD];
+// Selection and emission of one query-block row by one warp.  Lane j owns the key blocks
+// J = it*32 + j, it < ITEMS, whose scores arrive as sortable keys (0 = no candidate).
+template <int ITEMS>
+__device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const int I, const int bh, const int lane,
+                                                const SelParams& p, int32_t* __restrict__ row_ptr,
+                                                int32_t* __restrict__ col_idx, int32_t* __restrict__ tmp_idx,
+                                                int32_t* __restrict__ counts, const int R) {
   const int Nb = p.Nb;
-  const int bh = blockIdx.y;
-  const int I0 = blockIdx.x * SEL_WARPS;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int I = I0 + warp;
-  const bool row_ok = I < Nb;
-
-  for (int i = threadIdx.x; i < SEL_WARPS * D; i += blockDim.x) {
-    int w = i / D;
-    qs[i] = (I0 + w < Nb) ? qbar[((long long)bh * Nb + I0 + w) * D + (i % D)] : 0.f;
-  }
-  const float* kb = kbar + (long long)bh * Nb * D;
-
-  uint32_t key[ITEMS];
-#pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    key[it] = 0u;
-    if (it * 32 < Nb) {                      // uniform over the CTA
-      __syncthreads();
-      const int J = it * 32 + lane;
-      for (int cc = warp; cc < D / 4; cc += SEL_WARPS) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (J < Nb) v = __ldg(reinterpret_cast<const float4*>(kb + (long long)J * D) + cc);
-        ksT[(4 * cc + 0) * KT_LD + lane] = v.x;
-        ksT[(4 * cc + 1) * KT_LD + lane] = v.y;
-        ksT[(4 * cc + 2) * KT_LD + lane] = v.z;
-        ksT[(4 * cc + 3) * KT_LD + lane] = v.w;
-      }
-      __syncthreads();
-      float a0 = 0.f, a1 = 0.f;
-#pragma unroll 8
-      for (int c = 0; c < D; c += 4) {
-        const float4 qv = *reinterpret_cast<const float4*>(qs + warp * D + c);
-        a0 = fmaf(qv.x, ksT[(c + 0) * KT_LD + lane], a0);
-        a1 = fmaf(qv.y, ksT[(c + 1) * KT_LD + lane], a1);
-        a0 = fmaf(qv.z, ksT[(c + 2) * KT_LD + lane], a0);
-        a1 = fmaf(qv.w, ksT[(c + 3) * KT_LD + lane], a1);
-      }
-      const float v = (a0 + a1) * p.scale;
-      if (J < Nb) {
-        key[it] = score_key(v);
-        if (block_scores && row_ok) block_scores[((long long)bh * Nb + I) * Nb + J] = v;
-      }
-    }
-  }
-  if (!row_ok) return;
-
   // ---- selection
+  // The rule is sequential -- forced window first, then candidates by score (descending, ties to the
+  // lower index) until k blocks are kept or, in mode 1, the kept softmax mass reaches tau -- but what it
+  // keeps is "every candidate above a threshold key plus the first few of the candidates equal to it",
+  // so the threshold is found by a 32-step bisection on the key bits (each step: one compare per
+  // register, a warp reduction of the count and, in mode 1, of the mass) instead of up to k rounds of
+  // arg-max.  Decisions agree with the round-by-round form except where the mass comes within fp32
+  // summation noise of tau.
   uint32_t mask = 0;            // bit it set <=> block it*32+lane is kept
   int n = 0;
   float cum = 0.f, mx = 0.f, inv_z = 0.f;
+  float wgt[ITEMS];             // mode 1: softmax weight of every candidate
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) wgt[it] = 0.f;
   if (p.mode == 1) {
     uint32_t km = 0u;
 #pragma unroll
@@ -175,10 +132,12 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
     float z = 0.f;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it)
-      if (key[it]) z += expf(key_score(key[it]) - mx);
+      if (key[it]) { wgt[it] = expf(key_score(key[it]) - mx); z += wgt[it]; }
 #pragma unroll
     for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
     inv_z = 1.0f / z;
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) wgt[it] *= inv_z;
   }
   if (p.use_window) {
     float fm = 0.f;
@@ -188,8 +147,9 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
       const int J = it * 32 + lane;
       if (J < Nb && in_window(I, J, p)) {
         mask |= 1u << it; ++cnt;
-        if (p.mode == 1) fm += expf(key_score(key[it]) - mx) * inv_z;
+        fm += wgt[it];
         key[it] = 0u;                        // no longer a candidate
+        wgt[it] = 0.f;
       }
     }
 #pragma unroll
@@ -200,26 +160,65 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
     n = cnt; cum = fm;
   }
   const int kk = min(p.k, Nb);
-  while (true) {
-    if (n >= kk) break;
-    if (p.mode == 1 && n >= 1 && cum >= p.tau) break;
-    // lane-local best: highest key, lowest item on ties (strict > while scanning upwards)
-    uint32_t bkey = 0u;
-    int bit = 0;
+  if (n < kk && !(p.mode == 1 && n >= 1 && cum >= p.tau)) {
+    // count and mass of the candidates with key >= t
+    auto above = [&](uint32_t t, int& cnt, float& mass) {
+      int c = 0;
+      float g = 0.f;
 #pragma unroll
-    for (int it = 0; it < ITEMS; ++it)
-      if (key[it] > bkey) { bkey = key[it]; bit = it; }
-    const uint32_t top = __reduce_max_sync(0xffffffffu, bkey);
-    if (top == 0u) break;                     // nothing selectable left
-    const uint32_t win = __reduce_min_sync(0xffffffffu, bkey == top ? (uint32_t)(bit * 32 + lane) : 0x7fffffffu);
-    if ((int)(win & 31u) == lane) {
-      mask |= 1u << (win >> 5);
+      for (int it = 0; it < ITEMS; ++it) {
+        const bool ge = key[it] >= t && key[it] != 0u;
+        c += ge;
+        if (ge) g += wgt[it];
+      }
+      cnt = (int)__reduce_add_sync(0xffffffffu, (unsigned)c);
+      if (p.mode == 1) {
 #pragma unroll
-      for (int it = 0; it < ITEMS; ++it)
-        if (it == (int)(win >> 5)) key[it] = 0u;
+        for (int o = 16; o; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+      }
+      mass = g;
+    };
+    // largest threshold at which taking every candidate >= it ends the rule (0: never -> take them all)
+    uint32_t T = 0u;
+#pragma unroll 1
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t t = T | (1u << bit);
+      int c;
+      float g;
+      above(t, c, g);
+      if (n + c >= kk || (p.mode == 1 && c >= 1 && cum + g >= p.tau)) T = t;
     }
-    ++n;
-    if (p.mode == 1) cum += expf(key_score(top) - mx) * inv_z;
+    // everything above T, then ties at T in index order while the rule still runs
+    int G;
+    float Mg;
+    above(T + 1u, G, Mg);                    // T = 0: all candidates; T = 0xffffffff cannot be reached (see below)
+    int have = n + G;
+    float acc = cum + Mg;
+    const float wT = (p.mode == 1 && T != 0u) ? expf(key_score(T) - mx) * inv_z : 0.f;
+    int ties_wanted = 0;
+    if (T != 0u) {
+      int E = 0;
+#pragma unroll
+      for (int it = 0; it < ITEMS; ++it) E += (key[it] == T);
+      E = (int)__reduce_add_sync(0xffffffffu, (unsigned)E);
+      while (ties_wanted < E) {
+        if (have >= kk) break;
+        if (p.mode == 1 && have >= 1 && acc >= p.tau) break;
+        ++ties_wanted; ++have; acc += wT;
+      }
+    }
+    int seen = 0;                            // ties met so far, in index order
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+      const bool cand = key[it] != 0u;
+      const bool gt = cand && key[it] > T;
+      const bool eq = cand && T != 0u && key[it] == T;
+      const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+      const bool take = gt || (eq && seen + __popc(bal & ((1u << lane) - 1u)) < ties_wanted);
+      if (take) mask |= 1u << it;
+      seen += __popc(bal);
+    }
+    n = have;
   }
 
   // ---- emit ascending
@@ -243,6 +242,105 @@ score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kb
     uint32_t bal = __ballot_sync(0xffffffffu, sel);
     if (sel) out[base + __popc(bal & ((1u << lane) - 1u))] = it * 32 + lane;
     base += __popc(bal);
+  }
+}
+
+// One CTA scores and selects SEL_ROWS query-block rows of one head.  A warp takes RW rows: lane j
+// owns the key blocks J = it*32 + j and accumulates the RW rows' scores of a key together, so every
+// pooled-key value read from shared memory feeds RW FMAs (the kernel is bound by shared-memory
+// reads otherwise).  A chunk of 32 pooled keys is staged transposed in shared memory (lane j reads
+// key j conflict-free, the query values are 128-bit broadcasts), double-buffered: the next chunk's
+// global loads are in flight while the current one is used.  Afterwards the warp runs the selection
+// of its rows one after the other.
+// smem: qs[SEL_ROWS][D] | ksT[2][D][33]
+template <int D, int ITEMS, int RW>
+__global__ void __launch_bounds__(SEL_ROWS / RW * 32)
+score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, SelParams p,
+                    int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx,
+                    int32_t* __restrict__ tmp_idx, int32_t* __restrict__ counts,
+                    float* __restrict__ block_scores, int R) {
+  constexpr int NW = SEL_ROWS / RW;            // warps per CTA
+  constexpr int KT_LD = SEL_CHUNK + 1;
+  constexpr int PRE = D / 4 / NW;              // float4 loads per thread and chunk
+  __shared__ __align__(16) float qs[SEL_ROWS * D];
+  __shared__ float ksT[2][D * KT_LD];
+  const int Nb = p.Nb;
+  const int bh = blockIdx.y;
+  const int I0 = blockIdx.x * SEL_ROWS;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int i = threadIdx.x; i < SEL_ROWS * D; i += blockDim.x) {
+    int w = i / D;
+    qs[i] = (I0 + w < Nb) ? qbar[((long long)bh * Nb + I0 + w) * D + (i % D)] : 0.f;
+  }
+  const float* kb = kbar + (long long)bh * Nb * D;
+
+  float4 pre[PRE];
+  auto load_chunk = [&](int it) {
+    const int J = it * 32 + lane;
+#pragma unroll
+    for (int i = 0; i < PRE; ++i) {
+      pre[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (J < Nb) pre[i] = __ldg(reinterpret_cast<const float4*>(kb + (long long)J * D) + warp + NW * i);
+    }
+  };
+  auto store_chunk = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < PRE; ++i) {
+      const int cc = warp + NW * i;
+      ksT[buf][(4 * cc + 0) * KT_LD + lane] = pre[i].x;
+      ksT[buf][(4 * cc + 1) * KT_LD + lane] = pre[i].y;
+      ksT[buf][(4 * cc + 2) * KT_LD + lane] = pre[i].z;
+      ksT[buf][(4 * cc + 3) * KT_LD + lane] = pre[i].w;
+    }
+  };
+
+  uint32_t key[RW][ITEMS];
+  load_chunk(0);
+  store_chunk(0);
+  __syncthreads();
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+#pragma unroll
+    for (int r = 0; r < RW; ++r) key[r][it] = 0u;
+    if (it * 32 < Nb) {                      // uniform over the CTA
+      const bool more = it + 1 < ITEMS && (it + 1) * 32 < Nb;
+      if (more) load_chunk(it + 1);          // in flight during the FMAs below
+      const float* kt = ksT[it & 1];
+      float a0[RW], a1[RW];
+#pragma unroll
+      for (int r = 0; r < RW; ++r) { a0[r] = 0.f; a1[r] = 0.f; }
+#pragma unroll 4
+      for (int c = 0; c < D; c += 4) {
+        const float k0 = kt[(c + 0) * KT_LD + lane], k1 = kt[(c + 1) * KT_LD + lane];
+        const float k2 = kt[(c + 2) * KT_LD + lane], k3 = kt[(c + 3) * KT_LD + lane];
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {
+          const float4 qv = *reinterpret_cast<const float4*>(qs + (warp * RW + r) * D + c);
+          a0[r] = fmaf(qv.x, k0, a0[r]);
+          a1[r] = fmaf(qv.y, k1, a1[r]);
+          a0[r] = fmaf(qv.z, k2, a0[r]);
+          a1[r] = fmaf(qv.w, k3, a1[r]);
+        }
+      }
+      const int J = it * 32 + lane;
+      if (J < Nb) {
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {
+          const float v = (a0[r] + a1[r]) * p.scale;
+          key[r][it] = score_key(v);
+          const int I = I0 + warp * RW + r;
+          if (block_scores && I < Nb) block_scores[((long long)bh * Nb + I) * Nb + J] = v;
+        }
+      }
+      if (more) store_chunk((it + 1) & 1);
+      __syncthreads();
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    const int I = I0 + warp * RW + r;
+    if (I < Nb) select_and_emit<ITEMS>(key[r], I, bh, lane, p, row_ptr, col_idx, tmp_idx, counts, R);
   }
 }
 
@@ -356,15 +454,15 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   sp.win_t = s->win_t; sp.win_s = s->win_s; sp.bpf = sp.use_window ? s->blocks_per_frame : 1;
   sp.cap = cap; sp.fixed_n = fixed_n; sp.scale = m.scale; sp.tau = s->mass;
   const int items = (m.Nb + 31) / 32;
-  dim3 sg((m.Nb + SEL_WARPS - 1) / SEL_WARPS, m.B * m.H);
-#define SVA_SEL_LAUNCH(IT)                                                                          \
-  score_select_kernel<D, IT><<<sg, SEL_WARPS * 32, 0, st>>>(qbar, kbar, sp, row_ptr, col_idx, tmp_idx, \
-                                                             counts, block_scores, m.R)
-  if (items <= 4) SVA_SEL_LAUNCH(4);
-  else if (items <= 8) SVA_SEL_LAUNCH(8);
-  else if (items <= 12) SVA_SEL_LAUNCH(12);
-  else if (items <= 16) SVA_SEL_LAUNCH(16);
-  else SVA_SEL_LAUNCH(32);
+  dim3 sg((m.Nb + SEL_ROWS - 1) / SEL_ROWS, m.B * m.H);
+#define SVA_SEL_LAUNCH(IT, RWV)                                                                     \
+  score_select_kernel<D, IT, RWV><<<sg, SEL_ROWS / RWV * 32, 0, st>>>(qbar, kbar, sp, row_ptr, col_idx, \
+                                                                       tmp_idx, counts, block_scores, m.R)
+  if (items <= 4) SVA_SEL_LAUNCH(4, 2);
+  else if (items <= 8) SVA_SEL_LAUNCH(8, 2);
+  else if (items <= 12) SVA_SEL_LAUNCH(12, 2);
+  else if (items <= 16) SVA_SEL_LAUNCH(16, 2);
+  else SVA_SEL_LAUNCH(32, 2);
 #undef SVA_SEL_LAUNCH
   if (!fixed_n) {
     scan_kernel<<<1, 1024, 0, st>>>(counts, m.R, row_ptr);
