@@ -216,7 +216,8 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     aws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
-    launches_per_step = (4 if variable_rows else 2) + 2       # routing kernels + V transpose + attention
+    # routing kernels + V transpose + attention (+ the tile-list kernel of the 64-token-block path)
+    launches_per_step = (4 if variable_rows else 2) + 2 + (1 if w.block == 64 else 0)
 
     # V is prepared (tiled transposed copy) on a second stream while routing, which never reads V, runs
     # (lower priority: its CTAs fill the SMs that the latency-bound selection kernel leaves idle instead of
