@@ -143,12 +143,11 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * (16 for e4m3 Q/K).  Tensor-core kernels (bf16 or e4m3 x e4m3 MMA, fp32 accumulate) serve d = 128:
  * bf16 Q/K with 128- or 64-token blocks, e4m3 Q/K with 128-token blocks; other supported shapes run
  * on a CUDA-core kernel.
- * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The bf16 tensor-core kernel
+ * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The tensor-core kernel
  * keeps a tiled, transposed copy of V (2*B*H*Nb*block*d bytes), its row counter and, for 64-token
  * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
  * GPU need a workspace each);
- * the size is 0 -- and the pointer may be NULL -- for the e4m3 variant and for shapes served by
- * the CUDA-core kernel.
+ * the size is 0 -- and the pointer may be NULL -- for shapes served by the CUDA-core kernel.
  */
 size_t sva_attn_workspace_bytes(const sva_problem_t* p);
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
@@ -162,7 +161,7 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * The bf16 tensor-core path in two steps, for callers that can prepare V early -- on another stream
+ * The bf16 tensor-core path in two steps (bf16 Q/K only), for callers that can prepare V early -- on another stream
  * while routing runs (routing never reads V), or because the producer of V can be made to write
  * the prepared layout itself.  sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
  * and key block one contiguous tile [d][block keys], keys >= N zero) and resets the row counter in

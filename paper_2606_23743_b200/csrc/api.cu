@@ -3,13 +3,9 @@
 
 namespace sva {
 
-void set_tiles_per_cta(int n);
 void ts_set_prof_buffer(void* p);
 void ts_set_debug_mode(int v);
 int ts_set_wait_limit(long long cycles);
-void set_prof_buffer(void* p);
-void set_debug_mode(int v);
-int set_wait_limit(long long cycles);
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -59,10 +55,9 @@ static int validate_attn(const sva_problem_t* p, const void* q, const void* k, c
   return SVA_OK;
 }
 
-// Tensor-core kernels: bf16 with d = 128 and 128- or 64-token blocks runs on the all-TMEM-A kernel
-// (attn_ts_serves; it needs the transposed-V workspace), e4m3 Q/K with 128-token blocks and d = 128 on
-// the two-tile kernel (use_sm100); other supported shapes run on the CUDA-core kernel.
-static bool use_sm100(const Dims& m) { return m.block == 128 && m.d == 128; }
+// The tensor-core kernel (attn_ts_serves: d = 128; bf16 with 128- or 64-token blocks, e4m3 Q/K with
+// 128-token blocks; it needs the transposed-V workspace) or, for the other supported shapes, the
+// CUDA-core kernel.
 
 }  // namespace sva
 
@@ -119,8 +114,6 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
                                (cudaStream_t)stream);
 }
 
-static int g_bf16_kernel = 0;   /* tuning aid: 1 routes bf16 problems to the two-tile SS/TS kernel */
-
 size_t sva_attn_workspace_bytes(const sva_problem_t* p) {
   if (validate_problem(p)) return 0;
   Dims m = make_dims(p);
@@ -135,12 +128,9 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
   if (rc) return rc;
   if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (attn_ts_serves(m) && !(g_bf16_kernel && use_sm100(m)))
-    return launch_attn_ts(m, p, q, k, v, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
+  if (attn_ts_serves(m))
+    return launch_attn_ts(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
                           (cudaStream_t)stream);
-  if (use_sm100(m))
-    return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
-                             (cudaStream_t)stream);
   return launch_attn_simt(m, p, q, k, v, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status,
                           (cudaStream_t)stream);
 }
@@ -151,12 +141,9 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
   int rc = validate_attn(p, q, k, v, q_scale, k_scale, o);
   if (rc) return rc;
   Dims m = make_dims(p);
-  if (attn_ts_serves(m) && !(g_bf16_kernel && use_sm100(m)))
-    return launch_attn_ts(m, p, q, k, v, nullptr, nullptr, o, lse, device_status, workspace, workspace_bytes,
+  if (attn_ts_serves(m))
+    return launch_attn_ts(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status, workspace, workspace_bytes,
                           (cudaStream_t)stream);
-  if (use_sm100(m))
-    return launch_attn_sm100(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status,
-                             (cudaStream_t)stream);
   return launch_attn_simt(m, p, q, k, v, q_scale, k_scale, nullptr, nullptr, o, lse, device_status,
                           (cudaStream_t)stream);
 }
@@ -170,7 +157,7 @@ int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, s
   if ((rc = check_strides(p->v_stride, 8))) return rc;
   if (p->v_stride[2] < p->d) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_serves(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
   return launch_prepare_v_ts(m, p, v, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
@@ -183,8 +170,8 @@ int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, co
   if (rc) return rc;
   if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
-  return launch_attn_ts(m, p, q, k, nullptr, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
+  if (!attn_ts_serves(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  return launch_attn_ts(m, p, q, k, nullptr, nullptr, nullptr, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
                         (cudaStream_t)stream);
 }
 
@@ -225,16 +212,13 @@ const char* sva_status_string(int status) {
   }
 }
 
-/* bring-up switch (not part of the public header): 1 or 2 query tiles per CTA */
-void sva_debug_set_tiles_per_cta(int n) { set_tiles_per_cta(n); }
-/* tuning aid: 1 sends bf16 problems to the two-tile kernel that otherwise serves e4m3 (A/B timing) */
-void sva_debug_set_bf16_kernel(int v) { g_bf16_kernel = v; }
-/* tuning aid: device buffer of 5*8*8 int64 that CTA 64 fills with a clock64 timeline; NULL = off */
-void sva_debug_set_prof_buffer(void* p) { set_prof_buffer(p); ts_set_prof_buffer(p); }
-/* tuning aid: bit0 skips the softmax arithmetic (results are wrong; timing of the MMA side only) */
-void sva_debug_set_mode(int v) { set_debug_mode(v); ts_set_debug_mode(v); }
-/* test aid: cycles a device-side wait may last before the CTA gives up (<= 0 restores the default);
-   mode bit 16 starves tile 0 of its K tiles so that this limit is reached */
-int sva_debug_set_wait_limit(long long cycles) { return set_wait_limit(cycles) | ts_set_wait_limit(cycles); }
+/* tuning aid (not part of the public header): device buffer of 320 int64; entry 319 receives the longest
+   CTA's cycle count of the next attention launches; NULL = off */
+void sva_debug_set_prof_buffer(void* p) { ts_set_prof_buffer(p); }
+/* bit 0 skips the exponentials (tuning aid: results are wrong); bit 4 (test aid) withholds a row's K
+   tiles after the first so that a bounded wait runs out */
+void sva_debug_set_mode(int v) { ts_set_debug_mode(v); }
+/* test aid: cycles a device-side wait may last before the CTA gives up (<= 0 restores the default) */
+int sva_debug_set_wait_limit(long long cycles) { return ts_set_wait_limit(cycles); }
 
 }  // extern "C"

@@ -1,442 +1,659 @@
-// Block-sparse / dense attention forward for sm_100a: TMA-staged tiles gathered by block
-// index, tcgen05 MMAs with TMEM accumulators for Q K^T and P V, warp-specialised roles,
-// online softmax in registers.  (Paper: critical blocks "computed exactly"; dense fallback.)
+// Block-sparse / dense attention forward for sm_100a (tcgen05 / TMEM / TMA): every MMA of one form.
+// (Paper: critical blocks "computed exactly"; dense fallback.)
 //
-// One CTA owns NT query tiles (NT adjacent query blocks of one head, 128 rows each).
-//   warps [0, 4*NT)   softmax: warpgroup t owns tile t, thread <-> query row (TMEM lane)
-//   warp  4*NT        producer: one lane issues every TMA load (Q once, then K/V tiles)
-//   warp  4*NT + 1    MMA: one lane issues every tcgen05.mma and commit; owns TMEM alloc
-// TMEM columns (fp32): S_t at 128*t, O_t at 128*NT + 128*t; P_t (bf16 pairs) overlays the
-// first 64 columns of S_t and feeds the P V MMA as the A operand straight from TMEM.
-// Per tile and kept block j: S = Q K_j^T -> softmax warpgroup: row max, lazy rescale of O,
-// P = exp2(S*c - m) -> O += P V_j.  With NT = 2 the tensor pipe works on one tile while the
-// other tile's softmax runs.
+// The tensor pipe drains (~280 cycles, measured) whenever two consecutive MMAs differ in kind:
+// A operand from shared memory vs tensor memory, or another instruction descriptor.  Here both
+// S = Q K^T and O += P V have the same form -- A from TENSOR memory (Q resp. P, bf16 pairs), B
+// from shared memory, K-major, M = N = 128 -- so the pipe never drains:
+//   * Q is written into TMEM once per row by the softmax threads (straight from global memory);
+//   * V is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed copy
+//     that a small kernel writes into the caller's workspace first.
+// The kernel is persistent: CTA c processes the CSR rows c, c + gridDim.x, ... (one row = one query
+// block of one head, 128 query rows).  All barriers keep running across rows (every role derives the
+// same phase counters from the same row sequence), so the producers run ahead into the next row
+// while the softmax groups finish the current one.
+//   warps 0-3, 4-7  two softmax warpgroups; they take the kept key blocks alternately (even / odd
+//                   position in the row's list); thread <-> query row <-> TMEM lane
+//   warp  8         producer of the K tiles (TMA, one lane)
+//   warp  9         issues the Q K^T MMAs (one lane); owns the TMEM allocation
+//   warp  10        issues the P V MMAs (one lane)
+//   warp  11        producer of the V^T tiles (TMA, one lane)
+// TMEM columns: S of even blocks 0..127, S of odd blocks 128..255, O 256..383, Q 384..447 (bf16
+// pairs), P 448..511 (bf16 pairs).  Because P has columns of its own, an S buffer is free again as
+// soon as its warpgroup has read it into registers: the MMA warp computes S(j+2) while the softmax
+// of block j is still running.  P is single-buffered: block j's P is stored once P V(j-1) has
+// completed, which also staggers the two warpgroups so that one group's exponentials overlap the
+// other group's maximum pass and stores.
 //
-// Every wait is bounded: when one expires the CTA sets SVA_DEV_TIMEOUT, all roles leave
-// their loops, TMEM is released and the kernel returns.
+// The two warpgroups share one O accumulator, so they share the reference exponent of every row:
+// the group working on block j takes the reference left by block j-1 (published through shared
+// memory right after that block's row-maximum pass), raises it only when the new row maximum
+// exceeds it by more than 2^LAZY_LOG2, and in that (rare) case rescales its row of O once P V(j-1)
+// has completed.  Row sums are kept per group and merged in the epilogue, where each group
+// normalises its half of O into a swizzled staging panel that one TMA tile store writes out.
+//
+// e4m3 Q/K (template switch): Q goes into TMEM as bytes (32 columns), a K tile is one 128 x 128-byte
+// panel, S takes four kind::f8f6f4 MMAs (A from TMEM like everything else), and the exponent's scale is
+// softmax_scale * q_scale[query block] * k_scale[key block] per block; P, V and O stay bf16 / fp32.
+//
+// 64-token blocks (template switch): the MMA tile stays 128 x 128, so one row of work is two adjacent
+// query blocks (A, B) and one tile two key blocks out of the ascending union of A's and B's lists
+// (pair_lists_kernel builds the tile lists).  The K / V^T producers fetch the two halves of a tile
+// from two key blocks; the softmax excludes, per query block, the half it does not keep -- with -inf
+// as the additive constant of the exponentials' FMA, at no cost -- and masks a ragged tail per half.
+// The price is the part of the union one of the two query blocks does not keep (adjacent query
+// blocks share most of their lists).
+//
+// Every wait is bounded: when one expires the CTA sets SVA_DEV_TIMEOUT, all roles leave their
+// loops, TMEM is released and the kernel returns.  Parity waits never run a whole phase ahead of
+// their barrier (each wait on a barrier is preceded by a wait on its previous phase).
 #include "tc_ptx.cuh"
 
 namespace sva {
 
-struct AttnParams {
+struct TsParams {
+  const __nv_bfloat16* q;     // e4m3 variant: bytes (strides in elements either way)
+  Strides sq;
+  const float* q_scale;       // e4m3 variant: one scale per (b, h, block) for Q and for K
+  const float* k_scale;
   const int32_t* row_ptr;     // null = dense
   const int32_t* col_idx;
-  const float* q_scale;       // fp8 only
-  const float* k_scale;
   __nv_bfloat16* o;
   float* lse;
   int32_t* status;
   Strides so;
-  int H, N, Nb, R;
+  int H, N, Nb, R;            // Nb: key blocks per head; R: rows handed out (128-query tiles)
+  int Nt;                     // 128-query tiles per head (= Nb for 128-token blocks, ceil(Nb/2) for 64-token blocks)
+  const int32_t* tile_cnt;    // 64-token blocks only: per tile row, number of 128-key tiles ...
+  const int32_t* tile_beg;    // ... and where its descriptors start
+  const uint32_t* tile_desc;  // two 16-bit halves {key block (14 bits), kept by query block A, kept by B}
   float scale_log2;           // softmax_scale * log2(e)
-  long long* prof;            // optional timeline buffer (tuning aid), normally null
-  int debug;                  // tuning aid: bit0 = skip the softmax arithmetic (wrong results)
+  int32_t* next_row;          // device counter (starts at 0): the next CSR row to hand out
+  long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
+  int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
+                              // bit4: starve the pipeline so that a wait runs out (test aid)
 };
 
-// Timeline probe: CTA 64 records clock64() for iterations 16..23, [role][j-16][event].
-#define SVA_PROF(role, j, ev)                                                                   \
-  do {                                                                                          \
-    if (prm.prof && blockIdx.x == 64 && (j) >= 16 && (j) < 24)                                  \
-      prm.prof[(((role) * 8) + ((j) - 16)) * 8 + (ev)] = clock64();                             \
-  } while (0)
+namespace ts {
+constexpr int D = 128;
+constexpr int TILE = BS * D * 2;            // one bf16 tile: 32 KB
+constexpr int KS = 2;                       // K tiles in flight
+constexpr int VS = 3;                       // V^T tiles in flight
+constexpr int THREADS = 384;
+constexpr int QD = 4;                       // depth of the row queue
+constexpr int OFF_K = 0;
+constexpr int OFF_V = OFF_K + KS * TILE;
+constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][128 B] panels (one per softmax group)
+constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
+constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers, reference exponents, row sums (two rows), row queue
+constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;      // + alignment slack
+constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
+// The reference exponent of a row is raised only when a block's maximum exceeds it by more than this
+// many powers of two.  P then reaches at most 2^32 and a row sum 2^32 * N: far inside fp32 (and bf16
+// has fp32's exponent range), while raises -- each one a pass over the row's O accumulator -- become rare.
+constexpr float LAZY_LOG2 = 32.0f;
+}  // namespace ts
 
-template <int D, int NT, bool F8>
-struct Cfg {
-  static constexpr int QK_ELEM = F8 ? 1 : 2;
-  static constexpr int Q_BYTES = BS * D * QK_ELEM;       // one Q (or K) tile
-  static constexpr int VH_BYTES = (BS / 2) * D * 2;      // half a V tile: 64 keys
-  static constexpr int K_SLOT = BS * D * 2;              // slot size of a K tile (bf16 size also for e4m3)
-  static constexpr int KS = NT == 2 ? 1 : 2;             // K tiles in flight per query tile
-  static constexpr int VS = NT == 2 ? 3 : 6;             // V half-tiles in flight per query tile
-  static constexpr int THREADS = NT * 128 + 128;         // softmax warpgroups + one warpgroup for TMA/MMA
-  static constexpr int TMEM_COLS = 512;
-  // dynamic shared memory: 1024-aligned tiles first, then the control block
-  static constexpr int OFF_Q = 0;
-  static constexpr int Q_SLOT = (Q_BYTES + 1023) / 1024 * 1024;
-  static constexpr int OFF_K = OFF_Q + NT * Q_SLOT;      // K slots of tile t at OFF_K + t*KS*K_SLOT
-  static constexpr int OFF_V = OFF_K + NT * KS * K_SLOT; // V half slots of tile t at OFF_V + t*VS*VH_BYTES
-  static constexpr int OFF_CTRL = OFF_V + NT * VS * VH_BYTES;
-  static constexpr int CTRL_BYTES = 384;
-  static constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;   // + alignment slack
-};
+// control block (bytes from OFF_CTRL):
+//   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
+//   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
+//   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
+//   3328 row queue: QD entries {row, count, start, first entry, second entry, -, -, -} | 3456 rq_full[QD] | 3488 rq_empty[QD]
 
-// control block layout (bytes from OFF_CTRL):
-//   0   q_full[2]   16 s_full[2]   32 p_full[t] at 32 + 16*t   64 o_done[2]
-//   96 + 128*t : k_full[2] | +16 k_empty[2] | +32 v_full[6] | +80 v_empty[6]
-//   352 tmem_base   356 abort   360 n_list[2]   368 beg[2]   376 issue lock
+// Work list of row r (a 128-query tile): count and start.  128-token blocks: the CSR row itself (a corrupt
+// row_ptr pair gives an empty row).  64-token blocks: the tile row's list of 128-key tiles that
+// pair_lists_kernel built from the two CSR rows of the tile.  Every role calls this with the same
+// inputs and so reaches the same answer.
+template <bool B64>
+__device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int& beg) {
+  if (B64) { n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r); return; }
+  if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return; }
+  beg = __ldg(prm.row_ptr + r);
+  n = __ldg(prm.row_ptr + r + 1) - beg;
+  if (n < 0 || n > prm.Nb || beg < 0) n = 0;
+}
+// Entry j of a work list.  128-token blocks: the key block (an out-of-range entry is replaced by block 0;
+// the producer reports it).  64-token blocks: the tile descriptor.
+template <bool B64>
+__device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j) {
+  if (B64) return __ldg(prm.tile_desc + beg + j);
+  if (prm.row_ptr == nullptr) return (uint32_t)j;
+  const int J = __ldg(prm.col_idx + beg + j);
+  return (J < 0 || J >= prm.Nb) ? 0u : (uint32_t)J;
+}
 
-template <int D, int NT, bool F8>
-__global__ void __launch_bounds__(NT * 128 + 128, 1)
-attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const AttnParams prm) {
-  using C = Cfg<D, NT, F8>;
+// Persistent kernel.  Rows are handed out in their natural order from one device-wide counter (so the
+// CTAs work on neighbouring rows at any time -- their K/V tiles share the L2 -- and rows of unequal
+// length balance by themselves): the K producer, which runs furthest ahead, draws the next row,
+// zero-fills it if its list is empty, and otherwise publishes {row, count, start, first two entries}
+// in a small shared-memory queue that every other role reads in the same order.  All barriers keep running across rows, so the producers and the S
+// issuer run ahead into the next row while the softmax groups finish the current one.
+template <bool B64, bool F8>
+__global__ void __launch_bounds__(384, 1)
+attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
+               const __grid_constant__ CUtensorMap tm_o, const TsParams prm) {
+  using namespace ts;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
-  uint8_t* ctrl = smem + C::OFF_CTRL;
-  const uint32_t cbase = sbase + C::OFF_CTRL;
-  const uint32_t bar_q_full = cbase + 0, bar_s_full = cbase + 16, bar_p_half = cbase + 32,
-                 bar_o_done = cbase + 64, bar_tile = cbase + 96;
-  volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 352);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 356);
-  volatile int* n_list = reinterpret_cast<volatile int*>(ctrl + 360);
-  volatile int* beg_list = reinterpret_cast<volatile int*>(ctrl + 368);
+  uint8_t* ctrl = smem + OFF_CTRL;
+  const uint32_t cb = sbase + OFF_CTRL;
+  const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
+                 bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
+                 bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
+                 bar_ost = cb + 224, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
+  volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
+  volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
+  volatile float* lx = reinterpret_cast<volatile float*>(ctrl + 1280);      // [2][2][128]
+  volatile int* rowq = reinterpret_cast<volatile int*>(ctrl + 3328);        // [QD][8]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int W_PROD = 4 * NT, W_MMA = 4 * NT + 2;   // producers: W_PROD + t; MMA issuers: W_MMA + t
-  const int row0 = blockIdx.x * NT;                    // first CSR row of this CTA
-  const int Nb = prm.Nb;
-  const bool dense = prm.row_ptr == nullptr;
+  const int Nb = prm.Nt;             // row index arithmetic: rows per head
+  constexpr int KB = B64 ? 64 : BS;  // tokens per key block
 
   // ---------------------------------------------------------------- set-up
+  const long long t_cta0 = prm.prof ? clock64() : 0;
   if (threadIdx.x == 0) {
-    for (int t = 0; t < 2; ++t) {
-      mbar_init(bar_q_full + 8 * t, 1);
-      mbar_init(bar_s_full + 8 * t, 1);
-      mbar_init(bar_p_half + 16 * t, 128);
-      mbar_init(bar_p_half + 16 * t + 8, 128);
-      mbar_init(bar_o_done + 8 * t, 1);
+    mbar_init(bar_q_ready, 256);
+    mbar_init(bar_o_free, 256);
+    mbar_init(bar_xch, 256);
+    for (int w = 0; w < 2; ++w) {
+      mbar_init(bar_s_full + 8 * w, 1);
+      mbar_init(bar_p_full + 8 * w, 128);
+      mbar_init(bar_pv_done + 8 * w, 1);
+      mbar_init(bar_ref + 8 * w, 128);
+      mbar_init(bar_s_free + 8 * w, 128);
+      mbar_init(bar_ost + 8 * w, 128);
     }
-    for (int s = 0; s < 32; ++s) mbar_init(bar_tile + 8 * s, 1);      // k/v full and empty, both tiles
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(bar_k_full + 8 * s, 1);
+      mbar_init(bar_k_empty + 8 * s, 1);
+      mbar_init(bar_v_full + 8 * s, 1);
+      mbar_init(bar_v_empty + 8 * s, 1);
+    }
+    for (int i = 0; i < QD; ++i) {
+      mbar_init(bar_rq_full + 8 * i, 1);
+      mbar_init(bar_rq_empty + 8 * i, 11);       // 3 producer / issuer lanes + one lane of each softmax warp
+    }
     *abort_flag = 0;
-    *reinterpret_cast<volatile int*>(ctrl + 376) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == W_PROD && lane == 0) {
-    prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-  }
-  if (warp == W_MMA) {
+  if (warp == 8 && lane == 0) prefetch_tmap(&tm_k);
+  if (warp == 11 && lane == 0) prefetch_tmap(&tm_vt);
+  if (warp == 0 && lane == 0) prefetch_tmap(&tm_o);
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(cbase + 352), "r"((uint32_t)C::TMEM_COLS) : "memory");
+                 ::"r"(cb + 216), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  // warp 4t validates the CSR row of tile t; a row holding a bad entry is treated as empty
-  if (warp < 4 * NT && (warp & 3) == 0) {
-    const int t = warp >> 2;
-    const int r = row0 + t;
-    int n = 0, beg = 0;
-    if (r < prm.R) {
-      if (dense) {
-        n = Nb;
-      } else {
-        beg = prm.row_ptr[r];
-        const int end = prm.row_ptr[r + 1];
-        bool bad = end < beg || end - beg > Nb || beg < 0;
-        if (!bad) {
-          for (int base = beg; base < end; base += 32) {
-            const int e = base + lane;
-            const int J = e < end ? __ldg(prm.col_idx + e) : 0;
-            bad |= (J < 0 || J >= Nb);
-          }
-        }
-        bad = __any_sync(0xffffffffu, bad);
-        if (bad) {
-          if (lane == 0 && prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX);
-        } else {
-          n = end - beg;
-        }
-      }
-    }
-    if (lane == 0) { n_list[t] = n; beg_list[t] = beg; }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_p;
-  int nl[2];
-  nl[0] = n_list[0];
-  nl[1] = NT == 2 ? n_list[1] : 0;
-  int lbeg[2];
-  lbeg[0] = beg_list[0];
-  lbeg[1] = NT == 2 ? beg_list[1] : 0;
+  constexpr uint32_t IDESC = instr_desc(128, 128, 1, false);   // bf16 x bf16 -> fp32, A and B K-major
+  constexpr uint32_t IDESC_QK = F8 ? instr_desc(128, 128, 0, false) : IDESC;   // e4m3 x e4m3 for S in the e4m3 variant
+  constexpr int KTILE = F8 ? TILE / 2 : TILE;                  // bytes of one K tile
+  constexpr int PANEL16 = (BS * 128) >> 4;                      // one 128-row x 128-byte panel
 
-  // Register re-partition: the TMA/MMA warpgroup needs few registers, a softmax thread holds a
-  // whole 128-wide row.  Issued at the top of each branch so the limit is tied to that branch.
-  if (warp >= 4 * NT) {
-    if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
-    if (warp >= W_PROD && warp < W_PROD + NT) {
-      // ---------------------------------------------------------- producer of tile t
-      // lane 0 streams Q and the K tiles, lane 1 the V half-tiles (64 keys each); the two streams
-      // have their own slots and barriers so that V runs a whole block ahead.
-      const int t = warp - W_PROD;
-      const int n = nl[t];
-      const int bh_t = (row0 + t) / Nb;
-      const int hh = bh_t % prm.H, bb = bh_t / prm.H;
-      const uint32_t bt = bar_tile + 128 * t;
-      if (lane == 0 && n > 0) {
-        const int I = (row0 + t) % Nb;
-        mbar_expect_tx(bar_q_full + 8 * t, C::Q_BYTES);
-        const uint32_t qdst = sbase + C::OFF_Q + t * C::Q_SLOT;
-        tma_load_4d(qdst, &tm_q, bar_q_full + 8 * t, 0, I * BS, hh, bb);
-        if (!F8 && D == 128) tma_load_4d(qdst + C::Q_BYTES / 2, &tm_q, bar_q_full + 8 * t, 64, I * BS, hh, bb);
-        int ks = 0;
-        uint32_t kphase = 0;
-        for (int j = 0; j < n; ++j) {
-          if ((prm.debug & 16) && t == 0 && j >= 1) break;   // test aid: starve the pipeline so that a wait runs out
-          if (!mbar_wait(bt + 16 + 8 * ks, kphase ^ 1u, abort_flag, prm.status)) break;
-          const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
-          const uint32_t dst = sbase + C::OFF_K + (t * C::KS + ks) * C::K_SLOT;
-          const uint32_t bar = bt + 8 * ks;
-          mbar_expect_tx(bar, C::Q_BYTES);
-          tma_load_4d(dst, &tm_k, bar, 0, J * BS, hh, bb);
-          if (!F8 && D == 128) tma_load_4d(dst + C::Q_BYTES / 2, &tm_k, bar, 64, J * BS, hh, bb);
-          if (++ks == C::KS) { ks = 0; kphase ^= 1u; }
-        }
-      } else if (lane == 1 && n > 0) {
-        int vs = 0;
-        uint32_t vphase = 0;
-        for (int i = 0; i < 2 * n; ++i) {
-          if (!mbar_wait<60>(bt + 80 + 8 * vs, vphase ^ 1u, abort_flag, prm.status)) break;
-          const int J = dense ? (i >> 1) : __ldg(prm.col_idx + lbeg[t] + (i >> 1));
-          const uint32_t dst = sbase + C::OFF_V + (t * C::VS + vs) * C::VH_BYTES;
-          const uint32_t bar = bt + 32 + 8 * vs;
-          mbar_expect_tx(bar, C::VH_BYTES);
-          tma_load_4d(dst, &tm_v, bar, 0, J * BS + (i & 1) * (BS / 2), hh, bb);
-          if (D == 128) tma_load_4d(dst + C::VH_BYTES / 2, &tm_v, bar, 64, J * BS + (i & 1) * (BS / 2), hh, bb);
-          if (++vs == C::VS) { vs = 0; vphase ^= 1u; }
-        }
-      }
-    } else if (warp >= W_MMA && warp < W_MMA + NT) {
-      // ---------------------------------------------------------- MMA issuer of tile t (one lane)
-      // Per block j: P V (two V half-tiles), then S(j+1).  Each issuer blocks only on its own
-      // tile's barriers; a lock taken around every group of MMAs makes the two tiles' groups
-      // reach the tensor pipe one after the other, which keeps the two softmax warpgroups out of
-      // phase (so that one tile's exponentials overlap the other tile's MMAs).
-      const int t = warp - W_MMA;
-      if (lane == 0 && nl[t] > 0) {
-        const uint32_t IDESC_QK = instr_desc(128, BS, F8 ? 0 : 1, false);
-        const uint32_t IDESC_PV = instr_desc(128, D, 1, true);
-        constexpr int QK_KSTEPS = D * C::QK_ELEM / 32;              // 32 bytes of K per MMA
-        const int n = nl[t];
-        int* lock = reinterpret_cast<int*>(ctrl + 376);
-        const uint32_t bt = bar_tile + 128 * t;
-        const uint64_t qd = smem_desc(sbase + C::OFF_Q + t * C::Q_SLOT, 16, 1024);
-        const uint64_t kdesc0 = smem_desc(sbase + C::OFF_K + t * C::KS * C::K_SLOT, 16, 1024);
-        // V half-tile: two 64-wide d panels of 64 keys x 128 bytes, panel stride = half of the slot
-        const uint64_t vdesc0 = smem_desc(sbase + C::OFF_V + t * C::VS * C::VH_BYTES, C::VH_BYTES / 2, 1024);
-        const uint32_t s_tmem = tmem_base + 128 * t;
-        const uint32_t o_tmem = tmem_base + 128 * NT + 128 * t;
-        int ks = 0, vs = 0;
-        uint32_t kphase = 0, vphase = 0;
-        auto acquire = [&]() -> bool {
-          if (NT == 1 || (prm.debug & 8)) return true;
-          uint32_t spins = 0;
-          const long long t0 = clock64();
-          while (atomicCAS(lock, 0, 1) != 0) {
-            if ((++spins & 63u) == 0u) {
-              if (*abort_flag) return false;
-              if (clock64() - t0 > g_wait_limit) {
-                *abort_flag = 1;
-                if (prm.status) atomicOr(prm.status, SVA_DEV_TIMEOUT);
-                return false;
-              }
+  // Entry i of the row sequence (the same for every role): false when a wait ran out.  r >= R ends the
+  // sequence.  `arrive` tells whether this thread signs the entry off (one thread per consumer).
+  auto fetch_row = [&](uint32_t i, int& r, int& n, int& beg, uint32_t& e0, uint32_t& e1, bool arrive) -> bool {
+    const uint32_t slot = i % QD;
+    if (!mbar_wait(bar_rq_full + 8 * slot, (i / QD) & 1u, abort_flag, prm.status)) return false;
+    r = rowq[8 * slot];
+    n = rowq[8 * slot + 1];
+    beg = rowq[8 * slot + 2];
+    e0 = (uint32_t)rowq[8 * slot + 3];
+    e1 = (uint32_t)rowq[8 * slot + 4];
+    if (warp < 8) __syncwarp();                  // softmax warps: every lane has read the entry before lane 0 signs
+    if (arrive) mbar_arrive(bar_rq_empty + 8 * slot);
+    return true;
+  };
+
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
+    if (warp == 8) {
+      // ---------------------------------------------------------- K producer (one lane)
+      if (lane == 0) {
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (uint32_t i = 0; ok; ++i) {
+          // ---- row scheduling: draw the next row with a non-empty list and publish it
+          const uint32_t slot = i % QD;
+          if (i >= QD && !mbar_wait(bar_rq_empty + 8 * slot, (i / QD - 1u) & 1u, abort_flag, prm.status)) break;
+          int r, n = 0, beg = 0;
+          for (;;) {
+            r = atomicAdd(prm.next_row, 1);
+            if (r >= prm.R) break;
+            row_list<B64>(prm, r, n, beg);
+            if (n > 0) break;
+            // nothing kept (or a corrupt row_ptr pair): zeros and lse = -inf; rare, so this one lane does it
+            const int I = r % Nb, bh0 = r / Nb;
+            for (int t = 0; t < BS; ++t) {
+              const int qi = I * BS + t;
+              if (qi >= prm.N) break;
+              __nv_bfloat16* orow = prm.o + (long long)(bh0 / prm.H) * prm.so.b + (long long)(bh0 % prm.H) * prm.so.h +
+                                    (long long)qi * prm.so.n;
+              for (int cc = 0; cc < D; cc += 8) *reinterpret_cast<uint4*>(orow + cc) = make_uint4(0, 0, 0, 0);
+              if (prm.lse) prm.lse[(long long)bh0 * prm.N + qi] = -INFINITY;
             }
           }
-          return true;
-        };
-        auto release = [&]() { if (NT == 2 && !(prm.debug & 8)) atomicExch(lock, 0); };
-        auto issue_s = [&](int j) {                                  // K(j) must be resident
-          const uint64_t kd = kdesc0 + (uint64_t)(ks * (C::K_SLOT >> 4));
+          uint32_t e0 = 0u, e1 = 0u;
+          if (r < prm.R) { e0 = list_block<B64>(prm, beg, 0); if (n > 1) e1 = list_block<B64>(prm, beg, 1); }
+          rowq[8 * slot] = r;
+          rowq[8 * slot + 1] = n;
+          rowq[8 * slot + 2] = beg;
+          rowq[8 * slot + 3] = (int)e0;
+          rowq[8 * slot + 4] = (int)e1;
+          mbar_arrive(bar_rq_full + 8 * slot);
+          if (r >= prm.R) break;
+          // ---- K tiles of the row
+          const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          for (int j = 0; j < n; ++j) {
+            if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
+            if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+            const uint32_t dst = sbase + OFF_K + s * TILE;
+            mbar_expect_tx(bar_k_full + 8 * s, KTILE);
+            if (B64) {
+              // two 64-key blocks side by side: rows 0..63 and 64..127 of both d-panels
+              const uint32_t dsc = __ldg(prm.tile_desc + beg + j);
 #pragma unroll
-          for (int kk = 0; kk < QK_KSTEPS; ++kk) {
-            constexpr int PANEL16 = (BS * 128) >> 4;
-            const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
-            tc_mma_ss<F8>(s_tmem, qd + off, kd + off, IDESC_QK, kk > 0 ? 1u : 0u, 1u);
+              for (int h = 0; h < 2; ++h) {
+                const int J = (int)((dsc >> (16 * h)) & 0x3fffu);
+                tma_load_4d(dst + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 0, J * KB, hh, bb);
+                tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 64, J * KB, hh, bb);
+              }
+            } else {
+              int J = j;
+              if (prm.row_ptr) {
+                J = __ldg(prm.col_idx + beg + j);
+                if (J < 0 || J >= prm.Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
+              }
+              tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);      // e4m3: the whole tile (128 x 128 bytes)
+              if (!F8) tma_load_4d(dst + TILE / 2, &tm_k, bar_k_full + 8 * s, 64, J * BS, hh, bb);
+            }
+            if (++s == KS) { s = 0; ph ^= 1u; }
           }
-          tc_commit(bt + 16 + 8 * ks, 1u);
-          tc_commit(bar_s_full + 8 * t, 1u);
-          SVA_PROF(2 + t, j - 1, 5);
-          if (++ks == C::KS) { ks = 0; kphase ^= 1u; }
-        };
-        auto issue_pv_half = [&](int j, int half) {                  // V half-tile vs must be resident
-          const uint64_t vd = vdesc0 + (uint64_t)(vs * (C::VH_BYTES >> 4));
-#pragma unroll
-          for (int kk = 0; kk < BS / 32; ++kk)
-            tc_mma_ts(o_tmem, s_tmem + 8 * (kk + half * (BS / 32)), vd + (uint64_t)(kk * (2048 >> 4)), IDESC_PV,
-                      (j > 0 || half > 0 || kk > 0) ? 1u : 0u, 1u);
-          tc_commit(bt + 80 + 8 * vs, 1u);
-          if (++vs == C::VS) { vs = 0; vphase ^= 1u; }
-        };
-        bool ok = mbar_wait(bar_q_full + 8 * t, 0, abort_flag, prm.status) &&
-                  mbar_wait(bt + 8 * ks, kphase, abort_flag, prm.status);
-        if (ok) {
-          tc_fence_after();
-          ok = acquire();
-          if (ok) { issue_s(0); release(); }
         }
-        for (int j = 0; j < n && ok; ++j) {
-          // One group per block: P V (two V half-tiles) directly followed by S of the next block.
-          // The tensor pipe drains whenever consecutive MMAs change kind (A from shared memory
-          // vs tensor memory, or another instruction descriptor), so kinds are kept together and
-          // the other tile's group never lands in the middle.
-          const bool more = j + 1 < n;
-          int vs2 = vs + 1;
-          uint32_t vphase2 = vphase;
-          if (vs2 == C::VS) { vs2 = 0; vphase2 ^= 1u; }
-          ok = mbar_wait(bar_p_half + 16 * t, (uint32_t)(j & 1), abort_flag, prm.status) &&
-               mbar_wait(bt + 32 + 8 * vs, vphase, abort_flag, prm.status) &&
-               mbar_wait(bt + 32 + 8 * vs2, vphase2, abort_flag, prm.status);
-          if (!ok) break;
-          SVA_PROF(2 + t, j, 1);
-          tc_fence_after();
-          ok = acquire();
-          if (!ok) break;
-          SVA_PROF(2 + t, j, 0);
-          issue_pv_half(j, 0);
-          issue_pv_half(j, 1);
-          if (j == n - 1) tc_commit(bar_o_done + 8 * t, 1u);
-          SVA_PROF(2 + t, j, 2);
-          if (more && !mbar_test(bt + 8 * ks, kphase)) {
-            // K(j+1) has not landed yet: let the other tile use the pipe meanwhile
-            release();
-            ok = mbar_wait(bt + 8 * ks, kphase, abort_flag, prm.status) && acquire();
-            if (!ok) break;
+      }
+    } else if (warp == 11) {
+      // ---------------------------------------------------------- V^T producer (one lane)
+      // tile J of head (b,h): 128 d-rows x 128 keys, contiguous 32 KB, two 64-key panels
+      if (lane == 0) {
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
+          const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          for (int j = 0; j < n; ++j) {
+            if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+            const uint32_t e = list_block<B64>(prm, beg, j);
+            const uint32_t dst = sbase + OFF_V + s * TILE;
+            mbar_expect_tx(bar_v_full + 8 * s, TILE);
+            if (B64) {
+              // each 64-key panel of the tile is one key block's transposed V: [128 d rows][64 keys]
+              tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)(e & 0x3fffu) * D, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 0, (int)((e >> 16) & 0x3fffu) * D, hh, bb);
+            } else {
+              tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)e * BS, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, (int)e * BS, hh, bb);
+            }
+            if (++s == VS) { s = 0; ph ^= 1u; }
           }
-          if (more) issue_s(j + 1);
-          release();
+        }
+      }
+    } else if (warp == 9) {
+      // ---------------------------------------------------------- S issuer (one lane)
+      // per row: S(0), S(1), then S(j) into the buffer of S(j-2) as soon as that block's softmax
+      // has read it; the first S of a row also needs the row's Q in TMEM
+      if (lane == 0) {
+        const uint64_t kd0 = smem_desc(sbase + OFF_K, 16, 1024);
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t cs[2] = {0, 0};            // S tiles issued so far into buffer w
+        bool ok = true;
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
+          ok = mbar_wait(bar_q_ready, i & 1u, abort_flag, prm.status);
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            if (cs[w] > 0) {
+              ok = mbar_wait(bar_s_free + 8 * w, (cs[w] - 1u) & 1u, abort_flag, prm.status);
+              if (!ok) break;
+            }
+            ok = mbar_wait(bar_k_full + 8 * s, ph, abort_flag, prm.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t kd = kd0 + (uint64_t)(s * (TILE >> 4));
+            if (F8) {
+#pragma unroll
+              for (int kk = 0; kk < D / 32; ++kk)               // 32 e4m3 values (32 bytes, 8 TMEM columns) per step
+                tc_mma_ts<true>(tmem_base + 128 * w, tmem_base + COL_Q + 8 * kk, kd + (uint64_t)(kk * 2), IDESC_QK,
+                                kk > 0 ? 1u : 0u, 1u);
+            } else {
+#pragma unroll
+              for (int kk = 0; kk < D / 16; ++kk) {
+                const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+                tc_mma_ts(tmem_base + 128 * w, tmem_base + COL_Q + 8 * kk, kd + off, IDESC, kk > 0 ? 1u : 0u, 1u);
+              }
+            }
+            tc_commit(bar_k_empty + 8 * s, 1u);
+            tc_commit(bar_s_full + 8 * w, 1u);
+            ++cs[w];
+            if (++s == KS) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    } else {
+      // ---------------------------------------------------------- P V issuer (one lane)
+      if (lane == 0) {
+        const uint64_t vd0 = smem_desc(sbase + OFF_V, 16, 1024);
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t cp[2] = {0, 0};            // P V groups issued so far for parity w
+        bool ok = true;
+        for (uint32_t i = 0; ok; ++i) {
+          int r, n, beg;
+          uint32_t e0, e1;
+          if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
+          // the first P V of a row overwrites O: the previous row's O must have been read
+          if (i > 0) ok = mbar_wait(bar_o_free, (i - 1u) & 1u, abort_flag, prm.status);
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            const uint64_t vd = vd0 + (uint64_t)(s * (TILE >> 4));
+            ok = mbar_wait(bar_p_full + 8 * w, cp[w] & 1u, abort_flag, prm.status) &&
+                 mbar_wait(bar_v_full + 8 * s, ph, abort_flag, prm.status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < BS / 16; ++kk) {
+              const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+              tc_mma_ts(tmem_base + COL_O, tmem_base + COL_P + 8 * kk, vd + off, IDESC, (j > 0 || kk > 0) ? 1u : 0u, 1u);
+            }
+            tc_commit(bar_v_empty + 8 * s, 1u);
+            tc_commit(bar_pv_done + 8 * w, 1u);
+            if (!ok) break;
+            ++cp[w];
+            if (++s == VS) { s = 0; ph ^= 1u; }
+          }
         }
       }
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
-    // warpgroup t owns tile t; thread <-> query row <-> TMEM lane, all 128 key columns
-    if (NT == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
-    const int t = warp >> 2;
-    const int r = row0 + t;
-    const int n = nl[t];
-    const int row = (warp & 3) * 32 + lane;
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+    const int w = warp >> 2;                                 // this group takes blocks j = w, w+2, ... of a row
+    const int row = (warp & 3) * 32 + lane;                  // query row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_tmem = tmem_base + lane_addr + 128 * t;
-    const uint32_t o_tmem = tmem_base + lane_addr + 128 * NT + 128 * t;
-    const bool probe = (threadIdx.x & 127) == 0;
-    if (r < prm.R) {
-      const int I = r % Nb;
-      const int bh_t = r / Nb;
+    const uint32_t s_tmem = tmem_base + lane_addr + 128 * w;
+    const uint32_t o_tmem = tmem_base + lane_addr + COL_O;
+    const uint32_t p_tmem = tmem_base + lane_addr + COL_P;
+    const uint32_t q_tmem = tmem_base + lane_addr + COL_Q + (F8 ? 16 : 32) * w;
+    const int tail_keys = prm.N - (prm.Nb - 1) * KB;         // valid keys of the last key block
+    const int qh = row >> 6;                                 // 64-token blocks: which query block of the tile I am in
+    float c = prm.scale_log2;      // e4m3 variant: times the scales of the query block and of the key block, per block
+    uint32_t cnt[2] = {0, 0};      // blocks of parity 0 / 1 completed in earlier rows (barrier phase bases)
+    uint32_t rows_done = 0;        // non-empty rows finished
+    bool ok = true;
+
+    // this group's half (d columns 64w..64w+63) of a row's Q: global -> registers -> TMEM
+    auto load_q = [&](int r, uint32_t* qv) {
+#pragma unroll
+      for (int e = 0; e < 32; ++e) qv[e] = 0u;
+      if (r >= prm.R) return;
+      const int bh = r / Nb, qi = (r % Nb) * BS + row;
+      if (qi >= prm.N) return;
+      const long long eoff = (long long)(bh / prm.H) * prm.sq.b + (long long)(bh % prm.H) * prm.sq.h +
+                             (long long)qi * prm.sq.n + 64 * w;           // in elements
+      const uint4* src = F8 ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(prm.q) + eoff)
+                            : reinterpret_cast<const uint4*>(prm.q + eoff);
+#pragma unroll
+      for (int e = 0; e < (F8 ? 4 : 8); ++e) {                            // 64 elements: 64 or 128 bytes
+        const uint4 u = __ldg(src + e);
+        qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
+      }
+    };
+    auto store_q = [&](const uint32_t* qv) {
+      if (F8) tmem_st16(q_tmem, qv); else tmem_st32(q_tmem, qv);
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_q_ready);
+    };
+
+    // The row sequence comes from the queue the K producer fills.  The entry after the current one is
+    // read in the epilogue (the producer has published it by then: it runs about two blocks ahead),
+    // so the next row's Q and first list entries are at hand when the row changes.
+    const bool signs = lane == 0;                             // one lane per warp signs queue entries off
+    int r_c = prm.R, n_c = 0, beg_c = 0;
+    uint32_t e0_c = 0u, e1_c = 0u;
+    if (!fetch_row(0, r_c, n_c, beg_c, e0_c, e1_c, signs)) ok = false;
+    if (ok && r_c < prm.R) {
+      // first row: its Q goes in right away
+      uint32_t qv[32];
+      load_q(r_c, qv);
+      store_q(qv);
+    }
+    for (; ok && r_c < prm.R; ++rows_done) {
+      const int r = r_c, n = n_c, lbeg = beg_c;
+      uint32_t J = (w == 0) ? e0_c : e1_c;                           // my first list entry of the row
+      const int I = r % Nb, bh = r / Nb;
+      const int hh = bh % prm.H, bb = bh / prm.H;
       const int qi = I * BS + row;
-      const int tail_keys = prm.N - (Nb - 1) * BS;           // valid keys of the last block
-      float m_used = -INFINITY, l = 0.f;
-      float c = prm.scale_log2;
-      float qs = 1.f;
-      if (F8) qs = prm.q_scale[(long long)bh_t * Nb + I];
-      bool ok = true;
-      for (int j = 0; j < n; ++j) {
-        const int J = dense ? j : __ldg(prm.col_idx + lbeg[t] + j);
-        if (F8) c = prm.scale_log2 * qs * __ldg(prm.k_scale + (long long)bh_t * Nb + J);
-        const int valid = (J == Nb - 1) ? tail_keys : BS;      // key columns of this block that exist
-        if (probe) SVA_PROF(t, j, 0);
-        if (!mbar_wait(bar_s_full + 8 * t, (uint32_t)(j & 1), abort_flag, prm.status)) { ok = false; break; }
-        if (probe) SVA_PROF(t, j, 1);
-        tc_fence_after();
-        if (prm.debug & 1) {
-          tc_fence_before();
-          mbar_arrive(bar_p_half + 16 * t);
-          l = 1.f;
-          continue;
+      const int wl = (n - 1) & 1;                                     // group that takes the row's last block
+      const uint32_t last = cnt[wl] + (uint32_t)((n - 1) >> 1);       // phase index of that block
+      float m_mine = -INFINITY;      // reference exponent my partial row sum is relative to
+      float l = 0.f;                 // partial row sum over this group's blocks
+      float qs_row = 1.f, ks_next = 1.f;
+      if (F8) {
+        qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + I) * prm.scale_log2;
+        if (w < n) ks_next = __ldg(prm.k_scale + (long long)bh * prm.Nb + (int)J);
+      }
+      for (int j = w; j < n; j += 2) {
+        const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
+        const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
+        // valid keys of the tile's two 64-key halves (64-token blocks: a half whose key block this
+        // thread's query block does not keep counts as 0; uniform over a warp)
+        int v0, v1;
+        if (B64) {
+          const int u0 = (int)(J & 0x3fffu), u1 = (int)((J >> 16) & 0x3fffu);
+          v0 = ((J >> (14 + qh)) & 1u) ? (u0 == prm.Nb - 1 ? tail_keys : 64) : 0;
+          v1 = ((J >> (30 + qh)) & 1u) ? (u1 == prm.Nb - 1 ? tail_keys : 64) : 0;
+        } else {
+          v0 = ((int)J == prm.Nb - 1) ? tail_keys : BS;      // 128-token blocks: all valid keys counted in v0
+          v1 = 0;
         }
-        if (valid < BS) {
-          // ragged last key block: keys that do not exist become -inf in TMEM before S is read (a short
-          // rolled loop -- this keeps 128 compare/select pairs out of the hot instruction stream)
+        if (F8) c = qs_row * ks_next;
+        if (j + 2 < n) {                                               // one entry ahead
+          J = list_block<B64>(prm, lbeg, j + 2);
+          if (F8) ks_next = __ldg(prm.k_scale + (long long)bh * prm.Nb + (int)J);
+        }
+        if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
+        tc_fence_after();
+        if (B64 ? (v0 + v1 < BS) : (v0 < BS)) {
+          // Keys that do not exist (ragged last key block) become -inf in TMEM before S is read: a short
+          // rolled loop, which keeps 128 compare/select pairs out of the hot instruction stream.  A half
+          // that is not kept at all (64-token blocks) is left alone here: it is excluded below.
+          if (B64) {
+            if (v0 > 0) {
 #pragma unroll 1
-          for (int i = valid; i < BS; ++i) tmem_st1(s_tmem + i, 0xff800000u);
+              for (int e = v0; e < 64; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+            }
+            if (v1 > 0) {
+#pragma unroll 1
+              for (int e = 64 + v1; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+            }
+          } else {
+#pragma unroll 1
+            for (int e = v0; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+          }
           tc_wait_st();
         }
-        // ---- row maximum over the 128 columns (whole row in registers)
         uint32_t sv[128];
         tmem_ld32(s_tmem + 0, sv + 0);
         tmem_ld32(s_tmem + 32, sv + 32);
         tmem_ld32(s_tmem + 64, sv + 64);
         tmem_ld32(s_tmem + 96, sv + 96);
         tc_wait_ld();
-        if (probe) SVA_PROF(t, j, 2);
+        tc_fence_before();
+        mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
         float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+        float mx0, mx1;
+        if (B64) {                                           // a, b: keys 0..63; c, d: keys 64..127
 #pragma unroll
-        for (int i = 0; i < 128; i += 8) {
-          mxa = max3(mxa, __uint_as_float(sv[i + 0]), __uint_as_float(sv[i + 1]));
-          mxb = max3(mxb, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
-          mxc = max3(mxc, __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
-          mxd = max3(mxd, __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
+          for (int e = 0; e < 64; e += 4) {
+            mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+            mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+            mxc = max3(mxc, __uint_as_float(sv[e + 64]), __uint_as_float(sv[e + 65]));
+            mxd = max3(mxd, __uint_as_float(sv[e + 66]), __uint_as_float(sv[e + 67]));
+          }
+          mx0 = v0 > 0 ? fmaxf(mxa, mxb) : -INFINITY;        // a half this query block does not keep has no say
+          mx1 = v1 > 0 ? fmaxf(mxc, mxd) : -INFINITY;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 128; e += 8) {
+            mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+            mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+            mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
+            mxd = max3(mxd, __uint_as_float(sv[e + 6]), __uint_as_float(sv[e + 7]));
+          }
+          mx0 = fmaxf(mxa, mxb);
+          mx1 = fmaxf(mxc, mxd);
         }
-        const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd)) * c;
-        // lazy rescale: move the reference maximum only when it would grow by more than 2^32 (P then stays
-        // below 2^32 and a row sum below 2^32 * N: far inside fp32 and bf16 range, and rescales of O are rare)
-        if (__any_sync(0xffffffffu, mx > m_used + 32.0f)) {
-          const float m_new = fmaxf(m_used, mx);
-          const float alpha = ex2(m_used - m_new);            // first block: exp2(-inf) = 0
-          l *= alpha;
-          m_used = m_new;
-          if (j > 0) {
+        const float mx = fmaxf(mx0, mx1) * c;
+        // reference exponent left by block j-1 (other group)
+        float m_prev = -INFINITY;
+        if (j > 0) {
+          if (!mbar_wait(bar_ref + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          m_prev = ref[(w ^ 1) * 128 + row];
+        }
+        // lazy rule: raise the reference only when the row maximum outgrows it by more than 2^LAZY_LOG2
+        const float m_new = (mx > m_prev + LAZY_LOG2) ? mx : m_prev;
+        ref[w * 128 + row] = m_new;
+        mbar_arrive(bar_ref + 8 * w);
+        if (m_new != m_mine) { l *= ex2(m_mine - m_new); m_mine = m_new; }      // first block: 0 * 2^-inf
+        bool pv_waited = false;
+        if (j > 0 && __any_sync(0xffffffffu, m_new != m_prev)) {
+          // rescale this row of O once P V(j-1) has completed (O is then quiescent: P V(j) waits for us)
+          if (!mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          pv_waited = true;
+          tc_fence_after();
+          const float alpha = ex2(m_prev - m_new);
 #pragma unroll 1
-            for (int cc = 0; cc < D; cc += 16) {
-              uint32_t ov[16];
-              tmem_ld16(o_tmem + cc, ov);
-              tc_wait_ld();
+          for (int cc = 0; cc < D; cc += 16) {
+            uint32_t ov[16];
+            tmem_ld16(o_tmem + cc, ov);
+            tc_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-              tmem_st16(o_tmem + cc, ov);
-            }
+            for (int e = 0; e < 16; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+            tmem_st16(o_tmem + cc, ov);
+          }
+          tc_wait_st();
+        }
+        // P = 2^(S*c - m); the packed bf16 pairs overwrite sv[0..63]
+        // (64-token blocks: -inf instead of -m for a half that is not kept, or while the row has seen no
+        // kept key yet, makes those P exactly 0 at no cost)
+        float nm = -m_new, nmh1 = -m_new;
+        if (B64) {
+          if (m_new == -INFINITY || v0 == 0) nm = -INFINITY;
+          if (m_new == -INFINITY || v1 == 0) nmh1 = -INFINITY;
+        }
+        const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm), nm2h1 = B64 ? pack2(nmh1, nmh1) : nm2;
+        uint64_t sum2 = pack2(0.f, 0.f);
+        if (!(prm.debug & 1)) {
+#pragma unroll
+          for (int e = 0; e < 128; e += 2) {
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, e < 64 ? nm2 : nm2h1), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            sum2 = add2(sum2, pack2(p0, p1));
+            sv[e / 2] = pack_bf16(p0, p1);
           }
         }
-        if (probe) SVA_PROF(t, j, 3);
-        // ---- P = 2^(S*c - m_used); the packed bf16 pairs overwrite sv[0..63]
-        const float nm = -m_used;
-        const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
-        uint64_t sum2 = pack2(0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < 128; i += 2) {
-          float x0, x1;
-          unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2), x0, x1);
-          const float p0 = ex2(x0), p1 = ex2(x1);
-          sum2 = add2(sum2, pack2(p0, p1));
-          sv[i / 2] = pack_bf16(p0, p1);
-          if (i == 62) tmem_st32(s_tmem, sv);
+        {
+          float sum_a, sum_b;
+          unpack2(sum2, sum_a, sum_b);
+          l += sum_a + sum_b;
         }
-        float sum_a, sum_b;
-        unpack2(sum2, sum_a, sum_b);
-        tmem_st32(s_tmem + 32, sv + 32);
-        l += sum_a + sum_b;
-        if (probe) SVA_PROF(t, j, 4);
+        // the P columns are free once P V(j-1) has completed (block 0: the previous row's last P V
+        // was waited for in that row's epilogue)
+        if (j > 0 && !pv_waited &&
+            !mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st32(p_tmem, sv);
+        tmem_st32(p_tmem + 32, sv + 32);
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p_half + 16 * t);
-        if (probe) SVA_PROF(t, j, 5);
+        mbar_arrive(bar_p_full + 8 * w);
       }
-      // ---- epilogue
-      __nv_bfloat16* orow = prm.o + (long long)(bh_t / prm.H) * prm.so.b + (long long)(bh_t % prm.H) * prm.so.h +
-                            (long long)qi * prm.so.n;
-      if (n == 0) {
-        if (qi < prm.N) {
+      if (!ok) break;
+      // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
+      // normalise and store (each group half of d)
+      if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
+      const int r_next = r_c;                                         // (the queue holds non-empty rows only)
+      uint32_t qn[32];
+      load_q(r_next, qn);                                             // in flight during the waits below
+      if (!mbar_wait(bar_ref + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+      const float m_fin = ref[wl * 128 + row];
+      if (m_mine != m_fin) { l *= ex2(m_mine - m_fin); m_mine = m_fin; }        // l = 0 for a group without blocks
+      volatile float* lxr = lx + (rows_done & 1u) * 256;
+      lxr[w * 128 + row] = l;
+      if ((threadIdx.x & 127) == 0) bulk_wait_read0();                // the previous row's store has read the staging panel
+      mbar_arrive(bar_xch);
+      if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
+      // both groups have seen all their S tiles: no MMA reads Q any more
+      if (r_next < prm.R) store_q(qn);
+      if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+      tc_fence_after();
+      const float lt = l + lxr[(w ^ 1) * 128 + row];
+      // (64-token blocks: a query block with an empty list beside one with work has lt = 0 -> zeros, lse = -inf)
+      const float inv = (!B64 || lt > 0.f) ? 1.0f / lt : 0.f;
+      {
+        uint32_t ov[64];
+        tmem_ld32(o_tmem + (D / 2) * w, ov);
+        tmem_ld32(o_tmem + (D / 2) * w + 32, ov + 32);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_o_free);                                      // the next row may overwrite O
+        // normalised bf16 row -> this group's staging panel (128-byte swizzle), then one tile store;
+        // rows beyond N are clipped by the tensor map
+        uint8_t* stg = smem + OFF_O + w * (TILE / 2) + row * 128;
 #pragma unroll
-          for (int cc = 0; cc < D; cc += 8) *reinterpret_cast<uint4*>(orow + cc) = make_uint4(0, 0, 0, 0);
-          if (prm.lse) prm.lse[(long long)bh_t * prm.N + qi] = -INFINITY;
+        for (int e = 0; e < 64; e += 8) {
+          uint4 v4;
+          v4.x = pack_bf16(__uint_as_float(ov[e + 0]) * inv, __uint_as_float(ov[e + 1]) * inv);
+          v4.y = pack_bf16(__uint_as_float(ov[e + 2]) * inv, __uint_as_float(ov[e + 3]) * inv);
+          v4.z = pack_bf16(__uint_as_float(ov[e + 4]) * inv, __uint_as_float(ov[e + 5]) * inv);
+          v4.w = pack_bf16(__uint_as_float(ov[e + 6]) * inv, __uint_as_float(ov[e + 7]) * inv);
+          *reinterpret_cast<uint4*>(stg + (((e >> 3) ^ (row & 7)) << 4)) = v4;
         }
-      } else if (ok && mbar_wait(bar_o_done + 8 * t, 0, abort_flag, prm.status)) {
-        tc_fence_after();
-        const float inv = 1.0f / l;
-#pragma unroll
-        for (int cc = 0; cc < D; cc += 32) {
-          uint32_t ov[32];
-          tmem_ld32(o_tmem + cc, ov);
-          tc_wait_ld();
-          if (qi < prm.N) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(ov[i + 0]) * inv, __uint_as_float(ov[i + 1]) * inv);
-              w.y = pack_bf16(__uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-              w.z = pack_bf16(__uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv);
-              w.w = pack_bf16(__uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + cc + i) = w;
-            }
+        fence_async_smem();
+        mbar_arrive(bar_ost + 8 * w);
+        if ((threadIdx.x & 127) == 0) {
+          // (a wait that runs out has raised the abort flag; the other threads leave at their next wait)
+          if (mbar_wait(bar_ost + 8 * w, rows_done & 1u, abort_flag, prm.status)) {
+            tma_store_4d(&tm_o, sbase + OFF_O + w * (TILE / 2), (D / 2) * w, I * BS, hh, bb);
+            bulk_commit();
           }
         }
-        if (prm.lse && qi < prm.N)
-          prm.lse[(long long)bh_t * prm.N + qi] = (m_used + log2f(l)) * 0.6931471805599453f;
+        if (qi < prm.N && prm.lse && w == 0) prm.lse[(long long)bh * prm.N + qi] = (m_fin + log2f(lt)) * 0.6931471805599453f;
       }
+      cnt[0] += (uint32_t)((n + 1) >> 1);
+      cnt[1] += (uint32_t)(n >> 1);
     }
+    if ((threadIdx.x & 127) == 0) bulk_wait0();                       // my output stores have completed
   }
 
   // ---------------------------------------------------------------- tear-down
+  if (prm.prof && threadIdx.x == 0)
+    atomicMax(reinterpret_cast<unsigned long long*>(prm.prof + 319), (unsigned long long)(clock64() - t_cta0));
   if (*abort_flag) {
     // give copies and MMAs still in flight time to land before shared memory and TMEM go away
     const long long t0 = clock64();
@@ -444,9 +661,114 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == W_MMA) {
+  if (warp == 9) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ V^T
+// V [B,H,N,d] (strided) -> tiled transposed copy: for every (b,h) and key block J (kb = 128 or 64
+// keys) one contiguous tile [d = 128 rows][kb keys], keys >= N zero.  A 128-key tile is then one
+// contiguous TMA box pair, exactly like a K tile; a 64-key tile is one box (one panel of a tile).
+__global__ void __launch_bounds__(256)
+transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
+                   int Nb, int d, int kb, int32_t* __restrict__ row_counter) {
+  // the attention kernel that follows draws its rows from this counter
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *row_counter = 0;
+  __shared__ __nv_bfloat16 tile[64][66];            // [d][key], padded
+  const int n0 = blockIdx.x * 64, d0 = blockIdx.y * 64, bh = blockIdx.z;
+  const int b = bh / H, h = bh % H;
+  const __nv_bfloat16* src = v + (long long)b * sv.b + (long long)h * sv.h;
+  {
+    const int c8 = threadIdx.x & 7;                 // 8 d-values (16 bytes)
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int key = (threadIdx.x >> 3) + 32 * pass;
+      uint4 u = make_uint4(0, 0, 0, 0);
+      if (n0 + key < N) u = __ldg(reinterpret_cast<const uint4*>(src + (long long)(n0 + key) * sv.n + d0) + c8);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&u);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) tile[c8 * 8 + q][key] = e[q];
+    }
+  }
+  __syncthreads();
+  {
+    const int k8 = threadIdx.x & 7;                 // 8 keys (16 bytes)
+    const int J = n0 / kb, kin = (n0 % kb) + k8 * 8;
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int dd = (threadIdx.x >> 3) + 32 * pass;
+      __align__(16) __nv_bfloat16 e[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) e[q] = tile[dd][k8 * 8 + q];
+      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * d + d0 + dd) * kb + kin) = *reinterpret_cast<uint4*>(e);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ 64-token blocks: tile lists
+// The MMA tile is 128 x 128, so with 64-token blocks one tile row is two adjacent query blocks (A, B)
+// and one tile two key blocks.  Per tile row this kernel merges the two CSR rows into the ascending
+// union of their key blocks, pairs the union up into tiles and notes for every key block which of the
+// two query blocks keeps it (the softmax excludes the other).  One warp per tile row: membership
+// bitmaps in shared memory, then every lane enumerates the bits of its word.  Entries are 16 bits
+// {key block (14), kept by A, kept by B}; tile j of the row is the 32-bit word at start + j.  The
+// start needs no scan: ceil((entries before the tile row + its index) / 2) leaves room for every earlier
+// row's ceil(|union| / 2) tiles.
+constexpr int PAIR_WARPS = 8;
+__global__ void __launch_bounds__(PAIR_WARPS * 32)
+pair_lists_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, int Nb, int Nt, int R2,
+                  int32_t* __restrict__ tile_cnt, int32_t* __restrict__ tile_beg, uint32_t* __restrict__ tile_desc,
+                  long long cap, int32_t* __restrict__ status) {
+  __shared__ uint32_t bm[PAIR_WARPS][2][32];
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * PAIR_WARPS + w;
+  if (t >= R2) return;
+  const int bh = t / Nt, I2 = t % Nt;
+  const int rA = bh * Nb + 2 * I2;
+  const bool hasB = 2 * I2 + 1 < Nb;
+  bm[w][0][lane] = 0u;
+  bm[w][1][lane] = 0u;
+  __syncwarp();
+  const int begA = __ldg(row_ptr + rA), endA = __ldg(row_ptr + rA + 1);
+  const int endB = hasB ? __ldg(row_ptr + rA + 2) : endA;
+  const bool bad = begA < 0 || endA < begA || endB < endA || endA - begA > Nb || endB - endA > Nb;
+  bool bad_idx = false;
+  if (!bad) {
+    for (int e = begA + lane; e < endB; e += 32) {
+      const int J = __ldg(col_idx + e);
+      if (J < 0 || J >= Nb) { bad_idx = true; continue; }
+      atomicOr(&bm[w][e < endA ? 0 : 1][J >> 5], 1u << (J & 31));
+    }
+  }
+  if ((bad || bad_idx) && status) atomicOr(status, SVA_DEV_BAD_INDEX);
+  __syncwarp();
+  const uint32_t a = bm[w][0][lane], b = bm[w][1][lane];
+  uint32_t u = a | b;
+  int incl = __popc(u);
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
+  }
+  const int total = __shfl_sync(0xffffffffu, incl, 31);
+  long long start = ((long long)(bad ? 0 : begA) + t + 1) / 2;
+  int ntile = (total + 1) / 2;
+  if (start + ntile > cap) { ntile = 0; if (lane == 0 && status) atomicOr(status, SVA_DEV_BAD_INDEX); }
+  if (ntile > 0) {
+    uint16_t* ent = reinterpret_cast<uint16_t*>(tile_desc) + 2 * start;
+    int p = incl - __popc(u);
+    while (u) {
+      const int bit = __ffs(u) - 1;
+      u &= u - 1;
+      ent[p++] = (uint16_t)((lane * 32 + bit) | (((a >> bit) & 1u) << 14) | (((b >> bit) & 1u) << 15));
+    }
+    if (lane == 0 && (total & 1)) ent[total] = 0;          // odd union: the last tile's second half is nobody's
+  }
+  if (lane == 0) {
+    tile_cnt[t] = ntile;
+    tile_beg[t] = (int32_t)start;
   }
 }
 
@@ -456,7 +778,7 @@ typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, v
                                 CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                 CUtensorMapFloatOOBfill);
 
-static encode_fn_t get_encode() {
+static encode_fn_t get_encode_ts() {
   static encode_fn_t fn = nullptr;
   if (!fn) {
     void* p = nullptr;
@@ -469,74 +791,174 @@ static encode_fn_t get_encode() {
   return fn;
 }
 
-// [B,H,N,d] tensor with element strides s, as a 4-D map (d, N, H, B); box = 128 bytes x 128 rows.
-static int make_map(CUtensorMap* map, const void* ptr, int elem_bytes, int B, int H, int N, int d,
-                    const Strides& s, int box_rows) {
-  encode_fn_t enc = get_encode();
+// 4-D map (inner, rows, H, B) of bf16 (or bytes) with byte strides; box = 128 bytes x box_rows, 128-byte swizzle.
+static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuuint64_t rows, int H, int B,
+                       cuuint64_t row_stride, cuuint64_t h_stride, cuuint64_t b_stride, int box_rows,
+                       int elem_bytes = 2) {
+  encode_fn_t enc = get_encode_ts();
   if (!enc) return SVA_ERR_CUDA;
-  cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
-  cuuint64_t strides[3] = {(cuuint64_t)s.n * elem_bytes, (cuuint64_t)s.h * elem_bytes, (cuuint64_t)s.b * elem_bytes};
+  cuuint64_t dims[4] = {inner, rows, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {row_stride, h_stride, b_stride};
   // a size-1 dimension may carry any stride; give it a legal one
-  if (H == 1) strides[1] = strides[0] * (cuuint64_t)N;
+  if (H == 1) strides[1] = strides[0] * rows;
   if (B == 1) strides[2] = strides[1] * (cuuint64_t)H;
   for (int i = 0; i < 3; ++i)
     if (strides[i] % 16 != 0 || strides[i] == 0) return SVA_ERR_ALIGNMENT;
-  int inner = 128 / elem_bytes;
-  if (inner > d) inner = d;
-  cuuint32_t box[4] = {(cuuint32_t)inner, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t box[4] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows, 1, 1};   // 128 bytes per row
   cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult rc = enc(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
-                    const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    (inner * elem_bytes == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult rc = enc(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? SVA_OK : SVA_ERR_CUDA;
 }
 
-static int g_tiles_per_cta = 2;   // bring-up switch, see sva_debug_set_tiles_per_cta
-static long long* g_prof = nullptr;   // tuning aid, see sva_debug_set_prof_buffer
-static int g_debug = 0;
+static long long* g_prof_ts = nullptr;
+static int g_debug_ts = 0;
 
-template <int D, int NT, bool F8>
-static int launch_cfg(const Dims& m, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                      const AttnParams& prm, cudaStream_t st) {
-  using C = Cfg<D, NT, F8>;
-  auto kern = attn_sm100_kernel<D, NT, F8>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+template <bool B64, bool F8>
+static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                     const TsParams& prm, cudaStream_t st) {
+  auto kern = attn_ts_kernel<B64, F8>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
     return SVA_ERR_CUDA;
-  const int grid = (m.R + NT - 1) / NT;
-  kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, tk, tv, prm);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return SVA_ERR_CUDA;
+  const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
+  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
-int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
-                      const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
-                      const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                      cudaStream_t st) {
-  if (m.block != BS || m.d != 128) return SVA_ERR_UNSUPPORTED;
-  CUtensorMap tq, tk, tv;
-  const int eb = m.fp8 ? 1 : 2;
-  int rc;
-  if ((rc = make_map(&tq, q, eb, m.B, m.H, m.N, m.d, make_strides(p->q_stride), BS)) != SVA_OK) return rc;
-  if ((rc = make_map(&tk, k, eb, m.B, m.H, m.N, m.d, make_strides(p->k_stride), BS)) != SVA_OK) return rc;
-  if ((rc = make_map(&tv, v, 2, m.B, m.H, m.N, m.d, make_strides(p->v_stride), BS / 2)) != SVA_OK) return rc;
-  AttnParams prm;
-  prm.row_ptr = row_ptr; prm.col_idx = col_idx; prm.q_scale = qs; prm.k_scale = ks;
-  prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
-  prm.so = make_strides(p->o_stride);
-  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.R = m.R;
-  prm.scale_log2 = m.scale * 1.4426950408889634f;
-  prm.prof = g_prof;
-  prm.debug = g_debug;
-  // a CTA's tiles must belong to one head: pair tiles only when Nb is even
-  const int nt = (g_tiles_per_cta == 2 && m.Nb % 2 == 0) ? 2 : 1;
-  if (m.fp8) return nt == 2 ? launch_cfg<128, 2, true>(m, tq, tk, tv, prm, st) : launch_cfg<128, 1, true>(m, tq, tk, tv, prm, st);
-  return nt == 2 ? launch_cfg<128, 2, false>(m, tq, tk, tv, prm, st) : launch_cfg<128, 1, false>(m, tq, tk, tv, prm, st);
+// Workspace layout: transposed V tiles | row counter (256 bytes) | 64-token blocks only: tile_cnt[R2],
+// tile_beg[R2], tile_desc[cap] with R2 = B*H*ceil(Nb/2) tile rows and cap the bound for a dense CSR.
+struct TsLayout {
+  size_t vt_bytes, counter_off, cnt_off, beg_off, desc_off, total;
+  long long cap;
+  int R2, Nt;
+};
+static TsLayout ts_layout(const Dims& m) {
+  TsLayout L;
+  L.vt_bytes = (size_t)m.B * m.H * m.Nb * m.block * m.d * 2;
+  L.counter_off = L.vt_bytes;
+  L.Nt = m.block == 64 ? (m.Nb + 1) / 2 : m.Nb;
+  L.R2 = m.B * m.H * L.Nt;
+  L.cnt_off = L.beg_off = L.desc_off = L.counter_off + 256;
+  L.cap = 0;
+  L.total = L.counter_off + 256;
+  if (m.block == 64) {
+    L.beg_off = L.cnt_off + (((size_t)L.R2 * 4 + 255) & ~(size_t)255);
+    L.desc_off = L.beg_off + (((size_t)L.R2 * 4 + 255) & ~(size_t)255);
+    L.cap = ((long long)m.R * m.Nb + L.R2) / 2 + 2;
+    L.total = L.desc_off + (((size_t)L.cap * 4 + 255) & ~(size_t)255);
+  }
+  return L;
 }
 
-void set_tiles_per_cta(int n) { g_tiles_per_cta = n == 1 ? 1 : 2; }
-void set_prof_buffer(void* p) { g_prof = (long long*)p; }
-void set_debug_mode(int v) { g_debug = v; }
-int set_wait_limit(long long cycles) {
+bool attn_ts_serves(const Dims& m) {
+  return m.d == 128 && m.Nb <= 16383 && (m.block == BS || (m.block == 64 && !m.fp8));
+}
+
+size_t attn_ts_workspace_bytes(const Dims& m) {
+  if (!attn_ts_serves(m)) return 0;
+  size_t bytes = ts_layout(m).total;
+  if (m.block == 64) {                      // the dense entry point runs 64-token blocks as 128-token blocks
+    Dims d = m;
+    d.block = BS; d.Nb = (m.N + BS - 1) / BS; d.R = m.B * m.H * d.Nb;
+    const size_t b2 = ts_layout(d).total;
+    if (b2 > bytes) bytes = b2;
+  }
+  return bytes;
+}
+
+static int check_ts_workspace(const Dims& m, const void* ws, size_t ws_bytes) {
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < attn_ts_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
+  return SVA_OK;
+}
+
+// V -> tiled transposed copy in the workspace, row counter of the scheduler = 0.
+int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
+                        cudaStream_t st) {
+  int rc = check_ts_workspace(m, ws, ws_bytes);
+  if (rc) return rc;
+  const TsLayout L = ts_layout(m);
+  const Strides sv = make_strides(p->v_stride);
+  dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
+                                         reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + L.counter_off));
+  return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
+}
+
+// v == nullptr: the workspace has been prepared by launch_prepare_v_ts (once per attention call).
+int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, const void* k, const void* v,
+                   const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                   void* ws, size_t ws_bytes, cudaStream_t st) {
+  int rc = check_ts_workspace(m_in, ws, ws_bytes);
+  if (rc) return rc;
+  // dense attention does not depend on the block size: 64-token blocks run as 128-token blocks
+  Dims m = m_in;
+  if (m.block == 64 && row_ptr == nullptr) {
+    m.block = BS;
+    m.Nb = (m.N + BS - 1) / BS;
+    m.R = m.B * m.H * m.Nb;
+  }
+  const bool b64 = m.block == 64;
+  const TsLayout L = ts_layout(m);
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  const Strides sk = make_strides(p->k_stride);
+  const Strides so = make_strides(p->o_stride);
+  CUtensorMap tk, tv, to;
+  if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2, BS)) != SVA_OK)
+    return rc;
+  const int eb = m.fp8 ? 1 : 2;
+  if ((rc = make_map_ts(&tk, k, m.d, m.N, m.H, m.B, (cuuint64_t)sk.n * eb, (cuuint64_t)sk.h * eb, (cuuint64_t)sk.b * eb,
+                        m.block, eb)) != SVA_OK)
+    return rc;
+  // transposed V: per (b,h) a [Nb*128 rows][block keys] matrix, key block J = rows J*128 .. J*128+127
+  const cuuint64_t vrows = (cuuint64_t)m.Nb * m.d;
+  if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
+                        vrows * m.block * 2 * m.H, BS)) != SVA_OK)
+    return rc;
+  if (v) {
+    // (the transposed copy is laid out for the block size of this launch)
+    const Strides sv = make_strides(p->v_stride);
+    dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+    transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
+                                           reinterpret_cast<int32_t*>(wsb + L.counter_off));
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+  } else if (m.block != m_in.block) {
+    return SVA_ERR_UNSUPPORTED;     // a workspace prepared for 64-token blocks cannot serve the dense path
+  }
+  TsParams prm;
+  prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
+  prm.q_scale = q_scale; prm.k_scale = k_scale;
+  prm.row_ptr = row_ptr; prm.col_idx = col_idx;
+  prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
+  prm.so = make_strides(p->o_stride);
+  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.Nt = L.Nt; prm.R = L.R2;
+  prm.tile_cnt = reinterpret_cast<const int32_t*>(wsb + L.cnt_off);
+  prm.tile_beg = reinterpret_cast<const int32_t*>(wsb + L.beg_off);
+  prm.tile_desc = reinterpret_cast<const uint32_t*>(wsb + L.desc_off);
+  prm.scale_log2 = m.scale * 1.4426950408889634f;
+  prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
+  prm.prof = g_prof_ts;
+  prm.debug = g_debug_ts;
+  if (b64) {
+    pair_lists_kernel<<<(L.R2 + PAIR_WARPS - 1) / PAIR_WARPS, PAIR_WARPS * 32, 0, st>>>(
+        row_ptr, col_idx, m.Nb, L.Nt, L.R2, reinterpret_cast<int32_t*>(wsb + L.cnt_off),
+        reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+    return launch_ts<true, false>(L.R2, tk, tv, to, prm, st);
+  }
+  if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, prm, st);
+  return launch_ts<false, false>(L.R2, tk, tv, to, prm, st);
+}
+
+void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }
+void ts_set_debug_mode(int v) { g_debug_ts = v; }
+int ts_set_wait_limit(long long cycles) {
   if (cycles <= 0) cycles = WAIT_LIMIT_CYCLES;
   return cudaMemcpyToSymbol(g_wait_limit, &cycles, sizeof(cycles)) == cudaSuccess ? 0 : 1;
 }

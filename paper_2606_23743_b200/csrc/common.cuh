@@ -55,16 +55,11 @@ int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const 
 int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
                      const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
                      const int32_t* col_idx, void* o, float* lse, int32_t* status, cudaStream_t st);
-int launch_attn_sm100(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
-                      const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
-                      const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                      cudaStream_t st);
-
 int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
-                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
+                   const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st);
 size_t attn_ts_workspace_bytes(const Dims& m);
-bool attn_ts_serves(const Dims& m);    // bf16, d = 128, 128- or 64-token blocks
+bool attn_ts_serves(const Dims& m);    // d = 128: bf16 with 128- or 64-token blocks, e4m3 Q/K with 128-token blocks
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
                         cudaStream_t st);
 

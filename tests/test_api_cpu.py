@@ -109,7 +109,7 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert B.attn_workspace_bytes(_problem(d=64)) == 0                   # CUDA-core kernel needs none
     # 64-token blocks: transposed V, counter, tile lists (R2 = 16 tile rows, 16 key blocks, 32 CSR rows)
     assert B.attn_workspace_bytes(_problem(block=64)) == 2 * 1024 * 128 * 2 + 256 + 256 + 256 + ((((32 * 16 + 16) // 2 + 2) * 4 + 255) // 256) * 256
-    assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 0             # e4m3 variant needs none
+    assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 1 * 2 * 8 * 128 * 128 * 2 + 256   # e4m3 Q/K: V is still bf16
     assert att(p) == 3                                                   # bf16 tensor-core path without workspace
     assert lib.sva_quantize_qk_fp8(C.byref(p), one, one, one, None, one, one, None) == 1
     bad = _problem(); bad.k_stride = (C.c_int64 * 3)(0, 0, 136)
