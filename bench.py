@@ -119,6 +119,9 @@ def oracle_sample(w, qb, kb, vb, n_rows):
     heads = -(-n_rows // w.Nb)
     q1, k1, v1 = qb[:1, :heads], kb[:1, :heads], vb[:1, :heads]
     t0 = time.perf_counter()
+    if w.fp8:       # FP8 variant: the quantiser is part of the path; routing and attention see the dequantised values
+        q1 = oracle.dequantize_e4m3(*oracle.quantize_e4m3(q1, w.N, w.block), w.N, w.block)
+        k1 = oracle.dequantize_e4m3(*oracle.quantize_e4m3(k1, w.N, w.block), w.N, w.block)
     sel, _ = oracle.select_from_qk(q1, k1, w.N, w.block, w.scale, w.mode, w.k, w.tau, w.win_t, w.win_s,
                                    w.blocks_per_frame if w.win_t >= 0 else 0)
     rows = list(range(n_rows))
@@ -185,7 +188,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=[k for k in WORKLOADS if not WORKLOADS[k].fp8])
+    ap.add_argument("--workload", default="large", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -209,6 +212,13 @@ def main():
     o = torch.empty_like(v)
     oh = torch.empty(o.shape, dtype=o.dtype).pin_memory()
     p = B.make_problem(q, k, v, o, w.N, w.block)
+    if w.fp8:
+        # FP8 variant: Q and K are quantised to e4m3 with per-block scales inside every step
+        q8, k8 = torch.zeros(q.shape, dtype=torch.uint8, device=dev), torch.zeros(k.shape, dtype=torch.uint8, device=dev)
+        qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device=dev)
+        ks = torch.zeros_like(qs)
+        pq = B.make_problem(q, k, None, None, w.N, w.block)
+        p = B.make_problem(q8, k8, v, o, w.N, w.block, 0.0, True)
     s = B.make_select(w.mode, w.k, w.tau, w.win_t, w.win_s, w.blocks_per_frame if w.win_t >= 0 else 0)
     ws = torch.empty(max(B.select_workspace_bytes(p, s), 256), dtype=torch.uint8, device=dev)
     row_ptr = torch.zeros(w.R + 1, dtype=torch.int32, device=dev)
@@ -217,7 +227,7 @@ def main():
     aws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
     # routing kernels + V transpose + attention (+ the tile-list kernel of the 64-token-block path)
-    launches_per_step = (4 if variable_rows else 2) + 2 + (1 if w.block == 64 else 0)
+    launches_per_step = (4 if variable_rows else 2) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
 
     # V is prepared (tiled transposed copy) on a second stream while routing, which never reads V, runs
     # (lower priority: its CTAs fill the SMs that the latency-bound selection kernel leaves idle instead of
@@ -234,11 +244,24 @@ def main():
             B.attn_prepare_v(p, v, aws)
             v_ready.record()
 
+    def route():
+        if w.fp8:
+            B.quantize_qk_fp8(pq, q, k, q8, k8, qs, ks)
+            B.block_select(p, s, q8, k8, row_ptr, col_idx, ws, qs, ks)
+        else:
+            prepare_v()
+            B.block_select(p, s, q, k, row_ptr, col_idx, ws)
+
+    def attend():
+        if w.fp8:       # (the two-step form takes bf16 Q/K only: the one call transposes V itself)
+            B.block_sparse_attn_fwd(p, q8, k8, v, row_ptr, col_idx, o, None, status, qs, ks, workspace=aws)
+        else:
+            torch.cuda.current_stream().wait_event(v_ready)
+            B.block_sparse_attn_fwd_prepared(p, q, k, row_ptr, col_idx, o, None, status, workspace=aws)
+
     def step():
-        prepare_v()
-        B.block_select(p, s, q, k, row_ptr, col_idx, ws)
-        torch.cuda.current_stream().wait_event(v_ready)
-        B.block_sparse_attn_fwd_prepared(p, q, k, row_ptr, col_idx, o, None, status, workspace=aws)
+        route()
+        attend()
 
     for _ in range(warmup):
         step()
@@ -258,12 +281,10 @@ def main():
     ev0.record()
     for i in range(args.steps):
         sel_ev[i][0].record()
-        prepare_v()
-        B.block_select(p, s, q, k, row_ptr, col_idx, ws)
+        route()
         sel_ev[i][1].record()
-        torch.cuda.current_stream().wait_event(v_ready)
         att_ev[i][0].record()
-        B.block_sparse_attn_fwd_prepared(p, q, k, row_ptr, col_idx, o, None, status, workspace=aws)
+        attend()
         att_ev[i][1].record()
     ev1.record()
     torch.cuda.synchronize()
@@ -310,7 +331,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": "e4m3 QK^T, bf16 PV" if w.fp8 else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
                    "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
                    "nnz_tiles": nnz, "parallelism": f"replicas x{world}",
@@ -321,7 +342,9 @@ def main():
         "select_gbs": sel_bytes / (sel_ms * 1e-3) / 1e9,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
-                     "kernel": "attn_ts_kernel (the V transpose runs beside routing on a second stream)",
+                     "kernel": "attn_ts_kernel" + (" with the V transpose in front of it" if w.fp8 else
+                                                  " (the V transpose runs beside routing on a second stream)"),
+                     "mixed_precision_ceiling": peak * 4.0 / 3.0 if w.fp8 else None,
                      "peak_source": f"{peak_kind} bf16 burst",
                      "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"])
                      if "bf16_tflops_sustained" in peaks else None,
