@@ -38,3 +38,30 @@ def test_same_frame_blocks_score_higher():
         frame = set(range(I // bpf * bpf, I // bpf * bpf + bpf))
         assert set(sel.kept(r).tolist()) == frame          # top-4 == the query's own frame
     assert sel.score_gap.min() > 0.5
+
+
+def test_tile_list_start_formula_leaves_room_for_every_earlier_row():
+    """64-token blocks: tile row t's descriptors start at ceil((CSR entries before it + t) / 2) -- no scan.
+    Every earlier tile row s needs ceil(|A_s u B_s| / 2) <= ceil((|A_s| + |B_s|) / 2) tiles; the starts must
+    leave at least that much room, for any row lengths, and stay below the capacity the workspace reserves."""
+    import numpy as np
+    rng = np.random.default_rng(7)
+    for Nb in (1, 2, 7, 16, 33):
+        for _ in range(50):
+            H = int(rng.integers(1, 4))
+            R = H * Nb
+            counts = rng.integers(0, Nb + 1, size=R)
+            row_ptr = np.concatenate([[0], np.cumsum(counts)])
+            Nt = (Nb + 1) // 2
+            starts, need = [], []
+            for t in range(H * Nt):
+                bh, I2 = divmod(t, Nt)
+                rA = bh * Nb + 2 * I2
+                a = counts[rA]
+                b = counts[rA + 1] if 2 * I2 + 1 < Nb else 0
+                starts.append((row_ptr[rA] + t + 1) // 2)
+                need.append((a + b + 1) // 2)          # worst case: disjoint lists
+            for t in range(len(starts) - 1):
+                assert starts[t] + need[t] <= starts[t + 1]
+            cap = (R * Nb + H * Nt) // 2 + 2
+            assert starts[-1] + need[-1] <= cap
