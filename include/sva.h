@@ -197,6 +197,25 @@ int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const 
 int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q8,
                         void* k8, float* q_scale, float* k_scale, void* stream);
 
+/*
+ * Token-subset gather / scatter (the paper's token pruning keeps a subset of the video tokens, about
+ * half of them, on some denoising calls; attention then runs over the kept tokens only, and the
+ * blocking of the routing applies to the gathered sequence).
+ *   gather : dst[b,h,m,:]              = src[b,h,token_idx[b,m],:]   m < M, token_idx[b,m] in [0, n_src)
+ *   scatter: dst[b,h,token_idx[b,m],:] = src[b,h,m,:]                token_idx[b,m] in [0, n_dst)
+ * src / dst are [B,H,*,d] tensors of elem_bytes-sized elements (1, 2 or 4), d contiguous, strides in
+ * elements, 16-byte aligned with d*elem_bytes a multiple of 16; token_idx is [B,M] int32 (the same
+ * subset for every head of a batch item; repeated indices make scatter order-dependent).  Rows that
+ * scatter does not name keep their contents.  An index out of range is reported in device_status
+ * (SVA_DEV_BAD_INDEX) and its row skipped.
+ */
+int sva_gather_tokens(const void* src, const int64_t src_stride[3], const int32_t* token_idx, int32_t B, int32_t H,
+                      int32_t M, int32_t n_src, int32_t d, int32_t elem_bytes, void* dst,
+                      const int64_t dst_stride[3], int32_t* device_status, void* stream);
+int sva_scatter_tokens(const void* src, const int64_t src_stride[3], const int32_t* token_idx, int32_t B, int32_t H,
+                       int32_t M, int32_t n_dst, int32_t d, int32_t elem_bytes, void* dst,
+                       const int64_t dst_stride[3], int32_t* device_status, void* stream);
+
 const char* sva_status_string(int status);
 
 #ifdef __cplusplus

@@ -201,3 +201,25 @@ def select_from_qk(q, k, N: int, block: int, scale: float, mode: int, kk: int, t
     """O1-O7 end to end. Returns (Selection, scores [B,H,Nb,Nb])."""
     s = block_scores(pool(q, N, block), pool(k, N, block), scale)
     return select(s, mode, kk, tau, win_t, win_s, blocks_per_frame), s
+
+
+def gather_tokens(x: np.ndarray, token_idx: np.ndarray) -> np.ndarray:
+    """Token-subset gather (the paper's token pruning keeps a subset of the tokens):
+    out[b, h, m, :] = x[b, h, token_idx[b, m], :].  The definition written out, one row at a time."""
+    Bq, Hq, _, d = x.shape
+    M = token_idx.shape[1]
+    out = np.zeros((Bq, Hq, M, d), x.dtype)
+    for b in range(Bq):
+        for m in range(M):
+            out[b, :, m, :] = x[b, :, int(token_idx[b, m]), :]
+    return out
+
+
+def scatter_tokens(x: np.ndarray, token_idx: np.ndarray, dst: np.ndarray) -> np.ndarray:
+    """Inverse of gather_tokens: a copy of dst with dst[b, h, token_idx[b, m], :] = x[b, h, m, :];
+    the rows that token_idx does not name keep their contents."""
+    out = dst.copy()
+    for b in range(x.shape[0]):
+        for m in range(token_idx.shape[1]):
+            out[b, :, int(token_idx[b, m]), :] = x[b, :, m, :]
+    return out

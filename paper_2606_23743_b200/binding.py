@@ -22,7 +22,7 @@ EXPORTS = [
     "sva_select_max_nnz", "sva_select_workspace_bytes", "sva_block_select",
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
-    "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared",
+    "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -78,6 +78,10 @@ def lib():
         L.sva_attn_prepare_v.argtypes = [C.POINTER(Problem), vp, vp, C.c_size_t, vp]
         L.sva_block_sparse_attn_fwd_prepared.restype = C.c_int
         L.sva_block_sparse_attn_fwd_prepared.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        for fn in (L.sva_gather_tokens, L.sva_scatter_tokens):
+            fn.restype = C.c_int
+            fn.argtypes = [vp, C.POINTER(C.c_int64), vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                           C.c_int32, vp, C.POINTER(C.c_int64), vp, vp]
         L.sva_quantize_qk_fp8.restype = C.c_int
         L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
         L.sva_status_string.restype = C.c_char_p
@@ -197,6 +201,26 @@ def block_sparse_attn_fwd_prepared(p: Problem, q, k, row_ptr, col_idx, o, lse=No
                                                   _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_fwd_prepared")
+
+
+def _token_move(name, src, token_idx, dst, status):
+    Bq, Hq, n_src, d = src.shape
+    M = token_idx.shape[1]
+    n_full = dst.shape[2] if name == "sva_scatter_tokens" else n_src
+    rc = getattr(lib(), name)(_ptr(src), _strides(src), _ptr(token_idx), Bq, Hq, M, n_full, d, src.element_size(),
+                              _ptr(dst), _strides(dst), _ptr(status), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, name)
+
+
+def gather_tokens(src, token_idx, dst, status=None) -> None:
+    """dst[b,h,m,:] = src[b,h,token_idx[b,m],:]; src [B,H,N,d], token_idx [B,M] int32, dst [B,H,>=M,d]."""
+    _token_move("sva_gather_tokens", src, token_idx, dst, status)
+
+
+def scatter_tokens(src, token_idx, dst, status=None) -> None:
+    """dst[b,h,token_idx[b,m],:] = src[b,h,m,:]; the other rows of dst keep their contents."""
+    _token_move("sva_scatter_tokens", src, token_idx, dst, status)
 
 
 def quantize_qk_fp8(p: Problem, q, k, q8, k8, q_scale, k_scale) -> None:

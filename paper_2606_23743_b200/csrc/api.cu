@@ -199,6 +199,37 @@ int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* 
   return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, (cudaStream_t)stream);
 }
 
+static int validate_token_move(const void* a, const int64_t sa[3], const void* b, const int64_t sb[3],
+                               const int32_t* idx, int B, int H, int M, int n_full, int d, int elem_bytes) {
+  if (!a || !b || !idx || !sa || !sb) return SVA_ERR_INVALID_ARG;
+  if (B <= 0 || H <= 0 || M <= 0 || n_full <= 0 || M > n_full || d <= 0) return SVA_ERR_INVALID_ARG;
+  if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4) return SVA_ERR_INVALID_ARG;
+  if ((d * elem_bytes) % 16 != 0) return SVA_ERR_UNSUPPORTED;
+  if (!aligned16(a) || !aligned16(b)) return SVA_ERR_ALIGNMENT;
+  for (int i = 0; i < 3; ++i)
+    if (sa[i] < 0 || sb[i] < 0 || (sa[i] * elem_bytes) % 16 != 0 || (sb[i] * elem_bytes) % 16 != 0) return SVA_ERR_ALIGNMENT;
+  if (sa[2] < d || sb[2] < d) return SVA_ERR_INVALID_ARG;
+  return SVA_OK;
+}
+
+int sva_gather_tokens(const void* src, const int64_t src_stride[3], const int32_t* token_idx, int32_t B, int32_t H,
+                      int32_t M, int32_t n_src, int32_t d, int32_t elem_bytes, void* dst,
+                      const int64_t dst_stride[3], int32_t* device_status, void* stream) {
+  int rc = validate_token_move(src, src_stride, dst, dst_stride, token_idx, B, H, M, n_src, d, elem_bytes);
+  if (rc) return rc;
+  return launch_token_move(false, src, src_stride, dst, dst_stride, token_idx, B, H, M, n_src, d, elem_bytes,
+                           device_status, (cudaStream_t)stream);
+}
+
+int sva_scatter_tokens(const void* src, const int64_t src_stride[3], const int32_t* token_idx, int32_t B, int32_t H,
+                       int32_t M, int32_t n_dst, int32_t d, int32_t elem_bytes, void* dst,
+                       const int64_t dst_stride[3], int32_t* device_status, void* stream) {
+  int rc = validate_token_move(src, src_stride, dst, dst_stride, token_idx, B, H, M, n_dst, d, elem_bytes);
+  if (rc) return rc;
+  return launch_token_move(true, src, src_stride, dst, dst_stride, token_idx, B, H, M, n_dst, d, elem_bytes,
+                           device_status, (cudaStream_t)stream);
+}
+
 const char* sva_status_string(int status) {
   switch (status) {
     case SVA_OK: return "ok";

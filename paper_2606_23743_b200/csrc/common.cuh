@@ -52,6 +52,9 @@ int launch_select_noalloc(const Dims& m, const sva_problem_t* p, const sva_selec
 int select_row_cap(const Dims& m, const sva_select_t* s);
 int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
                     void* k8, float* qs, float* ks, cudaStream_t st);
+int launch_token_move(bool scatter, const void* src, const int64_t ss[3], void* dst, const int64_t sd[3],
+                      const int32_t* idx, int B, int H, int M, int n_full, int d, int elem_bytes,
+                      int32_t* status, cudaStream_t st);
 int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const void* k,
                      const void* v, const float* qs, const float* ks, const int32_t* row_ptr,
                      const int32_t* col_idx, void* o, float* lse, int32_t* status, cudaStream_t st);

@@ -121,3 +121,19 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "_LIB_PATH", "/nonexistent/libsva.so")
     with pytest.raises(RuntimeError, match="no fallback"):
         B.lib()
+
+
+def test_token_move_rejects_bad_arguments_before_launch(lib):
+    one = C.c_void_p(256)
+    st3 = (C.c_int64 * 3)(2 * 1024 * 128, 1024 * 128, 128)
+    def mv(fn, src=one, idx=one, dst=one, B_=1, H=2, M=512, n=1024, d=128, eb=2, ss=st3, sd=st3):
+        return fn(src, ss, idx, B_, H, M, n, d, eb, dst, sd, None, None)
+    for fn in (lib.sva_gather_tokens, lib.sva_scatter_tokens):
+        assert mv(fn, src=None) == 1
+        assert mv(fn, idx=None) == 1
+        assert mv(fn, M=2048) == 1                       # more kept tokens than tokens
+        assert mv(fn, eb=3) == 1
+        assert mv(fn, d=100) == 2                        # rows must be whole 16-byte vectors
+        assert mv(fn, dst=C.c_void_p(8)) == 5
+        assert mv(fn, ss=(C.c_int64 * 3)(0, 0, 132)) == 5
+        assert mv(fn, ss=(C.c_int64 * 3)(0, 0, 64)) == 1  # row stride shorter than a row
