@@ -8,10 +8,10 @@
 //   * Q is written into TMEM once per row by the softmax threads (straight from global memory);
 //   * V is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed copy
 //     that a small kernel writes into the caller's workspace first.
-// The kernel is persistent: CTA c processes the CSR rows c, c + gridDim.x, ... (one row = one query
-// block of one head, 128 query rows).  All barriers keep running across rows (every role derives the
-// same phase counters from the same row sequence), so the producers run ahead into the next row
-// while the softmax groups finish the current one.
+// The kernel is persistent: one CTA per SM takes rows (one row = one query block of one head, 128
+// query rows) from a device-wide counter until none is left.  All barriers keep running across rows
+// (every role derives the same phase counters from the same row sequence), so the producers run
+// ahead into the next row while the softmax groups finish the current one.
 //   warps 0-3, 4-7  two softmax warpgroups; they take the kept key blocks alternately (even / odd
 //                   position in the row's list); thread <-> query row <-> TMEM lane
 //   warp  8         producer of the K tiles (TMA, one lane)
