@@ -166,8 +166,9 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
  * the prepared layout itself.  sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
  * and key block one contiguous tile [d][block keys], keys >= N zero) and resets the row counter in
  * `workspace`; sva_block_sparse_attn_fwd_prepared then runs the attention kernel alone (row_ptr ==
- * NULL means dense).  One prepare per attention call (the attention call uses the counter up), and
- * the caller orders the two (same stream, or an event).  Together they do exactly what
+ * NULL means dense).  A prepared workspace serves any number of attention calls on that V that do
+ * not overlap on the GPU (after a call that reported SVA_DEV_TIMEOUT, prepare again); the caller
+ * orders prepare and attention (same stream, or an event).  Together they do exactly what
  * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call.  SVA_ERR_UNSUPPORTED for problems
  * the bf16 tensor-core kernel does not serve (e4m3 Q/K, d other than 128) and for the dense form with
  * 64-token blocks: use the one-call entry points there.

@@ -68,7 +68,7 @@ struct TsParams {
   const int32_t* tile_beg;    // ... and where its descriptors start
   const uint32_t* tile_desc;  // two 16-bit halves {key block (14 bits), kept by query block A, kept by B}
   float scale_log2;           // softmax_scale * log2(e)
-  int32_t* next_row;          // device counter (starts at 0): the next CSR row to hand out
+  int32_t* next_row;          // two device counters (both start at 0): the next row to hand out, CTAs done drawing
   long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
   int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
                               // bit4: starve the pipeline so that a wait runs out (test aid)
@@ -249,7 +249,15 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           rowq[8 * slot + 3] = (int)e0;
           rowq[8 * slot + 4] = (int)e1;
           mbar_arrive(bar_rq_full + 8 * slot);
-          if (r >= prm.R) break;
+          if (r >= prm.R) {
+            // Every CTA ends by drawing one value >= R.  The last one to do so puts both counters back to 0,
+            // so a prepared workspace serves further attention calls on the same V.
+            if (atomicAdd(prm.next_row + 1, 1) == (int)gridDim.x - 1) {
+              prm.next_row[1] = 0;
+              prm.next_row[0] = 0;
+            }
+            break;
+          }
           // ---- K tiles of the row
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
           for (int j = 0; j < n; ++j) {
@@ -675,7 +683,10 @@ __global__ void __launch_bounds__(256)
 transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
                    int Nb, int d, int kb, int32_t* __restrict__ row_counter) {
   // the attention kernel that follows draws its rows from this counter
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *row_counter = 0;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) {
+    row_counter[0] = 0;     // next row to hand out
+    row_counter[1] = 0;     // CTAs that have finished drawing
+  }
   __shared__ __nv_bfloat16 tile[64][66];            // [d][key], padded
   const int n0 = blockIdx.x * 64, d0 = blockIdx.y * 64, bh = blockIdx.z;
   const int b = bh / H, h = bh % H;

@@ -114,6 +114,12 @@ def test_two_step_form_matches_the_one_call_form(name):
         assert int(status.item()) == 0
         ref_o, ref_l = (o1, l1) if sparse else (od, ld)
         assert torch.equal(o2[:, :, :w.N], ref_o[:, :, :w.N]) and torch.equal(l2, ref_l)   # rows >= N are never written
+        # the prepared workspace serves a second call on the same V
+        o2.fill_(3.0); l2.fill_(3.0)
+        B.block_sparse_attn_fwd_prepared(p, qd, kd, rp if sparse else None, ci if sparse else None, o2, l2, status,
+                                         workspace=ws)
+        torch.cuda.synchronize()
+        assert torch.equal(o2[:, :, :w.N], ref_o[:, :, :w.N]) and torch.equal(l2, ref_l)
 
 
 def test_empty_rows_and_bad_indices_are_reported_not_trapped():
