@@ -51,7 +51,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
     def __init__(self, device_index: int):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.reasons, self.max_mhz, self.power = [], set(), None, []
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -87,6 +87,7 @@ class ClockSampler:
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
                 self.reasons |= self._names(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
             except Exception:
                 pass
             time.sleep(0.002)
@@ -102,7 +103,7 @@ class ClockSampler:
             self._thread.join()
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "power_w_max": max(self.power) if self.power else None}
 
 
 def flops_per_tile(w):
