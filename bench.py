@@ -245,20 +245,26 @@ def main():
             B.attn_prepare_v(p, v, aws)
             v_ready.record()
 
+    # the two-step form serves what the bf16 tensor-core kernel serves; other shapes take the one call
+    two_step = (not w.fp8) and B.attn_workspace_bytes(p) > 0
+
     def route():
         if w.fp8:
             B.quantize_qk_fp8(pq, q, k, q8, k8, qs, ks)
             B.block_select(p, s, q8, k8, row_ptr, col_idx, ws, qs, ks)
         else:
-            prepare_v()
+            if two_step:
+                prepare_v()
             B.block_select(p, s, q, k, row_ptr, col_idx, ws)
 
     def attend():
         if w.fp8:       # (the two-step form takes bf16 Q/K only: the one call transposes V itself)
             B.block_sparse_attn_fwd(p, q8, k8, v, row_ptr, col_idx, o, None, status, qs, ks, workspace=aws)
-        else:
+        elif two_step:
             torch.cuda.current_stream().wait_event(v_ready)
             B.block_sparse_attn_fwd_prepared(p, q, k, row_ptr, col_idx, o, None, status, workspace=aws)
+        else:
+            B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status, workspace=aws)
 
     def step():
         route()
