@@ -106,7 +106,11 @@ constexpr float LAZY_LOG2 = 32.0f;
 // inputs and so reaches the same answer.
 template <bool B64>
 __device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int& beg) {
-  if (B64) { n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r); return; }
+  if (B64) {
+    if (prm.row_ptr == nullptr) { n = (prm.Nb + 1) >> 1; beg = 0; return; }     // dense: every pair of key blocks
+    n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r);
+    return;
+  }
   if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return; }
   beg = __ldg(prm.row_ptr + r);
   n = __ldg(prm.row_ptr + r + 1) - beg;
@@ -116,7 +120,13 @@ __device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int
 // the producer reports it).  64-token blocks: the tile descriptor.
 template <bool B64>
 __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j) {
-  if (B64) return __ldg(prm.tile_desc + beg + j);
+  if (B64) {
+    if (prm.row_ptr == nullptr) {        // dense: key blocks 2j and 2j+1 (if it exists), kept by both query blocks
+      const uint32_t u0 = 2u * (uint32_t)j, u1 = u0 + 1u;
+      return (u0 | 0xc000u) | (u1 < (uint32_t)prm.Nb ? (u1 | 0xc000u) << 16 : 0u);
+    }
+    return __ldg(prm.tile_desc + beg + j);
+  }
   if (prm.row_ptr == nullptr) return (uint32_t)j;
   const int J = __ldg(prm.col_idx + beg + j);
   return (J < 0 || J >= prm.Nb) ? 0u : (uint32_t)J;
@@ -267,12 +277,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             mbar_expect_tx(bar_k_full + 8 * s, KTILE);
             if (B64) {
               // two 64-key blocks side by side: rows 0..63 and 64..127 of both d-panels
-              const uint32_t dsc = __ldg(prm.tile_desc + beg + j);
+              // (e4m3: one 128-byte panel, so one load per key block)
+              const uint32_t dsc = list_block<B64>(prm, beg, j);
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
                 const int J = (int)((dsc >> (16 * h)) & 0x3fffu);
                 tma_load_4d(dst + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 0, J * KB, hh, bb);
-                tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 64, J * KB, hh, bb);
+                if (!F8) tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 64, J * KB, hh, bb);
               }
             } else {
               int J = j;
@@ -408,6 +419,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const int tail_keys = prm.N - (prm.Nb - 1) * KB;         // valid keys of the last key block
     const int qh = row >> 6;                                 // 64-token blocks: which query block of the tile I am in
     float c = prm.scale_log2;      // e4m3 variant: times the scales of the query block and of the key block, per block
+    float c1 = prm.scale_log2;     // e4m3 with 64-token blocks: the same for the tile's second key block
     uint32_t cnt[2] = {0, 0};      // blocks of parity 0 / 1 completed in earlier rows (barrier phase bases)
     uint32_t rows_done = 0;        // non-empty rows finished
     bool ok = true;
@@ -459,10 +471,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const uint32_t last = cnt[wl] + (uint32_t)((n - 1) >> 1);       // phase index of that block
       float m_mine = -INFINITY;      // reference exponent my partial row sum is relative to
       float l = 0.f;                 // partial row sum over this group's blocks
-      float qs_row = 1.f, ks_next = 1.f;
+      float qs_row = 1.f, ks_next = 1.f, ks_next1 = 1.f;
+      auto load_ks = [&](uint32_t e) {                                // scales of the key block(s) of list entry e
+        const float* ks = prm.k_scale + (long long)bh * prm.Nb;
+        if (B64) {
+          ks_next = __ldg(ks + (int)(e & 0x3fffu));
+          ks_next1 = __ldg(ks + (int)((e >> 16) & 0x3fffu));
+        } else {
+          ks_next = __ldg(ks + (int)e);
+        }
+      };
       if (F8) {
-        qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + I) * prm.scale_log2;
-        if (w < n) ks_next = __ldg(prm.k_scale + (long long)bh * prm.Nb + (int)J);
+        const int qb = B64 ? min(2 * I + qh, prm.Nb - 1) : I;         // my query block
+        qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + qb) * prm.scale_log2;
+        if (w < n) load_ks(J);
       }
       for (int j = w; j < n; j += 2) {
         const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
@@ -478,10 +500,10 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           v0 = ((int)J == prm.Nb - 1) ? tail_keys : BS;      // 128-token blocks: all valid keys counted in v0
           v1 = 0;
         }
-        if (F8) c = qs_row * ks_next;
+        if (F8) { c = qs_row * ks_next; if (B64) c1 = qs_row * ks_next1; }
         if (j + 2 < n) {                                               // one entry ahead
           J = list_block<B64>(prm, lbeg, j + 2);
-          if (F8) ks_next = __ldg(prm.k_scale + (long long)bh * prm.Nb + (int)J);
+          if (F8) load_ks(J);
         }
         if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
         tc_fence_after();
@@ -535,7 +557,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           mx0 = fmaxf(mxa, mxb);
           mx1 = fmaxf(mxc, mxd);
         }
-        const float mx = fmaxf(mx0, mx1) * c;
+        // (e4m3 with 64-token blocks: each half has its own scale; a half that is not kept stays -inf)
+        const float mx = (B64 && F8) ? fmaxf(v0 > 0 ? mx0 * c : -INFINITY, v1 > 0 ? mx1 * c1 : -INFINITY)
+                                     : fmaxf(mx0, mx1) * c;
         // reference exponent left by block j-1 (other group)
         float m_prev = -INFINITY;
         if (j > 0) {
@@ -574,12 +598,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (m_new == -INFINITY || v1 == 0) nmh1 = -INFINITY;
         }
         const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm), nm2h1 = B64 ? pack2(nmh1, nmh1) : nm2;
+        const uint64_t c2h1 = (B64 && F8) ? pack2(c1, c1) : c2;
         uint64_t sum2 = pack2(0.f, 0.f);
         if (!(prm.debug & 1)) {
 #pragma unroll
           for (int e = 0; e < 128; e += 2) {
             float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, e < 64 ? nm2 : nm2h1), x0, x1);
+            unpack2(fma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), e < 64 ? c2 : c2h1, e < 64 ? nm2 : nm2h1), x0, x1);
             const float p0 = ex2(x0), p1 = ex2(x1);
             sum2 = add2(sum2, pack2(p0, p1));
             sv[e / 2] = pack_bf16(p0, p1);
@@ -867,7 +892,7 @@ static TsLayout ts_layout(const Dims& m) {
 }
 
 bool attn_ts_serves(const Dims& m) {
-  return m.d == 128 && m.Nb <= 16383 && (m.block == BS || (m.block == 64 && !m.fp8));
+  return m.d == 128 && m.Nb <= 16383 && (m.block == BS || m.block == 64);
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {
@@ -910,7 +935,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   if (rc) return rc;
   // dense attention does not depend on the block size: 64-token blocks run as 128-token blocks
   Dims m = m_in;
-  if (m.block == 64 && row_ptr == nullptr) {
+  if (m.block == 64 && row_ptr == nullptr && !m.fp8) {     // (e4m3 scales are per 64-token block: that stays as it is)
     m.block = BS;
     m.Nb = (m.N + BS - 1) / BS;
     m.R = m.B * m.H * m.Nb;
@@ -957,11 +982,13 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
   if (b64) {
-    pair_lists_kernel<<<(L.R2 + PAIR_WARPS - 1) / PAIR_WARPS, PAIR_WARPS * 32, 0, st>>>(
-        row_ptr, col_idx, m.Nb, L.Nt, L.R2, reinterpret_cast<int32_t*>(wsb + L.cnt_off),
-        reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
-    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
-    return launch_ts<true, false>(L.R2, tk, tv, to, prm, st);
+    if (row_ptr) {                      // (dense, e4m3 only: the kernel makes up the tile lists itself)
+      pair_lists_kernel<<<(L.R2 + PAIR_WARPS - 1) / PAIR_WARPS, PAIR_WARPS * 32, 0, st>>>(
+          row_ptr, col_idx, m.Nb, L.Nt, L.R2, reinterpret_cast<int32_t*>(wsb + L.cnt_off),
+          reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
+      if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+    }
+    return m.fp8 ? launch_ts<true, true>(L.R2, tk, tv, to, prm, st) : launch_ts<true, false>(L.R2, tk, tv, to, prm, st);
   }
   if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, prm, st);
   return launch_ts<false, false>(L.R2, tk, tv, to, prm, st);

@@ -54,3 +54,27 @@ def test_fp8_select_and_attention(impl):
     rows = U.sample_rows(w.R, w.Nb, 10)
     r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
     print(f"fp8/{impl}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")
+
+
+@pytest.mark.parametrize("impl", ["tensor", "simt", "tensor-dense"])
+def test_fp8_64_token_blocks(impl):
+    """e4m3 Q/K with one scale per 64-token block: the tensor-core kernel pairs blocks into 128-wide
+    tiles, so the two halves of a tile (and of a tile row) carry different scales.  N = 3 * 1560 = 4680
+    = 73 blocks + 8 tokens: odd block count, ragged last block."""
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=3, block=64, mode=0, k=9)
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8, k8, qs, ks = _quantize(w, qd, kd)
+    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
+    sel, _ = U.oracle_select(w, qh, kh)
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    assert n_diff <= n_near
+    dense = impl == "tensor-dense"
+    o, lse, st = U.gpu_attn(w, q8, k8, vd, rp, ci, simt=(impl == "simt"), dense=dense, q_scale=qs, k_scale=ks,
+                            fp8=True)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, 6 if dense else 12)
+    r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, dense=dense, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
+    print(f"fp8 b64/{impl}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")
