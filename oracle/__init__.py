@@ -82,15 +82,36 @@ def e4m3_encode(x: float) -> int:
     return int(lib().svo_e4m3_encode(C.c_float(x)))
 
 
-def quantize_e4m3(x_bf16: np.ndarray, N: int, block: int):
-    """O10: per-(b,h,block) absmax scale, e4m3 codes. Returns (codes u8, scales f32 [B,H,Nb])."""
+def quantize_e4m3(x_bf16: np.ndarray, N: int, block: int, sub: np.ndarray | None = None):
+    """O10: per-(b,h,block) absmax scale, e4m3 codes. Returns (codes u8, scales f32 [B,H,Nb]).
+    sub ([B,H,d] fp32, optional) is subtracted from every token in fp32 first: the K smoothing step
+    of the 8-bit attention work the paper cites for its quantised attention (see k_mean)."""
     x = _c(x_bf16)
     B, H, n_alloc, d = x.shape
     Nb = -(-N // block)
     codes = np.zeros(x.shape, np.uint8)
     scales = np.zeros((B, H, Nb), np.float32)
-    lib().svo_quantize_e4m3(_p(x), B * H, N, n_alloc, d, block, _p(codes), _p(scales))
+    if sub is not None:
+        sub = _c(np.asarray(sub, np.float32))
+        assert sub.shape == (B, H, d)
+    lib().svo_quantize_e4m3(_p(x), _p(sub), B * H, N, n_alloc, d, block, _p(codes), _p(scales))
     return codes, scales
+
+
+def k_mean(k: np.ndarray, N: int) -> np.ndarray:
+    """K smoothing, step 1: the mean key of each (b,h) over the N tokens that exist -> [B,H,d] float64.
+    Subtracting it from every key adds the same amount, -scale*<q_i, mean>, to every logit of query i, so
+    the softmax over keys -- and with it O and the kept-mass of any block set -- does not change, while
+    the keys lose their common offset (which would otherwise eat the e4m3 range)."""
+    kf = bf16_to_f64(k) if k.dtype == np.uint16 else np.asarray(k, np.float64)
+    return kf[:, :, :N].mean(axis=2)
+
+
+def lse_shift(q: np.ndarray, mean: np.ndarray, N: int, scale: float) -> np.ndarray:
+    """K smoothing, step 2: what the smoothed problem's log-sum-exp is short of the original's,
+    scale * <q_i, mean> -> [B,H,N] float64 (lse_original = lse_smoothed + lse_shift)."""
+    qf = bf16_to_f64(q) if q.dtype == np.uint16 else np.asarray(q, np.float64)
+    return scale * np.einsum("bhnd,bhd->bhn", qf[:, :, :N], np.asarray(mean, np.float64))
 
 
 def dequantize_e4m3(codes: np.ndarray, scales: np.ndarray, N: int, block: int) -> np.ndarray:

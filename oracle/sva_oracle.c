@@ -103,8 +103,10 @@ uint8_t svo_e4m3_encode(float xf) {
 }
 
 /* Per (b,h,block) absmax scale in fp32, y = x / s in fp32, cast.  x is bf16
- * bits laid out [BH, n_alloc, d].  codes has the same layout; scales [BH, Nb]. */
-void svo_quantize_e4m3(const uint16_t *x, int BH, int N, int n_alloc, int d, int block,
+ * bits laid out [BH, n_alloc, d].  codes has the same layout; scales [BH, Nb].
+ * sub (may be NULL): [BH, d] fp32, subtracted from every token in fp32 before anything
+ * else -- the K smoothing step (k_j - mean over tokens), one rounding per element. */
+void svo_quantize_e4m3(const uint16_t *x, const float *sub, int BH, int N, int n_alloc, int d, int block,
                        uint8_t *codes, float *scales) {
   int Nb = (N + block - 1) / block;
 #pragma omp parallel for collapse(2) schedule(static)
@@ -114,7 +116,9 @@ void svo_quantize_e4m3(const uint16_t *x, int BH, int N, int n_alloc, int d, int
       float a = 0.0f;
       for (int i = lo; i < hi; ++i)
         for (int c = 0; c < d; ++c) {
-          float v = fabsf((float)bf16_to_f64(x[((size_t)bh * n_alloc + i) * d + c]));
+          volatile float xv = (float)bf16_to_f64(x[((size_t)bh * n_alloc + i) * d + c]);
+          if (sub) xv = xv - sub[(size_t)bh * d + c];
+          float v = fabsf(xv);
           if (v > a) a = v;
         }
       volatile float s = (a == 0.0f) ? 1.0f : a / 448.0f;
@@ -122,7 +126,9 @@ void svo_quantize_e4m3(const uint16_t *x, int BH, int N, int n_alloc, int d, int
       for (int i = lo; i < hi; ++i)
         for (int c = 0; c < d; ++c) {
           size_t o = ((size_t)bh * n_alloc + i) * d + c;
-          volatile float y = (float)bf16_to_f64(x[o]) / s;
+          volatile float xv = (float)bf16_to_f64(x[o]);
+          if (sub) xv = xv - sub[(size_t)bh * d + c];
+          volatile float y = xv / s;
           codes[o] = svo_e4m3_encode(y);
         }
     }

@@ -78,3 +78,75 @@ def test_quantize_blocks_scales_and_error_bound():
     big = np.abs(ref) > amax * 2.0 ** -6
     assert (err[big] <= np.abs(ref[big]) * 2.0 ** -4 * (1 + 1e-6)).all()
     assert (xhat[:, :, N:] == 0).all()
+
+
+# ------------------------------------------------------------------ K smoothing
+def _offset_qkv(seed=7, B=1, H=2, N=200, n_alloc=256, d=16, offset=6.0):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(B, H, n_alloc, d, generator=g).bfloat16()
+    k = (torch.randn(B, H, n_alloc, d, generator=g) + offset * torch.randn(B, H, 1, d, generator=g)).bfloat16()
+    v = torch.randn(B, H, n_alloc, d, generator=g).bfloat16()
+    q[:, :, N:] = 0; k[:, :, N:] = 50.0; v[:, :, N:] = 0             # absent keys must not enter the mean
+    bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+    return (q, k, v), (bits(q), bits(k), bits(v))
+
+
+def test_k_mean_closed_forms():
+    (q, k, v), (qb, kb, vb) = _offset_qkv()
+    N = 200
+    m = oracle.k_mean(kb, N)
+    assert m.shape == (1, 2, 16)
+    np.testing.assert_allclose(m, k.double()[:, :, :N].mean(dim=2).numpy(), rtol=1e-13, atol=1e-13)
+    # a constant key sequence is its own mean; an antisymmetric one has mean 0
+    c = np.full((1, 1, 8, 4), 2.5)
+    np.testing.assert_array_equal(oracle.k_mean(c, 6), np.full((1, 1, 4), 2.5))
+    a = np.arange(-3, 4, dtype=np.float64).reshape(1, 1, 7, 1) * np.ones((1, 1, 1, 4))
+    np.testing.assert_allclose(oracle.k_mean(a, 7), 0.0, atol=1e-15)
+
+
+def test_smoothing_leaves_softmax_unchanged_and_shifts_lse():
+    """Attention over (q, k - mean) equals attention over (q, k); lse moves by scale*<q, mean>."""
+    (q, k, v), (qb, kb, vb) = _offset_qkv()
+    N, block, scale = 200, 64, 0.25
+    qf, kf, vf = (oracle.bf16_to_f64(x) for x in (qb, kb, vb))
+    mean = oracle.k_mean(kb, N)
+    ks = kf - mean[:, :, None, :]
+    o0, l0 = oracle.dense_attn_rows(qf, kf, vf, N, block, scale)
+    o1, l1 = oracle.dense_attn_rows(qf, ks, vf, N, block, scale)
+    shift = oracle.lse_shift(qb, mean, N, scale)                      # [B,H,N]
+    Nb = -(-N // block)
+    for r in range(2 * Nb):
+        bh, I = divmod(r, Nb)
+        lo, hi = I * block, min((I + 1) * block, N)
+        np.testing.assert_allclose(o1[r, : hi - lo], o0[r, : hi - lo], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(l1[r, : hi - lo] + shift[0, bh, lo:hi], l0[r, : hi - lo], rtol=0, atol=1e-11)
+    # block routing sees the same thing: every row of the pooled scores moves by one constant
+    s0 = oracle.block_scores(oracle.pool(qf, N, block), oracle.pool(kf, N, block), scale)
+    s1 = oracle.block_scores(oracle.pool(qf, N, block), oracle.pool(ks, N, block), scale)
+    dlt = s0 - s1
+    np.testing.assert_allclose(dlt, dlt[..., :1] * np.ones_like(dlt), rtol=0, atol=1e-11)
+
+
+def test_quantize_with_subtraction():
+    (q, k, v), (qb, kb, vb) = _offset_qkv()
+    N, block = 200, 64
+    mean = oracle.k_mean(kb, N).astype(np.float32)
+    # no subtraction and a zero subtraction are the same thing
+    c0, s0 = oracle.quantize_e4m3(kb, N, block)
+    cz, sz = oracle.quantize_e4m3(kb, N, block, sub=np.zeros_like(mean))
+    np.testing.assert_array_equal(c0, cz); np.testing.assert_array_equal(s0, sz)
+    # against the library cast of the same fp32 arithmetic
+    cs, ss = oracle.quantize_e4m3(kb, N, block, sub=mean)
+    kc = k.float() - torch.from_numpy(mean)[:, :, None, :]
+    for h in range(2):
+        for I in range(4):
+            lo, hi = I * block, min((I + 1) * block, N)
+            a = kc[0, h, lo:hi].abs().max()
+            assert ss[0, h, I] == np.float32(a / 448.0)
+            lib = (kc[0, h, lo:hi] / torch.tensor(ss[0, h, I])).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+            np.testing.assert_array_equal(cs[0, h, lo:hi], lib)
+    # what it is for: with a common offset in K the smoothed codes reproduce K far better
+    kf = oracle.bf16_to_f64(kb)[:, :, :N]
+    e_plain = np.abs(oracle.dequantize_e4m3(c0, s0, N, block)[:, :, :N] - kf).mean()
+    e_smooth = np.abs(oracle.dequantize_e4m3(cs, ss, N, block)[:, :, :N] + mean[:, :, None, :].astype(np.float64) - kf).mean()
+    assert e_smooth < 0.6 * e_plain, (e_smooth, e_plain)
