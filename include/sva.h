@@ -199,6 +199,26 @@ int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* 
                         void* k8, float* q_scale, float* k_scale, void* stream);
 
 /*
+ * The same quantiser with K smoothing, the step the 8-bit attention work cited in the paper's related
+ * work on quantised attention puts before the cast: per (b,h) the mean key over the N tokens,
+ *   k_mean[b,h,:] = (1/N) sum_j k[b,h,j,:]        (fp32; per-block sums in a fixed order, then the blocks in
+ *                                                   index order, so the result is reproducible)
+ * is subtracted from every key in fp32 (one rounding) and k - k_mean is what gets scaled and cast.  Every
+ * logit of query i changes by the same -scale*<q_i, k_mean>, so softmax over keys, O, pooled-score order
+ * and kept mass are those of the original problem (up to rounding), while K loses the common offset that
+ * would otherwise use up the e4m3 range.  Only the log-sum-exp moves:
+ *   lse_original[b,h,i] = lse_of_the_quantised_problem[b,h,i] + lse_shift[b,h,i],
+ *   lse_shift[b,h,i] = scale * <q[b,h,i,:], k_mean[b,h,:]>   (from the bf16 q; optional, [B,H,N] fp32).
+ * Q is quantised as by sva_quantize_qk_fp8.  k_mean: [B,H,d] fp32, 16-byte aligned, written.  workspace:
+ * >= sva_smooth_workspace_bytes(p) = 4*B*H*Nb*d bytes, 16-byte aligned.
+ * Errors: as sva_quantize_qk_fp8, plus SVA_ERR_WORKSPACE.
+ */
+size_t sva_smooth_workspace_bytes(const sva_problem_t* p);
+int sva_quantize_qk_fp8_smooth_k(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q8,
+                                 void* k8, float* q_scale, float* k_scale, float* k_mean, float* lse_shift,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Token-subset gather / scatter (the paper's token pruning keeps a subset of the video tokens, about
  * half of them, on some denoising calls; attention then runs over the kept tokens only, and the
  * blocking of the routing applies to the gathered sequence).

@@ -23,6 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
+    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -84,6 +85,10 @@ def lib():
                            C.c_int32, vp, C.POINTER(C.c_int64), vp, vp]
         L.sva_quantize_qk_fp8.restype = C.c_int
         L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
+        L.sva_smooth_workspace_bytes.restype = C.c_size_t
+        L.sva_smooth_workspace_bytes.argtypes = [C.POINTER(Problem)]
+        L.sva_quantize_qk_fp8_smooth_k.restype = C.c_int
+        L.sva_quantize_qk_fp8_smooth_k.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.sva_status_string.restype = C.c_char_p
         L.sva_status_string.argtypes = [C.c_int]
         _lib = L
@@ -228,3 +233,15 @@ def quantize_qk_fp8(p: Problem, q, k, q8, k8, q_scale, k_scale) -> None:
                                    _ptr(k_scale), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_quantize_qk_fp8")
+
+
+def smooth_workspace_bytes(p: Problem) -> int:
+    return int(lib().sva_smooth_workspace_bytes(C.byref(p)))
+
+
+def quantize_qk_fp8_smooth_k(p: Problem, q, k, q8, k8, q_scale, k_scale, k_mean, lse_shift, workspace) -> None:
+    rc = lib().sva_quantize_qk_fp8_smooth_k(C.byref(p), _ptr(q), _ptr(k), _ptr(q8), _ptr(k8), _ptr(q_scale),
+                                            _ptr(k_scale), _ptr(k_mean), _ptr(lse_shift), _ptr(workspace),
+                                            C.c_size_t(workspace.numel() if workspace is not None else 0), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_quantize_qk_fp8_smooth_k")

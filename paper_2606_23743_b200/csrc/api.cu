@@ -195,7 +195,29 @@ int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* 
   if ((rc = check_strides(p->q_stride, 16))) return rc;
   if ((rc = check_strides(p->k_stride, 16))) return rc;
   Dims m = make_dims(p);
-  return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, (cudaStream_t)stream);
+  return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, nullptr, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+size_t sva_smooth_workspace_bytes(const sva_problem_t* p) {
+  if (validate_problem(p)) return 0;
+  return smooth_workspace_bytes(make_dims(p));
+}
+
+int sva_quantize_qk_fp8_smooth_k(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q8,
+                                 void* k8, float* q_scale, float* k_scale, float* k_mean, float* lse_shift,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q_bf16 || !k_bf16 || !q8 || !k8 || !q_scale || !k_scale || !k_mean) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q_bf16) || !aligned16(k_bf16) || !aligned16(q8) || !aligned16(k8) || !aligned16(k_mean))
+    return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, 16))) return rc;
+  if ((rc = check_strides(p->k_stride, 16))) return rc;
+  Dims m = make_dims(p);
+  if (!workspace || workspace_bytes < smooth_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return SVA_ERR_ALIGNMENT;
+  return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, k_mean, lse_shift, workspace,
+                         (cudaStream_t)stream);
 }
 
 static int validate_token_move(const void* a, const int64_t sa[3], const void* b, const int64_t sb[3],

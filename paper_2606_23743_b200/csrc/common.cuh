@@ -50,8 +50,9 @@ int launch_select_noalloc(const Dims& m, const sva_problem_t* p, const sva_selec
                           const void* q, const void* k, const float* q_scale, const float* k_scale,
                           int32_t* row_ptr, int32_t* col_idx, float* block_scores, cudaStream_t st);
 int select_row_cap(const Dims& m, const sva_select_t* s);
+size_t smooth_workspace_bytes(const Dims& m);
 int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
-                    void* k8, float* qs, float* ks, cudaStream_t st);
+                    void* k8, float* qs, float* ks, float* k_mean, float* lse_shift, void* ws, cudaStream_t st);
 int launch_token_move(bool scatter, const void* src, const int64_t ss[3], void* dst, const int64_t sd[3],
                       const int32_t* idx, int B, int H, int M, int n_full, int d, int elem_bytes,
                       int32_t* status, cudaStream_t st);

@@ -1,17 +1,57 @@
 // FP8 variant's quantiser: one absmax scale per (b, h, block), e4m3 codes.
 // One CTA per (block, head, tensor) keeps its 128 x d bf16 tile in registers between the
 // absmax pass and the cast, so Q and K are read once and written once (HBM-bound).
+// With K smoothing, two small kernels first reduce K to its mean key per (b, h) -- per-block sums
+// in a fixed order, then the blocks in index order, so the mean is reproducible -- and the
+// quantiser subtracts it from K in fp32 and writes scale * <q_i, mean> per query token.
 #include "common.cuh"
 
 namespace sva {
 
 static constexpr int QT = 256;
 
+// part[(bh*Nb + I)*D + c] = sum over the valid tokens of block I of k[.., c]   (grid Nb x BH)
+template <int D>
+__global__ void __launch_bounds__(QT)
+block_sum_kernel(const uint8_t* __restrict__ k, Strides sk, float* __restrict__ part, int H, int N, int block, int Nb) {
+  constexpr int VPR = D / 8, GROUPS = QT / VPR;
+  __shared__ float acc[GROUPS][D];
+  const int I = blockIdx.x, bh = blockIdx.y;
+  const uint8_t* src = k + ((long long)(bh / H) * sk.b + (long long)(bh % H) * sk.h) * 2;
+  const int lo = I * block, cnt = min(block, N - lo);
+  const int vec = threadIdx.x % VPR, grp = threadIdx.x / VPR;
+  float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int t = grp; t < cnt; t += GROUPS) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(src + (long long)(lo + t) * sk.n * 2) + vec);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { a[2 * e] += bf16lo(w[e]); a[2 * e + 1] += bf16hi(w[e]); }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[grp][vec * 8 + e] = a[e];
+  __syncthreads();
+  for (int c = threadIdx.x; c < D; c += QT) {
+    float t = 0.f;
+    for (int g = 0; g < GROUPS; ++g) t += acc[g][c];
+    part[((long long)bh * Nb + I) * D + c] = t;
+  }
+}
+
+// mean[bh*D + c] = (sum over blocks, in index order) / N                        (grid BH, D threads)
+__global__ void mean_key_kernel(const float* __restrict__ part, float* __restrict__ mean, int Nb, int D, int N) {
+  const int bh = blockIdx.x, c = threadIdx.x;
+  float t = 0.f;
+#pragma unroll 8
+  for (int I = 0; I < Nb; ++I) t += __ldg(part + ((long long)bh * Nb + I) * D + c);   // (loads run ahead; the order of the sum is fixed)
+  mean[(long long)bh * D + c] = __fdiv_rn(t, (float)N);
+}
+
 template <int D, int MAX_ROWS>
 __global__ void __launch_bounds__(QT)
 quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, Strides sq, Strides sk,
                 uint8_t* __restrict__ q8, uint8_t* __restrict__ k8, float* __restrict__ q_scale,
-                float* __restrict__ k_scale, int H, int N, int block, int Nb) {
+                float* __restrict__ k_scale, int H, int N, int block, int Nb,
+                const float* __restrict__ k_mean, float* __restrict__ lse_shift, float scale) {
   constexpr int VPR = D / 8;             // 16-byte vectors (8 bf16) per token row
   constexpr int GROUPS = QT / VPR;
   constexpr int PER = MAX_ROWS / GROUPS; // rows per thread
@@ -29,14 +69,39 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
 
   uint4 u[PER];
   float a = 0.f;
+  // K smoothing: this thread's 8 components of the head's mean key (K: subtracted; Q: dotted)
+  float mk[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (k_mean) {
+    const float4* mp = reinterpret_cast<const float4*>(k_mean + (long long)bh * D + vec * 8);
+    const float4 m0 = __ldg(mp), m1 = __ldg(mp + 1);
+    mk[0] = m0.x; mk[1] = m0.y; mk[2] = m0.z; mk[3] = m0.w; mk[4] = m1.x; mk[5] = m1.y; mk[6] = m1.z; mk[7] = m1.w;
+  }
+  const bool sub = k_mean != nullptr && which == 1;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     int t = grp + j * GROUPS;
     u[j] = make_uint4(0, 0, 0, 0);
     if (t < cnt) u[j] = __ldg(reinterpret_cast<const uint4*>(src + (long long)(lo + t) * s.n * 2) + vec);
     const uint32_t w[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
+    if (sub) {
+      if (t < cnt) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) a = fmaxf(a, fmaxf(fabsf(bf16lo(w[e])), fabsf(bf16hi(w[e]))));
+        for (int e = 0; e < 4; ++e)
+          a = fmaxf(a, fmaxf(fabsf(__fsub_rn(bf16lo(w[e]), mk[2 * e])), fabsf(__fsub_rn(bf16hi(w[e]), mk[2 * e + 1]))));
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) a = fmaxf(a, fmaxf(fabsf(bf16lo(w[e])), fabsf(bf16hi(w[e]))));
+    }
+    if (k_mean && which == 0 && lse_shift) {
+      // scale * <q_t, mean>: 8 products here, the rest of the row in the other VPR-1 lanes of the group
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) dot += bf16lo(w[e]) * mk[2 * e] + bf16hi(w[e]) * mk[2 * e + 1];
+#pragma unroll
+      for (int o = VPR / 2; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (vec == 0 && t < cnt) lse_shift[(long long)bh * N + lo + t] = dot * scale;
+    }
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
@@ -59,26 +124,41 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
     uint32_t out[2] = {0, 0};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      uint32_t c0 = __nv_cvt_float_to_fp8(__fdiv_rn(bf16lo(w[e]), sc), __NV_SATFINITE, __NV_E4M3);
-      uint32_t c1 = __nv_cvt_float_to_fp8(__fdiv_rn(bf16hi(w[e]), sc), __NV_SATFINITE, __NV_E4M3);
+      const float x0 = sub ? __fsub_rn(bf16lo(w[e]), mk[2 * e]) : bf16lo(w[e]);
+      const float x1 = sub ? __fsub_rn(bf16hi(w[e]), mk[2 * e + 1]) : bf16hi(w[e]);
+      uint32_t c0 = __nv_cvt_float_to_fp8(__fdiv_rn(x0, sc), __NV_SATFINITE, __NV_E4M3);
+      uint32_t c1 = __nv_cvt_float_to_fp8(__fdiv_rn(x1, sc), __NV_SATFINITE, __NV_E4M3);
       out[e >> 1] |= (c0 | (c1 << 8)) << (16 * (e & 1));
     }
     *reinterpret_cast<uint2*>(dst + (long long)(lo + t) * s.n + vec * 8) = make_uint2(out[0], out[1]);
   }
 }
 
+size_t smooth_workspace_bytes(const Dims& m) { return (size_t)m.B * m.H * m.Nb * m.d * sizeof(float); }
+
+// k_mean == nullptr: the plain quantiser.  Otherwise K smoothing: k_mean [B,H,d] is computed here (ws holds
+// the per-block sums), subtracted from K before the cast, and lse_shift (optional) [B,H,N] is written.
 int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
-                    void* k8, float* qs, float* ks, cudaStream_t st) {
+                    void* k8, float* qs, float* ks, float* k_mean, float* lse_shift, void* ws, cudaStream_t st) {
   dim3 g(m.Nb, m.B * m.H, 2);
   Strides sq = make_strides(p->q_stride), sk = make_strides(p->k_stride);
-  if (m.d == 128 && m.block <= 128)
+  if (!((m.d == 128 || m.d == 64) && m.block <= 128)) return SVA_ERR_UNSUPPORTED;
+  if (k_mean) {
+    dim3 g1(m.Nb, m.B * m.H);
+    if (m.d == 128)
+      block_sum_kernel<128><<<g1, QT, 0, st>>>((const uint8_t*)k, sk, (float*)ws, m.H, m.N, m.block, m.Nb);
+    else
+      block_sum_kernel<64><<<g1, QT, 0, st>>>((const uint8_t*)k, sk, (float*)ws, m.H, m.N, m.block, m.Nb);
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+    mean_key_kernel<<<m.B * m.H, m.d, 0, st>>>((const float*)ws, k_mean, m.Nb, m.d, m.N);
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+  }
+  if (m.d == 128)
     quantize_kernel<128, 128><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8,
-                                                (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb);
-  else if (m.d == 64 && m.block <= 128)
-    quantize_kernel<64, 128><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8,
-                                               (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb);
+                                                (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb, k_mean, lse_shift, m.scale);
   else
-    return SVA_ERR_UNSUPPORTED;
+    quantize_kernel<64, 128><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8,
+                                               (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb, k_mean, lse_shift, m.scale);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 

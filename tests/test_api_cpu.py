@@ -114,6 +114,14 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert lib.sva_quantize_qk_fp8(C.byref(p), one, one, one, None, one, one, None) == 1
     bad = _problem(); bad.k_stride = (C.c_int64 * 3)(0, 0, 136)
     assert lib.sva_quantize_qk_fp8(C.byref(bad), one, one, one, one, one, one, None) == 5
+    # the smoothing quantiser: k_mean and its workspace are required, the lse shift is optional
+    sm = lambda pp, mean=one, ws=one, nb=1 << 30: lib.sva_quantize_qk_fp8_smooth_k(
+        C.byref(pp), one, one, one, one, one, one, mean, None, ws, C.c_size_t(nb), None)
+    assert B.smooth_workspace_bytes(p) == 4 * 1 * 2 * 8 * 128
+    assert sm(p, mean=None) == 1
+    assert sm(p, ws=None) == 3 and sm(p, nb=B.smooth_workspace_bytes(p) - 1) == 3
+    assert sm(p, ws=vp(4096 + 8)) == 5
+    assert sm(bad) == 5
 
 
 def test_missing_library_fails_loudly(monkeypatch):

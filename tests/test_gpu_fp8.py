@@ -78,3 +78,77 @@ def test_fp8_64_token_blocks(impl):
     rows = U.sample_rows(w.R, w.Nb, 6 if dense else 12)
     r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, dense=dense, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
     print(f"fp8 b64/{impl}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")
+
+
+def _quantize_smooth(w, qd, kd, want_shift=True):
+    q8 = torch.zeros(qd.shape, dtype=torch.uint8, device="cuda")
+    k8 = torch.zeros(kd.shape, dtype=torch.uint8, device="cuda")
+    qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device="cuda")
+    ks = torch.zeros_like(qs)
+    mean = torch.full((w.B, w.H, w.d), 7.0, dtype=torch.float32, device="cuda")
+    shift = torch.full((w.B, w.H, w.N), 7.0, dtype=torch.float32, device="cuda") if want_shift else None
+    p = B.make_problem(qd, kd, None, None, w.N, w.block)
+    ws = torch.empty(B.smooth_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    B.quantize_qk_fp8_smooth_k(p, qd, kd, q8, k8, qs, ks, mean, shift, ws)
+    torch.cuda.synchronize()
+    return q8, k8, qs, ks, mean, shift
+
+
+@pytest.mark.parametrize("block", [128, 64])
+def test_smoothing_quantiser(block):
+    """Mean key against the fp64 mean; K codes and scales bit for bit against the oracle's quantiser
+    given that fp32 mean; Q untouched by the smoothing; lse shift against its definition."""
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=2, block=block)         # N = 3120, ragged
+    (q, k, _), (qb, kb, _) = U.host_inputs(w)
+    qd, kd = U.dev(q), U.dev(k)
+    q8, k8, qs, ks, mean, shift = _quantize_smooth(w, qd, kd)
+    m = mean.cpu().numpy()
+    m_ref = oracle.k_mean(kb, w.N)
+    assert np.abs(m - m_ref).max() <= 1e-5 * max(1.0, np.abs(m_ref).max())
+    codes, scales = oracle.quantize_e4m3(kb, w.N, w.block, sub=m)
+    np.testing.assert_array_equal(ks.cpu().numpy(), scales)
+    np.testing.assert_array_equal(k8.cpu().numpy()[:, :, :w.N], codes[:, :, :w.N])
+    assert (k8[:, :, w.N:] == 0).all()
+    qc, qsc = oracle.quantize_e4m3(qb, w.N, w.block)
+    np.testing.assert_array_equal(qs.cpu().numpy(), qsc)
+    np.testing.assert_array_equal(q8.cpu().numpy()[:, :, :w.N], qc[:, :, :w.N])
+    s_ref = oracle.lse_shift(qb, m, w.N, w.scale)
+    assert np.abs(shift.cpu().numpy() - s_ref).max() <= 1e-4 * max(1.0, np.abs(s_ref).max())
+    # the shift is optional
+    _quantize_smooth(w, qd, kd, want_shift=False)
+
+
+def test_smoothed_fp8_attention_is_closer_to_bf16_attention():
+    """Routing + attention on the smoothed codes: parity against the oracle on the dequantised
+    inputs (same tolerances as the plain FP8 variant), lse + shift against the oracle's lse of the
+    un-smoothed problem, and -- what the step is for -- a smaller distance to the attention of the
+    original bf16 Q, K than the plain FP8 variant has, on inputs whose keys share an offset."""
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=4)
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    g = torch.Generator().manual_seed(11)
+    k = (k.float() + 3.0 * torch.randn(w.B, w.H, 1, w.d, generator=g)).bfloat16()   # one offset per head, 3x the noise
+    k[:, :, w.N:] = 0
+    kb = k.view(torch.int16).numpy().view(np.uint16)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8, k8, qs, ks, mean, shift = _quantize_smooth(w, qd, kd)
+    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
+    sel, _ = U.oracle_select(w, qh, kh)
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    assert n_diff <= n_near
+    o, lse, st = U.gpu_attn(w, q8, k8, vd, rp, ci, q_scale=qs, k_scale=ks, fp8=True)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, 10)
+    U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
+    rpn, cin = rp.cpu().numpy(), ci.cpu().numpy()
+    # distance to the attention of the original bf16 inputs over the same block lists
+    # (lse: the smoothed problem's plus the shift, which is taken from the bf16 q, estimates the original's)
+    o_true, l_true = oracle.attn_rows(qb, kb, vb, w.N, w.block, w.scale, rpn, cin, rows=rows)
+    _, e_smooth, l_smooth = U.attn_errors(o, lse + shift, o_true, l_true, rows, w.N, w.block, w.H)
+    p8, pk8, pqs, pks = _quantize(w, qd, kd)
+    o_plain, lse_plain, st = U.gpu_attn(w, p8, pk8, vd, rp, ci, q_scale=pqs, k_scale=pks, fp8=True)
+    _, e_plain, l_plain = U.attn_errors(o_plain, lse_plain, o_true, l_true, rows, w.N, w.block, w.H)
+    print(f"to bf16 attention: rel-L2 plain fp8 {e_plain:.3e}, smoothed {e_smooth:.3e}; "
+          f"max lse error plain {l_plain:.3e}, smoothed {l_smooth:.3e}")
+    assert e_smooth < e_plain and l_smooth < l_plain
