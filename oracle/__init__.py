@@ -244,3 +244,27 @@ def scatter_tokens(x: np.ndarray, token_idx: np.ndarray, dst: np.ndarray) -> np.
         for m in range(token_idx.shape[1]):
             out[b, :, int(token_idx[b, m]), :] = x[b, :, m, :]
     return out
+
+
+def qk_norm_rope(x: np.ndarray, g: np.ndarray, cos: np.ndarray, sin: np.ndarray, N: int, eps: float) -> np.ndarray:
+    """The attention prologue the paper lists among its lossless fusion flags (fused QK-norm + RoPE), the two
+    steps one after the other in float64, for one of Q / K.  x [B,H,n_alloc,d] (bf16 bits or float64),
+    g [d], cos / sin [N, d/2].  Per token n and head:
+      RMS norm over the head dimension:  u_c = x_c / sqrt(mean_c(x_c^2) + eps) * g_c
+      rotary embedding on adjacent pairs: y_{2i}   = u_{2i} cos[n,i] - u_{2i+1} sin[n,i]
+                                          y_{2i+1} = u_{2i+1} cos[n,i] + u_{2i} sin[n,i]
+    Tokens >= N do not exist; their rows come back as zeros.  Returns float64 [B,H,n_alloc,d]."""
+    xf = bf16_to_f64(x) if x.dtype == np.uint16 else np.asarray(x, np.float64)
+    Bq, Hq, n_alloc, d = xf.shape
+    g = np.asarray(g, np.float64)
+    cos, sin = np.asarray(cos, np.float64), np.asarray(sin, np.float64)
+    assert g.shape == (d,) and cos.shape == (N, d // 2) and sin.shape == (N, d // 2)
+    out = np.zeros_like(xf)
+    for b in range(Bq):
+        for h in range(Hq):
+            xs = xf[b, h, :N]
+            u = xs / np.sqrt((xs * xs).mean(axis=1, keepdims=True) + eps) * g
+            ue, uo = u[:, 0::2], u[:, 1::2]
+            out[b, h, :N, 0::2] = ue * cos - uo * sin
+            out[b, h, :N, 1::2] = uo * cos + ue * sin
+    return out
