@@ -28,7 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2606_23743_b200 import dist as D  # noqa: E402
-from paper_2606_23743_b200.workloads import SEED_BASE, WORKLOADS, bf16_bits, make_qkv  # noqa: E402
+from paper_2606_23743_b200.workloads import SEED_BASE, WORKLOADS, bf16_bits, make_prologue_inputs, make_qkv  # noqa: E402
 
 METRIC = "block-sparse attn fwd effective TFLOPS (selected blocks)"
 UNIT = "TFLOP/s"
@@ -192,6 +192,9 @@ def main():
     ap.add_argument("--workload", default="large", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--prologue", action="store_true",
+                    help="extended step: the fused QK-norm + RoPE prologue in front (it also writes the block means, "
+                         "and the e4m3 codes of an FP8 workload, so routing skips its pooling pass and the quantiser)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -213,12 +216,17 @@ def main():
     o = torch.empty_like(v)
     oh = torch.empty(o.shape, dtype=o.dtype).pin_memory()
     p = B.make_problem(q, k, v, o, w.N, w.block)
+    pq = B.make_problem(q, k, None, None, w.N, w.block)
+    if args.prologue:
+        gq, gk, cos_t, sin_t = (x.to(dev) for x in make_prologue_inputs(w))
+        qn, kn = torch.empty_like(q), torch.empty_like(k)
+        qm = torch.empty(w.B, w.H, w.Nb, w.d, dtype=torch.float32, device=dev)
+        km = torch.empty_like(qm)
     if w.fp8:
         # FP8 variant: Q and K are quantised to e4m3 with per-block scales inside every step
         q8, k8 = torch.zeros(q.shape, dtype=torch.uint8, device=dev), torch.zeros(k.shape, dtype=torch.uint8, device=dev)
         qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device=dev)
         ks = torch.zeros_like(qs)
-        pq = B.make_problem(q, k, None, None, w.N, w.block)
         p = B.make_problem(q8, k8, v, o, w.N, w.block, 0.0, True)
     s = B.make_select(w.mode, w.k, w.tau, w.win_t, w.win_s, w.blocks_per_frame if w.win_t >= 0 else 0)
     ws = torch.empty(max(B.select_workspace_bytes(p, s), 256), dtype=torch.uint8, device=dev)
@@ -229,6 +237,8 @@ def main():
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
     # routing kernels + V transpose + attention (+ the tile-list kernel of the 64-token-block path)
     launches_per_step = (4 if variable_rows else 2) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
+    if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
+        launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
 
     # V is prepared (tiled transposed copy) on a second stream while routing, which never reads V, runs
     # (lower priority: its CTAs fill the SMs that the latency-bound selection kernel leaves idle instead of
@@ -249,7 +259,15 @@ def main():
     two_step = (not w.fp8) and B.attn_workspace_bytes(p) > 0
 
     def route(qq, kk, vv):
-        if w.fp8:
+        if args.prologue:
+            if two_step:
+                prepare_v(vv)
+            if w.fp8:
+                B.qk_norm_rope_pool(pq, qq, kk, gq, gk, cos_t, sin_t, 1e-6, qn, kn, qm, km, q8, k8, qs, ks)
+            else:
+                B.qk_norm_rope_pool(pq, qq, kk, gq, gk, cos_t, sin_t, 1e-6, qn, kn, qm, km)
+            B.block_select_pooled(p, s, qm, km, row_ptr, col_idx, ws)
+        elif w.fp8:
             B.quantize_qk_fp8(pq, qq, kk, q8, k8, qs, ks)
             B.block_select(p, s, q8, k8, row_ptr, col_idx, ws, qs, ks)
         else:
@@ -258,6 +276,8 @@ def main():
             B.block_select(p, s, qq, kk, row_ptr, col_idx, ws)
 
     def attend(qq, kk, vv, oo):
+        if args.prologue:
+            qq, kk = qn, kn
         if w.fp8:       # (the two-step form takes bf16 Q/K only: the one call transposes V itself)
             B.block_sparse_attn_fwd(p, q8, k8, vv, row_ptr, col_idx, oo, None, status, qs, ks, workspace=aws)
         elif two_step:
@@ -369,7 +389,7 @@ def main():
         "vs_baseline": None, "dtype": "e4m3 QK^T, bf16 PV" if w.fp8 else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
                    "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
-                   "nnz_tiles": nnz, "parallelism": f"replicas x{world}",
+                   "nnz_tiles": nnz, "parallelism": f"replicas x{world}", "prologue": bool(args.prologue),
                    "l2": "inputs (%.0f MB) larger than L2; no flush" % (3 * sel_bytes / 2 / 1e6)},
         "tokens_per_s": world * w.B * w.N / (ms_per_step * 1e-3),
         "attention_ms": attn_ms, "select_ms": sel_ms,
@@ -387,7 +407,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not args.prologue:   # (the oracle leg times the plain step)
             import oracle
             oracle.build()
             line["cpu_baseline"] = cpu_baseline(w, bf16_bits(qh), bf16_bits(kh), bf16_bits(vh))

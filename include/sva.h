@@ -106,6 +106,36 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                      size_t workspace_bytes, void* stream);
 
 /*
+ * The same routing from block means the caller already holds (sva_qk_norm_rope_pool writes them): the
+ * pooling pass over Q and K is skipped, everything else is sva_block_select.
+ *   q_mean, k_mean : [B,H,Nb,d] fp32 contiguous, 16-byte aligned; the mean over the valid tokens of each block
+ * workspace as for sva_block_select (the part that held the means stays unused).
+ */
+int sva_block_select_pooled(const sva_problem_t* p, const sva_select_t* s, const float* q_mean, const float* k_mean,
+                            int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/*
+ * Attention prologue in one pass over Q and K (the paper lists the fused QK-norm + RoPE among the
+ * lossless fusion flags of its deployments), per token n and head, in fp32:
+ *   RMS norm over the head dimension :  u_c = x_c / sqrt(mean_c(x_c^2) + eps) * g_c      (g_q for Q, g_k for K)
+ *   rotary embedding, adjacent pairs :  y_2i   = u_2i * cos[n,i] - u_2i+1 * sin[n,i]
+ *                                        y_2i+1 = u_2i+1 * cos[n,i] + u_2i * sin[n,i]
+ * y is rounded to bf16 and written to q_out / k_out (strides of p; may be q / k themselves).  From the
+ * rounded values, in the same pass:
+ *   q_mean, k_mean (optional, both or neither): block means for sva_block_select_pooled;
+ *   q8, k8, q_scale, k_scale (optional, all or none): what sva_quantize_qk_fp8 would produce from q_out, k_out.
+ * g_q, g_k: [d] fp32; cos_table, sin_table: [N, d/2] fp32 (shared by all heads and batch items; any
+ * position-to-angle rule, e.g. a 3-D one for video, is the caller's); all 16-byte aligned.  Token rows >= N
+ * are neither read nor written.  p->qk_dtype is ignored (the inputs are bf16).
+ * Errors: INVALID_ARG (null, eps < 0, half-given optional group), ALIGNMENT, UNSUPPORTED.
+ */
+int sva_qk_norm_rope_pool(const sva_problem_t* p, const void* q, const void* k, const float* g_q, const float* g_k,
+                          const float* cos_table, const float* sin_table, float eps, void* q_out, void* k_out,
+                          float* q_mean, float* k_mean, void* q8, void* k8, float* q_scale, float* k_scale,
+                          void* stream);
+
+/*
  * Routing for callers that cannot allocate device memory.  (The paper has no counterpart;
  * this is a packaging variant of sva_block_select, same kernels, same results.)
  *

@@ -23,7 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
-    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k",
+    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -89,6 +89,11 @@ def lib():
         L.sva_smooth_workspace_bytes.argtypes = [C.POINTER(Problem)]
         L.sva_quantize_qk_fp8_smooth_k.restype = C.c_int
         L.sva_quantize_qk_fp8_smooth_k.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_block_select_pooled.restype = C.c_int
+        L.sva_block_select_pooled.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_qk_norm_rope_pool.restype = C.c_int
+        L.sva_qk_norm_rope_pool.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp, vp, vp,
+                                            vp, vp, vp]
         L.sva_status_string.restype = C.c_char_p
         L.sva_status_string.argtypes = [C.c_int]
         _lib = L
@@ -245,3 +250,19 @@ def quantize_qk_fp8_smooth_k(p: Problem, q, k, q8, k8, q_scale, k_scale, k_mean,
                                             C.c_size_t(workspace.numel() if workspace is not None else 0), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_quantize_qk_fp8_smooth_k")
+
+
+def block_select_pooled(p: Problem, s: Select, q_mean, k_mean, row_ptr, col_idx, workspace, block_scores=None) -> None:
+    rc = lib().sva_block_select_pooled(C.byref(p), C.byref(s), _ptr(q_mean), _ptr(k_mean), _ptr(row_ptr), _ptr(col_idx),
+                                       _ptr(block_scores), _ptr(workspace), C.c_size_t(workspace.numel()), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_select_pooled")
+
+
+def qk_norm_rope_pool(p: Problem, q, k, g_q, g_k, cos_table, sin_table, eps, q_out, k_out, q_mean=None, k_mean=None,
+                      q8=None, k8=None, q_scale=None, k_scale=None) -> None:
+    rc = lib().sva_qk_norm_rope_pool(C.byref(p), _ptr(q), _ptr(k), _ptr(g_q), _ptr(g_k), _ptr(cos_table),
+                                     _ptr(sin_table), C.c_float(eps), _ptr(q_out), _ptr(k_out), _ptr(q_mean),
+                                     _ptr(k_mean), _ptr(q8), _ptr(k8), _ptr(q_scale), _ptr(k_scale), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_qk_norm_rope_pool")

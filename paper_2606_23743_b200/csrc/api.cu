@@ -95,6 +95,42 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                        workspace_bytes, (cudaStream_t)stream);
 }
 
+int sva_block_select_pooled(const sva_problem_t* p, const sva_select_t* s, const float* q_mean, const float* k_mean,
+                            int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  Dims m = make_dims(p);
+  if ((rc = validate_select(m, s))) return rc;
+  if (!q_mean || !k_mean || !row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q_mean) || !aligned16(k_mean)) return SVA_ERR_ALIGNMENT;
+  if (!workspace) return SVA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SVA_ERR_ALIGNMENT;
+  return launch_select_pooled(m, p, s, q_mean, k_mean, row_ptr, col_idx, block_scores, workspace, workspace_bytes,
+                              (cudaStream_t)stream);
+}
+
+int sva_qk_norm_rope_pool(const sva_problem_t* p, const void* q, const void* k, const float* g_q, const float* g_k,
+                          const float* cos_table, const float* sin_table, float eps, void* q_out, void* k_out,
+                          float* q_mean, float* k_mean, void* q8, void* k8, float* q_scale, float* k_scale,
+                          void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q || !k || !g_q || !g_k || !cos_table || !sin_table || !q_out || !k_out) return SVA_ERR_INVALID_ARG;
+  if (!(eps >= 0.f)) return SVA_ERR_INVALID_ARG;
+  if ((q_mean == nullptr) != (k_mean == nullptr)) return SVA_ERR_INVALID_ARG;
+  const int n8 = (q8 != nullptr) + (k8 != nullptr) + (q_scale != nullptr) + (k_scale != nullptr);
+  if (n8 != 0 && n8 != 4) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(q_out) || !aligned16(k_out) || !aligned16(g_q) || !aligned16(g_k) ||
+      !aligned16(cos_table) || !aligned16(sin_table) || (q8 && (!aligned16(q8) || !aligned16(k8))))
+    return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, q8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->k_stride, q8 ? 16 : 8))) return rc;
+  Dims m = make_dims(p);
+  return launch_prologue(m, p, q, k, g_q, g_k, cos_table, sin_table, eps, q_out, k_out, q_mean, k_mean, q8, k8,
+                         q_scale, k_scale, (cudaStream_t)stream);
+}
+
 /* Same routing, scratch taken from the library's built-in device array: no allocation. */
 int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, const void* q,
                              const void* k, const float* q_scale, const float* k_scale,

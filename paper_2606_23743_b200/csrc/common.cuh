@@ -37,6 +37,25 @@ __device__ __forceinline__ float e4m3_to_float(uint32_t byte) {
   return __half2float(__half(h));
 }
 
+// x / s for the e4m3 cast, s and y = RN(1/s) fixed for a whole block: q0 = x*y, one exact residual, one
+// correction -- the correctly rounded quotient (Markstein's sequence) in three FMA-pipe operations instead of
+// the dozen of a general division, valid while s is in [2^-60, 2^60] and its significand is not all ones
+// (div_fast_ok; otherwise the caller divides).  |x| below s*2^-12 may come out one unit off, which the cast
+// sends to zero all the same.  The residual is formed negated, t = q0*s - x, so that a zero x keeps its
+// sign through both steps (-0 stays -0, as in a true division).
+__device__ __forceinline__ bool div_fast_ok(float s) {
+  return s >= 8.673617379884035e-19f && s <= 1.152921504606847e18f && (__float_as_uint(s) & 0x7fffffu) != 0x7fffffu;
+}
+__device__ __forceinline__ float div_fast(float x, float s, float y) {
+  const float q0 = x * y;
+  const float t = fmaf(q0, s, -x);
+  return fmaf(-t, y, q0);
+}
+// two fp32 -> two e4m3 bytes (round to nearest even, saturating), first value in the low byte
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+}
+
 // host-side argument checks shared by the entry points
 int validate_problem(const sva_problem_t* p);
 
@@ -46,6 +65,12 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
                   int32_t* col_idx, float* block_scores, void* ws, size_t ws_bytes,
                   cudaStream_t st);
 size_t select_workspace_bytes(const Dims& m, const sva_select_t* s);
+int launch_select_pooled(const Dims& m, const sva_problem_t* p, const sva_select_t* s, const float* qbar,
+                         const float* kbar, int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* ws,
+                         size_t ws_bytes, cudaStream_t st);
+int launch_prologue(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const float* gq,
+                    const float* gk, const float* cosn, const float* sinn, float eps, void* qo, void* ko,
+                    float* qbar, float* kbar, void* q8, void* k8, float* qs, float* ks, cudaStream_t st);
 int launch_select_noalloc(const Dims& m, const sva_problem_t* p, const sva_select_t* s,
                           const void* q, const void* k, const float* q_scale, const float* k_scale,
                           int32_t* row_ptr, int32_t* col_idx, float* block_scores, cudaStream_t st);
@@ -63,7 +88,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st);
 size_t attn_ts_workspace_bytes(const Dims& m);
-bool attn_ts_serves(const Dims& m);    // d = 128: bf16 with 128- or 64-token blocks, e4m3 Q/K with 128-token blocks
+bool attn_ts_serves(const Dims& m);    // d = 128 (bf16 or e4m3 Q/K, 128- or 64-token blocks)
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
                         cudaStream_t st);
 

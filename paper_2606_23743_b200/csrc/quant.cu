@@ -4,6 +4,8 @@
 // With K smoothing, two small kernels first reduce K to its mean key per (b, h) -- per-block sums
 // in a fixed order, then the blocks in index order, so the mean is reproducible -- and the
 // quantiser subtracts it from K in fp32 and writes scale * <q_i, mean> per query token.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace sva {
@@ -46,7 +48,8 @@ __global__ void mean_key_kernel(const float* __restrict__ part, float* __restric
   mean[(long long)bh * D + c] = __fdiv_rn(t, (float)N);
 }
 
-template <int D, int MAX_ROWS>
+// SMOOTH: the K smoothing variant (k_mean given).
+template <int D, int MAX_ROWS, bool SMOOTH>
 __global__ void __launch_bounds__(QT)
 quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, Strides sq, Strides sk,
                 uint8_t* __restrict__ q8, uint8_t* __restrict__ k8, float* __restrict__ q_scale,
@@ -56,7 +59,8 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
   constexpr int GROUPS = QT / VPR;
   constexpr int PER = MAX_ROWS / GROUPS; // rows per thread
   __shared__ float red[QT / 32];
-  __shared__ float s_scale;
+  __shared__ float s_scale, s_rcp;
+  __shared__ int s_fast;
 
   const int I = blockIdx.x, bh = blockIdx.y, which = blockIdx.z;
   const int b = bh / H, h = bh % H;
@@ -71,12 +75,13 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
   float a = 0.f;
   // K smoothing: this thread's 8 components of the head's mean key (K: subtracted; Q: dotted)
   float mk[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  if (k_mean) {
+  if (SMOOTH) {
     const float4* mp = reinterpret_cast<const float4*>(k_mean + (long long)bh * D + vec * 8);
     const float4 m0 = __ldg(mp), m1 = __ldg(mp + 1);
     mk[0] = m0.x; mk[1] = m0.y; mk[2] = m0.z; mk[3] = m0.w; mk[4] = m1.x; mk[5] = m1.y; mk[6] = m1.z; mk[7] = m1.w;
   }
-  const bool sub = k_mean != nullptr && which == 1;
+  const bool sub = SMOOTH && which == 1;
+  __nv_bfloat162 am2 = __floats2bfloat162_rn(0.f, 0.f);
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     int t = grp + j * GROUPS;
@@ -90,10 +95,11 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
           a = fmaxf(a, fmaxf(fabsf(__fsub_rn(bf16lo(w[e]), mk[2 * e])), fabsf(__fsub_rn(bf16hi(w[e]), mk[2 * e + 1]))));
       }
     } else {
+      // |.| and max on the packed pairs; folded into `a` after the loop
 #pragma unroll
-      for (int e = 0; e < 4; ++e) a = fmaxf(a, fmaxf(fabsf(bf16lo(w[e])), fabsf(bf16hi(w[e]))));
+      for (int e = 0; e < 4; ++e) am2 = __hmax2(am2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[e])));
     }
-    if (k_mean && which == 0 && lse_shift) {
+    if (SMOOTH && which == 0 && lse_shift) {
       // scale * <q_t, mean>: 8 products here, the rest of the row in the other VPR-1 lanes of the group
       float dot = 0.f;
 #pragma unroll
@@ -103,6 +109,7 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
       if (vec == 0 && t < cnt) lse_shift[(long long)bh * N + lo + t] = dot * scale;
     }
   }
+  a = fmaxf(a, fmaxf(__low2float(am2), __high2float(am2)));
 #pragma unroll
   for (int o = 16; o; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
@@ -112,26 +119,33 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
     for (int i = 0; i < QT / 32; ++i) m = fmaxf(m, red[i]);
     float sc = m == 0.f ? 1.0f : __fdiv_rn(m, 448.0f);
     s_scale = sc;
+    s_rcp = __frcp_rn(sc);
+    s_fast = div_fast_ok(sc) ? 1 : 0;
     (which ? k_scale : q_scale)[(long long)bh * Nb + I] = sc;
   }
   __syncthreads();
-  const float sc = s_scale;
+  const float sc = s_scale, rcp = s_rcp;
+  // (one loop per division method, chosen per block, so that the common case carries no trace of the other)
+  auto cast_rows = [&](auto fast_tag) {
+    constexpr bool FAST = decltype(fast_tag)::value;
 #pragma unroll
-  for (int j = 0; j < PER; ++j) {
-    int t = grp + j * GROUPS;
-    if (t >= cnt) continue;
-    const uint32_t w[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
-    uint32_t out[2] = {0, 0};
+    for (int j = 0; j < PER; ++j) {
+      int t = grp + j * GROUPS;
+      if (t >= cnt) continue;
+      const uint32_t w[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
+      uint32_t c[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float x0 = sub ? __fsub_rn(bf16lo(w[e]), mk[2 * e]) : bf16lo(w[e]);
-      const float x1 = sub ? __fsub_rn(bf16hi(w[e]), mk[2 * e + 1]) : bf16hi(w[e]);
-      uint32_t c0 = __nv_cvt_float_to_fp8(__fdiv_rn(x0, sc), __NV_SATFINITE, __NV_E4M3);
-      uint32_t c1 = __nv_cvt_float_to_fp8(__fdiv_rn(x1, sc), __NV_SATFINITE, __NV_E4M3);
-      out[e >> 1] |= (c0 | (c1 << 8)) << (16 * (e & 1));
+      for (int e = 0; e < 4; ++e) {
+        const float x0 = sub ? __fsub_rn(bf16lo(w[e]), mk[2 * e]) : bf16lo(w[e]);
+        const float x1 = sub ? __fsub_rn(bf16hi(w[e]), mk[2 * e + 1]) : bf16hi(w[e]);
+        c[e] = FAST ? e4m3x2(div_fast(x0, sc, rcp), div_fast(x1, sc, rcp))
+                    : e4m3x2(__fdiv_rn(x0, sc), __fdiv_rn(x1, sc));
+      }
+      *reinterpret_cast<uint2*>(dst + (long long)(lo + t) * s.n + vec * 8) =
+          make_uint2(__byte_perm(c[0], c[1], 0x5410), __byte_perm(c[2], c[3], 0x5410));
     }
-    *reinterpret_cast<uint2*>(dst + (long long)(lo + t) * s.n + vec * 8) = make_uint2(out[0], out[1]);
-  }
+  };
+  if (s_fast) cast_rows(std::true_type{}); else cast_rows(std::false_type{});
 }
 
 size_t smooth_workspace_bytes(const Dims& m) { return (size_t)m.B * m.H * m.Nb * m.d * sizeof(float); }
@@ -153,12 +167,12 @@ int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const 
     mean_key_kernel<<<m.B * m.H, m.d, 0, st>>>((const float*)ws, k_mean, m.Nb, m.d, m.N);
     if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
   }
-  if (m.d == 128)
-    quantize_kernel<128, 128><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8,
-                                                (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb, k_mean, lse_shift, m.scale);
-  else
-    quantize_kernel<64, 128><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8,
-                                               (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb, k_mean, lse_shift, m.scale);
+#define SVA_QUANT_LAUNCH(DD, SM)                                                                            \
+  quantize_kernel<DD, 128, SM><<<g, QT, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, (uint8_t*)q8, \
+                                                 (uint8_t*)k8, qs, ks, m.H, m.N, m.block, m.Nb, k_mean, lse_shift, m.scale)
+  if (m.d == 128) { if (k_mean) SVA_QUANT_LAUNCH(128, true); else SVA_QUANT_LAUNCH(128, false); }
+  else { if (k_mean) SVA_QUANT_LAUNCH(64, true); else SVA_QUANT_LAUNCH(64, false); }
+#undef SVA_QUANT_LAUNCH
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 

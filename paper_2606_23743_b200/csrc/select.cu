@@ -427,11 +427,13 @@ template <int D>
 static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_select_t* s,
                            const void* q, const void* k, const float* q_scale,
                            const float* k_scale, int32_t* row_ptr, int32_t* col_idx,
-                           float* block_scores, void* ws, cudaStream_t st) {
+                           float* block_scores, void* ws, cudaStream_t st,
+                           const float* qbar_in = nullptr, const float* kbar_in = nullptr) {
   size_t pooled = align256((size_t)m.B * m.H * m.Nb * m.d * sizeof(float));
   char* w = static_cast<char*>(ws);
-  float* qbar = reinterpret_cast<float*>(w);
-  float* kbar = reinterpret_cast<float*>(w + pooled);
+  // (block means supplied by the caller -- the fused prologue writes them -- are used where they are)
+  float* qbar = qbar_in ? const_cast<float*>(qbar_in) : reinterpret_cast<float*>(w);
+  float* kbar = kbar_in ? const_cast<float*>(kbar_in) : reinterpret_cast<float*>(w + pooled);
   const int cap = select_row_cap(m, s);
   const int fixed_n = fixed_count(m, s);
   int32_t* tmp_idx = nullptr;
@@ -442,7 +444,8 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   }
   dim3 pg(m.Nb, m.B * m.H, 2);
   Strides sq = make_strides(p->q_stride), sk = make_strides(p->k_stride);
-  if (m.fp8)
+  if (qbar_in) {
+  } else if (m.fp8)
     pool_kernel<D, 1><<<pg, POOL_THREADS, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, q_scale,
                                                    k_scale, m.H, m.N, m.block, m.Nb, qbar, kbar);
   else
@@ -481,6 +484,19 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
     return launch_select_d<128>(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, ws, st);
   if (m.d == 64)
     return launch_select_d<64>(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, ws, st);
+  return SVA_ERR_UNSUPPORTED;
+}
+
+// Routing from block means the caller already has (qbar, kbar: [B,H,Nb,d] fp32).
+int launch_select_pooled(const Dims& m, const sva_problem_t* p, const sva_select_t* s, const float* qbar,
+                         const float* kbar, int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* ws,
+                         size_t ws_bytes, cudaStream_t st) {
+  if (ws_bytes < select_workspace_bytes(m, s)) return SVA_ERR_WORKSPACE;
+  if (m.Nb > 1024) return SVA_ERR_UNSUPPORTED;
+  if (m.d == 128)
+    return launch_select_d<128>(m, p, s, nullptr, nullptr, nullptr, nullptr, row_ptr, col_idx, block_scores, ws, st, qbar, kbar);
+  if (m.d == 64)
+    return launch_select_d<64>(m, p, s, nullptr, nullptr, nullptr, nullptr, row_ptr, col_idx, block_scores, ws, st, qbar, kbar);
   return SVA_ERR_UNSUPPORTED;
 }
 

@@ -122,3 +122,24 @@ def bf16_bits(x: torch.Tensor):
     """bf16 CPU tensor -> numpy uint16 view of the same bits."""
     import numpy as np
     return x.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def make_prologue_inputs(w: Workload, seed: int | None = None):
+    """Inputs of the QK-norm + RoPE prologue for a workload's token grid: norm weights g_q, g_k [d] near 1,
+    and rotary tables cos, sin [N, d/2] fp32 for a video's (frame, row, column) position -- the d/2
+    frequencies split evenly over the three axes, angle = position * 10000^(-i / n) within an axis."""
+    import math
+    g = torch.Generator(device="cpu")
+    g.manual_seed((SEED_BASE + w.cfg if seed is None else seed) + 7919)
+    gq = 1.0 + 0.1 * torch.randn(w.d, generator=g, dtype=torch.float32)
+    gk = 1.0 + 0.1 * torch.randn(w.d, generator=g, dtype=torch.float32)
+    tok = torch.arange(w.N)
+    pos = (tok // (w.Hg * w.Wg), (tok // w.Wg) % w.Hg, tok % w.Wg)
+    half = w.d // 2
+    bounds = [0, half // 3, 2 * (half // 3), half]
+    ang = torch.zeros(w.N, half, dtype=torch.float64)
+    for a in range(3):
+        n = bounds[a + 1] - bounds[a]
+        freq = torch.tensor([math.pow(10000.0, -i / n) for i in range(n)], dtype=torch.float64)
+        ang[:, bounds[a]:bounds[a + 1]] = pos[a].double()[:, None] * freq[None, :]
+    return gq, gk, torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()

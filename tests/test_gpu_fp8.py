@@ -152,3 +152,39 @@ def test_smoothed_fp8_attention_is_closer_to_bf16_attention():
     print(f"to bf16 attention: rel-L2 plain fp8 {e_plain:.3e}, smoothed {e_smooth:.3e}; "
           f"max lse error plain {l_plain:.3e}, smoothed {l_smooth:.3e}")
     assert e_smooth < e_plain and l_smooth < l_plain
+
+
+def test_quantiser_every_bf16_value_under_many_scales():
+    """The cast divides by the block scale with a short exact-division sequence: every finite bf16 value
+    (both zeros, subnormals) not above the block's absmax, under absmax values spread over the exponent
+    range (among them significands of all ones and the extremes that take the general division), bit for
+    bit against the oracle."""
+    pat = np.arange(1 << 16, dtype=np.uint32).astype(np.uint16)
+    val = torch.from_numpy(pat.view(np.int16)).view(torch.bfloat16).float().numpy()
+    fin = np.isfinite(val)
+    rng = np.random.default_rng(5)
+    amax_bits = [0x3F80, 0x3FFF, 0x7F7F, 0x0080, 0x0001, 0x5F7F, 0x1F01] + \
+                [int(e) << 7 | int(m) for e, m in zip(rng.integers(60, 200, 9), rng.integers(0, 128, 9))]
+    blocks = []
+    for ab in amax_bits:
+        a = val[ab]
+        mine = pat[fin & (np.abs(val) <= a)]
+        for lo in range(0, mine.size, 16383):
+            blk = np.zeros(16384, np.uint16)
+            chunk = mine[lo:lo + 16383]
+            blk[:chunk.size] = chunk
+            blk[-1] = ab                                              # the block's absmax is always present
+            blocks.append(blk.reshape(128, 128))
+    x = np.stack(blocks).reshape(1, 1, -1, 128)
+    N = x.shape[2]
+    xt = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).cuda()
+    w = shrink(WORKLOADS["large_fp8"], H=1, T=1)
+    q8 = torch.zeros(xt.shape, dtype=torch.uint8, device="cuda"); k8 = torch.zeros_like(q8)
+    qs = torch.zeros(1, 1, N // 128, dtype=torch.float32, device="cuda"); ks = torch.zeros_like(qs)
+    p = B.make_problem(xt, xt, None, None, N, 128)
+    B.quantize_qk_fp8(p, xt, xt, q8, k8, qs, ks)
+    torch.cuda.synchronize()
+    codes, scales = oracle.quantize_e4m3(x, N, 128)
+    np.testing.assert_array_equal(qs.cpu().numpy(), scales)
+    np.testing.assert_array_equal(q8.cpu().numpy(), codes)
+    np.testing.assert_array_equal(k8.cpu().numpy(), codes)
