@@ -42,9 +42,17 @@ block_sum_kernel(const uint8_t* __restrict__ k, Strides sk, float* __restrict__ 
 // mean[bh*D + c] = (sum over blocks, in index order) / N                        (grid BH, D threads)
 __global__ void mean_key_kernel(const float* __restrict__ part, float* __restrict__ mean, int Nb, int D, int N) {
   const int bh = blockIdx.x, c = threadIdx.x;
+  const float* src = part + (long long)bh * Nb * D + c;
   float t = 0.f;
-#pragma unroll 8
-  for (int I = 0; I < Nb; ++I) t += __ldg(part + ((long long)bh * Nb + I) * D + c);   // (loads run ahead; the order of the sum is fixed)
+  int I = 0;
+  for (; I + 16 <= Nb; I += 16) {          // 16 loads in flight; the order of the sum stays the index order
+    float v[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) v[e] = __ldg(src + (long long)(I + e) * D);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) t += v[e];
+  }
+  for (; I < Nb; ++I) t += __ldg(src + (long long)I * D);
   mean[(long long)bh * D + c] = __fdiv_rn(t, (float)N);
 }
 
@@ -83,10 +91,14 @@ quantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, St
   const bool sub = SMOOTH && which == 1;
   __nv_bfloat162 am2 = __floats2bfloat162_rn(0.f, 0.f);
 #pragma unroll
-  for (int j = 0; j < PER; ++j) {
+  for (int j = 0; j < PER; ++j) {          // all loads first: nothing below stands between them
     int t = grp + j * GROUPS;
     u[j] = make_uint4(0, 0, 0, 0);
     if (t < cnt) u[j] = __ldg(reinterpret_cast<const uint4*>(src + (long long)(lo + t) * s.n * 2) + vec);
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    int t = grp + j * GROUPS;
     const uint32_t w[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
     if (sub) {
       if (t < cnt) {

@@ -114,6 +114,22 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert lib.sva_quantize_qk_fp8(C.byref(p), one, one, one, None, one, one, None) == 1
     bad = _problem(); bad.k_stride = (C.c_int64 * 3)(0, 0, 136)
     assert lib.sva_quantize_qk_fp8(C.byref(bad), one, one, one, one, one, one, None) == 5
+    # the fused prologue: optional outputs come in whole groups
+    pro = lambda pp, q=one, g=one, qo=one, qm=one, km=one, q8=None, k8=None, qs=None, ks=None, eps=1e-6: \
+        lib.sva_qk_norm_rope_pool(C.byref(pp), q, one, g, one, one, one, C.c_float(eps), qo, one, qm, km, q8, k8, qs, ks, None)
+    assert pro(p, q=None) == 1 and pro(p, g=None) == 1 and pro(p, qo=None) == 1
+    assert pro(p, eps=-1.0) == 1
+    assert pro(p, km=None) == 1                                           # one mean without the other
+    assert pro(p, q8=one) == 1 and pro(p, q8=one, k8=one, qs=one) == 1    # codes without all of their scales
+    assert pro(p, q=vp(264)) == 5
+    assert pro(bad, q8=one, k8=one, qs=one, ks=one) == 5                  # stride 136 is fine for bf16, not for the codes
+    # routing from given means
+    selp = lambda pp, ss, qm=one, km=one, rp=one, ci=one, ws=one, wsb=1 << 30: \
+        lib.sva_block_select_pooled(C.byref(pp), C.byref(ss), qm, km, rp, ci, None, ws, C.c_size_t(wsb), None)
+    assert selp(p, s, qm=None) == 1 and selp(p, s, ci=None) == 1
+    assert selp(p, s, ws=None) == 3 and selp(p, s, wsb=16) == 3
+    assert selp(p, s, qm=vp(260)) == 5
+    assert selp(p, B.make_select(0, 0)) == 1
     # the smoothing quantiser: k_mean and its workspace are required, the lse shift is optional
     sm = lambda pp, mean=one, ws=one, nb=1 << 30: lib.sva_quantize_qk_fp8_smooth_k(
         C.byref(pp), one, one, one, one, one, one, mean, None, ws, C.c_size_t(nb), None)
