@@ -145,7 +145,7 @@ int sva_qk_norm_rope_pool(const sva_problem_t* p, const void* q, const void* k, 
  * a caller has nowhere to get the `workspace` that sva_block_select asks for.
  *
  * Here the scratch lives inside the library: a file-scope device array of
- * SVA_NOALLOC_SCRATCH_BYTES (8 MiB), present on every GPU that loads the library for as long
+ * SVA_NOALLOC_SCRATCH_BYTES (16 MiB), present on every GPU that loads the library for as long
  * as the process lives.  The call allocates and frees nothing.  Arguments and results are
  * those of sva_block_select minus workspace/workspace_bytes.
  *   - Limit: sva_select_workspace_bytes(p, s) must be <= SVA_NOALLOC_SCRATCH_BYTES, otherwise
@@ -158,7 +158,7 @@ int sva_qk_norm_rope_pool(const sva_problem_t* p, const void* q, const void* k, 
  *     Two calls that may overlap on the GPU (different streams, no dependency) race on it:
  *     serialise them.
  */
-#define SVA_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define SVA_NOALLOC_SCRATCH_BYTES (16u << 20)
 int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, const void* q,
                              const void* k, const float* q_scale, const float* k_scale,
                              int32_t* row_ptr, int32_t* col_idx, float* block_scores,

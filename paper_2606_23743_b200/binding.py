@@ -25,7 +25,7 @@ EXPORTS = [
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
     "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool",
 ]
-NOALLOC_SCRATCH_BYTES = 8 << 20
+NOALLOC_SCRATCH_BYTES = 16 << 20
 
 
 class Problem(C.Structure):

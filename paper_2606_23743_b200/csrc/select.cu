@@ -77,8 +77,6 @@ pool_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k, Stride
   }
 }
 
-static constexpr int SEL_ROWS = 16;     // query-block rows per CTA
-static constexpr int SEL_CHUNK = 32;    // key blocks staged per pass
 
 struct SelParams {
   int H, Nb, mode, k, use_window, win_t, win_s, bpf, cap, fixed_n;
@@ -115,32 +113,38 @@ __device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const in
   // keeps is "every candidate above a threshold key plus the first few of the candidates equal to it",
   // so the threshold is found by a 32-step bisection on the key bits (each step: one compare per
   // register, a warp reduction of the count and, in mode 1, of the mass) instead of up to k rounds of
-  // arg-max.  Decisions agree with the round-by-round form except where the mass comes within fp32
-  // summation noise of tau.
+  // arg-max.  The masses are summed in fixed point (weights in units of 2^-31: a warp-wide integer add is
+  // one instruction where a float sum is five shuffle rounds, and the result does not depend on the order),
+  // so decisions agree with the round-by-round form except where the mass comes within about 1e-7 --
+  // fp32 summation noise -- of tau.
   uint32_t mask = 0;            // bit it set <=> block it*32+lane is kept
   int n = 0;
-  float cum = 0.f, mx = 0.f, inv_z = 0.f;
-  float wgt[ITEMS];             // mode 1: softmax weight of every candidate
+  uint32_t cum = 0u;            // kept mass so far, units of 2^-31
+  const uint32_t tau_q = __float2uint_rn(fminf(fmaxf(p.tau, 0.f), 1.f) * 2147483648.f);
+  float mx = 0.f, inv_z = 0.f;
+  uint32_t wgt[ITEMS];          // mode 1: softmax weight of every candidate, units of 2^-31
 #pragma unroll
-  for (int it = 0; it < ITEMS; ++it) wgt[it] = 0.f;
+  for (int it = 0; it < ITEMS; ++it) wgt[it] = 0u;
   if (p.mode == 1) {
     uint32_t km = 0u;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) km = max(km, key[it]);
     km = __reduce_max_sync(0xffffffffu, km);
     mx = key_score(km);
-    float z = 0.f;
+    float z = 0.f, ew[ITEMS];
 #pragma unroll
-    for (int it = 0; it < ITEMS; ++it)
-      if (key[it]) { wgt[it] = expf(key_score(key[it]) - mx); z += wgt[it]; }
+    for (int it = 0; it < ITEMS; ++it) {
+      ew[it] = 0.f;
+      if (key[it]) { ew[it] = expf(key_score(key[it]) - mx); z += ew[it]; }
+    }
 #pragma unroll
     for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
     inv_z = 1.0f / z;
 #pragma unroll
-    for (int it = 0; it < ITEMS; ++it) wgt[it] *= inv_z;
+    for (int it = 0; it < ITEMS; ++it) wgt[it] = __float2uint_rn(ew[it] * inv_z * 2147483648.f);
   }
   if (p.use_window) {
-    float fm = 0.f;
+    uint32_t fm = 0u;
     int cnt = 0;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
@@ -149,22 +153,18 @@ __device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const in
         mask |= 1u << it; ++cnt;
         fm += wgt[it];
         key[it] = 0u;                        // no longer a candidate
-        wgt[it] = 0.f;
+        wgt[it] = 0u;
       }
     }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-      cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-      fm += __shfl_xor_sync(0xffffffffu, fm, o);
-    }
-    n = cnt; cum = fm;
+    n = (int)__reduce_add_sync(0xffffffffu, (unsigned)cnt);
+    cum = __reduce_add_sync(0xffffffffu, fm);
   }
   const int kk = min(p.k, Nb);
-  if (n < kk && !(p.mode == 1 && n >= 1 && cum >= p.tau)) {
+  if (n < kk && !(p.mode == 1 && n >= 1 && cum >= tau_q)) {
     // count and mass of the candidates with key >= t
-    auto above = [&](uint32_t t, int& cnt, float& mass) {
+    auto above = [&](uint32_t t, int& cnt, uint32_t& mass) {
       int c = 0;
-      float g = 0.f;
+      uint32_t g = 0u;
 #pragma unroll
       for (int it = 0; it < ITEMS; ++it) {
         const bool ge = key[it] >= t && key[it] != 0u;
@@ -172,11 +172,7 @@ __device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const in
         if (ge) g += wgt[it];
       }
       cnt = (int)__reduce_add_sync(0xffffffffu, (unsigned)c);
-      if (p.mode == 1) {
-#pragma unroll
-        for (int o = 16; o; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-      }
-      mass = g;
+      mass = p.mode == 1 ? __reduce_add_sync(0xffffffffu, g) : 0u;
     };
     // largest threshold at which taking every candidate >= it ends the rule (0: never -> take them all)
     uint32_t T = 0u;
@@ -184,26 +180,30 @@ __device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const in
     for (int bit = 31; bit >= 0; --bit) {
       const uint32_t t = T | (1u << bit);
       int c;
-      float g;
+      uint32_t g;
       above(t, c, g);
-      if (n + c >= kk || (p.mode == 1 && c >= 1 && cum + g >= p.tau)) T = t;
+      if (n + c >= kk || (p.mode == 1 && c >= 1 && cum + g >= tau_q)) T = t;
     }
     // everything above T, then ties at T in index order while the rule still runs
     int G;
-    float Mg;
+    uint32_t Mg;
     above(T + 1u, G, Mg);                    // T = 0: all candidates; T = 0xffffffff cannot be reached (see below)
     int have = n + G;
-    float acc = cum + Mg;
-    const float wT = (p.mode == 1 && T != 0u) ? expf(key_score(T) - mx) * inv_z : 0.f;
+    uint32_t acc = cum + Mg;
     int ties_wanted = 0;
     if (T != 0u) {
       int E = 0;
+      uint32_t wT = 0u;                      // weight of a candidate equal to T (they all have the same)
 #pragma unroll
-      for (int it = 0; it < ITEMS; ++it) E += (key[it] == T);
+      for (int it = 0; it < ITEMS; ++it) {
+        E += (key[it] == T);
+        if (key[it] == T) wT = wgt[it];
+      }
       E = (int)__reduce_add_sync(0xffffffffu, (unsigned)E);
+      wT = __reduce_max_sync(0xffffffffu, wT);
       while (ties_wanted < E) {
         if (have >= kk) break;
-        if (p.mode == 1 && have >= 1 && acc >= p.tau) break;
+        if (p.mode == 1 && have >= 1 && acc >= tau_q) break;
         ++ties_wanted; ++have; acc += wT;
       }
     }
@@ -245,103 +245,89 @@ __device__ __forceinline__ void select_and_emit(uint32_t (&key)[ITEMS], const in
   }
 }
 
-// One CTA scores and selects SEL_ROWS query-block rows of one head.  A warp takes RW rows: lane j
-// owns the key blocks J = it*32 + j and accumulates the RW rows' scores of a key together, so every
-// pooled-key value read from shared memory feeds RW FMAs (the kernel is bound by shared-memory
-// reads otherwise).  A chunk of 32 pooled keys is staged transposed in shared memory (lane j reads
-// key j conflict-free, the query values are 128-bit broadcasts), double-buffered: the next chunk's
-// global loads are in flight while the current one is used.  Afterwards the warp runs the selection
-// of its rows one after the other.
-// smem: qs[SEL_ROWS][D] | ksT[2][D][33]
-template <int D, int ITEMS, int RW>
-__global__ void __launch_bounds__(SEL_ROWS / RW * 32)
-score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, SelParams p,
-                    int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx,
-                    int32_t* __restrict__ tmp_idx, int32_t* __restrict__ counts,
-                    float* __restrict__ block_scores, int R) {
-  constexpr int NW = SEL_ROWS / RW;            // warps per CTA
-  constexpr int KT_LD = SEL_CHUNK + 1;
-  constexpr int PRE = D / 4 / NW;              // float4 loads per thread and chunk
-  __shared__ __align__(16) float qs[SEL_ROWS * D];
-  __shared__ float ksT[2][D * KT_LD];
-  const int Nb = p.Nb;
-  const int bh = blockIdx.y;
-  const int I0 = blockIdx.x * SEL_ROWS;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  for (int i = threadIdx.x; i < SEL_ROWS * D; i += blockDim.x) {
-    int w = i / D;
-    qs[i] = (I0 + w < Nb) ? qbar[((long long)bh * Nb + I0 + w) * D + (i % D)] : 0.f;
-  }
+// Block scores of one head as a small fp32 GEMM: S[I][J] = scale * <qbar_I, kbar_J>.  A CTA computes a
+// 64 x 64 tile from the two 64 x D panels in shared memory (row stride D + 4 floats: 128-bit reads of
+// eight consecutive rows touch every bank once); a thread owns a 4 x 4 patch -- rows 4*ty..4*ty+3 (one
+// address per half-warp: a broadcast), keys tx, tx+16, tx+32, tx+48 -- and keeps two partial sums per
+// entry (dimensions 0,2 mod 4 and 1,3 mod 4, each in ascending order; that order is part of the
+// result: it is what makes the scores reproducible bit for bit).  32 independent FMA chains per thread
+// hide the shared-memory latency that bounded the earlier one-warp-per-row form.
+static constexpr int SC_TILE = 64;
+template <int D>
+__global__ void __launch_bounds__(256)
+block_scores_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, int Nb, float scale,
+                    float* __restrict__ scores) {
+  constexpr int LD = D + 4;
+  extern __shared__ __align__(16) float sc_smem[];
+  float* qs = sc_smem;                     // [64][LD]
+  float* ks = sc_smem + SC_TILE * LD;      // [64][LD]
+  const int bh = blockIdx.z, I0 = blockIdx.y * SC_TILE, J0 = blockIdx.x * SC_TILE;
+  const float* qb = qbar + (long long)bh * Nb * D;
   const float* kb = kbar + (long long)bh * Nb * D;
-
-  float4 pre[PRE];
-  auto load_chunk = [&](int it) {
-    const int J = it * 32 + lane;
-#pragma unroll
-    for (int i = 0; i < PRE; ++i) {
-      pre[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (J < Nb) pre[i] = __ldg(reinterpret_cast<const float4*>(kb + (long long)J * D) + warp + NW * i);
-    }
-  };
-  auto store_chunk = [&](int buf) {
-#pragma unroll
-    for (int i = 0; i < PRE; ++i) {
-      const int cc = warp + NW * i;
-      ksT[buf][(4 * cc + 0) * KT_LD + lane] = pre[i].x;
-      ksT[buf][(4 * cc + 1) * KT_LD + lane] = pre[i].y;
-      ksT[buf][(4 * cc + 2) * KT_LD + lane] = pre[i].z;
-      ksT[buf][(4 * cc + 3) * KT_LD + lane] = pre[i].w;
-    }
-  };
-
-  uint32_t key[RW][ITEMS];
-  load_chunk(0);
-  store_chunk(0);
+  for (int idx = threadIdx.x; idx < SC_TILE * (D / 4); idx += 256) {
+    const int row = idx / (D / 4), c4 = idx % (D / 4);
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (I0 + row < Nb) a = __ldg(reinterpret_cast<const float4*>(qb + (long long)(I0 + row) * D) + c4);
+    if (J0 + row < Nb) b = __ldg(reinterpret_cast<const float4*>(kb + (long long)(J0 + row) * D) + c4);
+    *reinterpret_cast<float4*>(qs + row * LD + 4 * c4) = a;
+    *reinterpret_cast<float4*>(ks + row * LD + 4 * c4) = b;
+  }
   __syncthreads();
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  float a0[4][4], a1[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { a0[i][j] = 0.f; a1[i][j] = 0.f; }
+#pragma unroll 2
+  for (int c = 0; c < D; c += 4) {
+    float4 qv[4], kv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) qv[i] = *reinterpret_cast<const float4*>(qs + (ty * 4 + i) * LD + c);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) kv[j] = *reinterpret_cast<const float4*>(ks + (tx + 16 * j) * LD + c);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        a0[i][j] = fmaf(qv[i].x, kv[j].x, a0[i][j]);
+        a1[i][j] = fmaf(qv[i].y, kv[j].y, a1[i][j]);
+        a0[i][j] = fmaf(qv[i].z, kv[j].z, a0[i][j]);
+        a1[i][j] = fmaf(qv[i].w, kv[j].w, a1[i][j]);
+      }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int I = I0 + ty * 4 + i;
+    if (I >= Nb) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int J = J0 + tx + 16 * j;
+      if (J < Nb) scores[((long long)bh * Nb + I) * Nb + J] = (a0[i][j] + a1[i][j]) * scale;
+    }
+  }
+}
+
+// Selection: one warp per query-block row, its Nb scores read straight from the score matrix (lane j owns
+// the key blocks it*32 + j).  No shared memory and few registers, so the SMs hold enough warps to hide the
+// serial chain of the threshold search.
+static constexpr int SEL_WARPS = 8;
+template <int ITEMS>
+__global__ void __launch_bounds__(SEL_WARPS * 32)
+select_rows_kernel(const float* __restrict__ scores, SelParams p, int32_t* __restrict__ row_ptr,
+                   int32_t* __restrict__ col_idx, int32_t* __restrict__ tmp_idx, int32_t* __restrict__ counts, int R) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * SEL_WARPS + (threadIdx.x >> 5);
+  if (r >= R) return;
+  const int Nb = p.Nb, bh = r / Nb, I = r % Nb;
+  const float* srow = scores + (long long)r * Nb;
+  uint32_t key[ITEMS];
 #pragma unroll
   for (int it = 0; it < ITEMS; ++it) {
-#pragma unroll
-    for (int r = 0; r < RW; ++r) key[r][it] = 0u;
-    if (it * 32 < Nb) {                      // uniform over the CTA
-      const bool more = it + 1 < ITEMS && (it + 1) * 32 < Nb;
-      if (more) load_chunk(it + 1);          // in flight during the FMAs below
-      const float* kt = ksT[it & 1];
-      float a0[RW], a1[RW];
-#pragma unroll
-      for (int r = 0; r < RW; ++r) { a0[r] = 0.f; a1[r] = 0.f; }
-#pragma unroll 4
-      for (int c = 0; c < D; c += 4) {
-        const float k0 = kt[(c + 0) * KT_LD + lane], k1 = kt[(c + 1) * KT_LD + lane];
-        const float k2 = kt[(c + 2) * KT_LD + lane], k3 = kt[(c + 3) * KT_LD + lane];
-#pragma unroll
-        for (int r = 0; r < RW; ++r) {
-          const float4 qv = *reinterpret_cast<const float4*>(qs + (warp * RW + r) * D + c);
-          a0[r] = fmaf(qv.x, k0, a0[r]);
-          a1[r] = fmaf(qv.y, k1, a1[r]);
-          a0[r] = fmaf(qv.z, k2, a0[r]);
-          a1[r] = fmaf(qv.w, k3, a1[r]);
-        }
-      }
-      const int J = it * 32 + lane;
-      if (J < Nb) {
-#pragma unroll
-        for (int r = 0; r < RW; ++r) {
-          const float v = (a0[r] + a1[r]) * p.scale;
-          key[r][it] = score_key(v);
-          const int I = I0 + warp * RW + r;
-          if (block_scores && I < Nb) block_scores[((long long)bh * Nb + I) * Nb + J] = v;
-        }
-      }
-      if (more) store_chunk((it + 1) & 1);
-      __syncthreads();
-    }
+    const int J = it * 32 + lane;
+    key[it] = J < Nb ? score_key(__ldg(srow + J)) : 0u;
   }
-#pragma unroll
-  for (int r = 0; r < RW; ++r) {
-    const int I = I0 + warp * RW + r;
-    if (I < Nb) select_and_emit<ITEMS>(key[r], I, bh, lane, p, row_ptr, col_idx, tmp_idx, counts, R);
-  }
+  select_and_emit<ITEMS>(key, I, bh, lane, p, row_ptr, col_idx, tmp_idx, counts, R);
 }
 
 // Exclusive scan of counts[R] -> row_ptr[R+1]; one CTA, chunks of 1024 with a running carry.
@@ -420,6 +406,7 @@ size_t select_workspace_bytes(const Dims& m, const sva_select_t* s) {
     bytes += align256((size_t)m.R * select_row_cap(m, s) * sizeof(int32_t));
     bytes += align256((size_t)m.R * sizeof(int32_t));
   }
+  bytes += align256((size_t)m.R * m.Nb * sizeof(float));      // the score matrix (unused when the caller asks for it)
   return bytes;
 }
 
@@ -456,16 +443,29 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   sp.use_window = (s->win_t >= 0 && s->win_s >= 0 && s->blocks_per_frame > 0) ? 1 : 0;
   sp.win_t = s->win_t; sp.win_s = s->win_s; sp.bpf = sp.use_window ? s->blocks_per_frame : 1;
   sp.cap = cap; sp.fixed_n = fixed_n; sp.scale = m.scale; sp.tau = s->mass;
+  // scores: into the caller's matrix if it wants one, else into the workspace (after the staging arrays)
+  float* scores = block_scores;
+  if (!scores) {
+    size_t off = 2 * pooled;
+    if (!fixed_n) off += align256((size_t)m.R * cap * sizeof(int32_t)) + align256((size_t)m.R * sizeof(int32_t));
+    scores = reinterpret_cast<float*>(w + off);
+  }
+  {
+    auto kern = block_scores_kernel<D>;
+    constexpr int smem = 2 * SC_TILE * (D + 4) * (int)sizeof(float);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SVA_ERR_CUDA;
+    const int nt = (m.Nb + SC_TILE - 1) / SC_TILE;
+    kern<<<dim3(nt, nt, m.B * m.H), 256, smem, st>>>(qbar, kbar, m.Nb, m.scale, scores);
+  }
   const int items = (m.Nb + 31) / 32;
-  dim3 sg((m.Nb + SEL_ROWS - 1) / SEL_ROWS, m.B * m.H);
-#define SVA_SEL_LAUNCH(IT, RWV)                                                                     \
-  score_select_kernel<D, IT, RWV><<<sg, SEL_ROWS / RWV * 32, 0, st>>>(qbar, kbar, sp, row_ptr, col_idx, \
-                                                                       tmp_idx, counts, block_scores, m.R)
-  if (items <= 4) SVA_SEL_LAUNCH(4, 2);
-  else if (items <= 8) SVA_SEL_LAUNCH(8, 2);
-  else if (items <= 12) SVA_SEL_LAUNCH(12, 2);
-  else if (items <= 16) SVA_SEL_LAUNCH(16, 2);
-  else SVA_SEL_LAUNCH(32, 2);
+  const int sg = (m.R + SEL_WARPS - 1) / SEL_WARPS;
+#define SVA_SEL_LAUNCH(IT) \
+  select_rows_kernel<IT><<<sg, SEL_WARPS * 32, 0, st>>>(scores, sp, row_ptr, col_idx, tmp_idx, counts, m.R)
+  if (items <= 4) SVA_SEL_LAUNCH(4);
+  else if (items <= 8) SVA_SEL_LAUNCH(8);
+  else if (items <= 12) SVA_SEL_LAUNCH(12);
+  else if (items <= 16) SVA_SEL_LAUNCH(16);
+  else SVA_SEL_LAUNCH(32);
 #undef SVA_SEL_LAUNCH
   if (!fixed_n) {
     scan_kernel<<<1, 1024, 0, st>>>(counts, m.R, row_ptr);
@@ -479,7 +479,7 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
                   int32_t* col_idx, float* block_scores, void* ws, size_t ws_bytes,
                   cudaStream_t st) {
   if (ws_bytes < select_workspace_bytes(m, s)) return SVA_ERR_WORKSPACE;
-  if (m.Nb > 1024) return SVA_ERR_UNSUPPORTED;    // score rows live in shared memory, kept flags in one word per lane
+  if (m.Nb > 1024) return SVA_ERR_UNSUPPORTED;    // a lane holds at most 32 scores of a row, kept flags in one word per lane
   if (m.d == 128)
     return launch_select_d<128>(m, p, s, q, k, q_scale, k_scale, row_ptr, col_idx, block_scores, ws, st);
   if (m.d == 64)

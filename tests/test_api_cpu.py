@@ -51,9 +51,10 @@ def test_workspace_and_capacity(lib):
     Nb, R = 8, 16
     assert B.select_max_nnz(p, s) == R * 4
     pooled = 2 * (2 * Nb * 128 * 4)
-    assert B.select_workspace_bytes(p, s) == pooled                      # fixed-count rows: no staging
+    scores = R * Nb * 4                                                   # the score matrix
+    assert B.select_workspace_bytes(p, s) == pooled + scores             # fixed-count rows: no staging
     sm = B.make_select(1, 4, 0.9)
-    assert B.select_workspace_bytes(p, sm) >= pooled + R * 4 * 4 + R * 4  # staged rows + counts
+    assert B.select_workspace_bytes(p, sm) >= pooled + scores + R * 4 * 4 + R * 4  # staged rows + counts
     sw = B.make_select(0, 4, 1.0, 1, 1, 4)                                # 3x3 window > k
     assert B.select_max_nnz(p, sw) == R * 8                               # window clipped to Nb = 8
     assert B.select_max_nnz(p, B.make_select(0, 100)) == R * Nb          # k above Nb means Nb
