@@ -64,6 +64,11 @@ def test_full_size_fp8():
     p = B.make_problem(qd, kd, None, None, w.N, w.block)
     B.quantize_qk_fp8(p, qd, kd, q8, k8, qs, ks)
     torch.cuda.synchronize()
+    # the quantiser at full size, bit for bit
+    for bits, g8, gs in ((qb, q8, qs), (kb, k8, ks)):
+        codes, scales = oracle.quantize_e4m3(bits, w.N, w.block)
+        np.testing.assert_array_equal(gs.cpu().numpy(), scales)
+        assert np.array_equal(g8.cpu().numpy()[:, :, :w.N], codes[:, :, :w.N])
     qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
     kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
     rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
@@ -75,3 +80,43 @@ def test_full_size_fp8():
     rows = U.sample_rows(w.R, w.Nb, 12, seed=5)
     r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
     print(f"large_fp8: differing {n_diff} near {n_near} max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}")
+
+
+def test_full_size_prologue():
+    """The fused QK-norm + RoPE prologue in the launch configuration `bench.py --prologue` times
+    (cfg 5 shape: bf16 write-back, block means and e4m3 codes in one launch): three sampled heads against
+    the oracle, then routing from its means against routing that pools the written Q, K itself."""
+    from paper_2606_23743_b200 import binding as B
+    from paper_2606_23743_b200.workloads import bf16_bits, make_prologue_inputs
+    w = WORKLOADS["large_fp8"]
+    (q, k, _), (qb, kb, _) = U.host_inputs(w)
+    qd, kd = U.dev(q), U.dev(k)
+    gq, gk, cos, sin = make_prologue_inputs(w)
+    qo, ko = torch.full_like(qd, 7.0), torch.full_like(kd, 7.0)
+    qm = torch.zeros(w.B, w.H, w.Nb, w.d, dtype=torch.float32, device="cuda"); km = torch.zeros_like(qm)
+    q8 = torch.zeros(qd.shape, dtype=torch.uint8, device="cuda"); k8 = torch.zeros_like(q8)
+    qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device="cuda"); ks = torch.zeros_like(qs)
+    p = B.make_problem(qd, kd, None, None, w.N, w.block)
+    B.qk_norm_rope_pool(p, qd, kd, gq.cuda(), gk.cuda(), cos.cuda(), sin.cuda(), 1e-6, qo, ko, qm, km, q8, k8, qs, ks)
+    torch.cuda.synchronize()
+    for h in (0, 11, w.H - 1):
+        for bits, g, out, mean, c8, sc in ((qb, gq, qo, qm, q8, qs), (kb, gk, ko, km, k8, ks)):
+            ref = oracle.qk_norm_rope(bits[:, h:h + 1], g.numpy(), cos.numpy(), sin.numpy(), w.N, 1e-6)[:, :, :w.N]
+            got = out[:, h:h + 1, :w.N].float().cpu().numpy().astype(np.float64)
+            assert (np.abs(got - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-5).all()
+            assert (got == torch.from_numpy(ref).to(torch.bfloat16).float().numpy()).mean() > 0.999
+            ob = bf16_bits(out[:, h:h + 1].cpu())
+            np.testing.assert_allclose(mean[:, h:h + 1].cpu().numpy(), oracle.pool(ob, w.N, w.block), rtol=2e-6, atol=2e-7)
+            codes, scales = oracle.quantize_e4m3(ob, w.N, w.block)
+            np.testing.assert_array_equal(sc[:, h:h + 1].cpu().numpy(), scales)
+            assert np.array_equal(c8[:, h:h + 1, :w.N].cpu().numpy(), codes[:, :, :w.N])
+    assert (qo[:, :, w.N:] == 7.0).all() and (ko[:, :, w.N:] == 7.0).all()
+    s = B.make_select(w.mode, w.k, w.tau)
+    pb = B.make_problem(qo, ko, None, None, w.N, w.block)
+    rp = torch.zeros(w.R + 1, dtype=torch.int32, device="cuda")
+    ci = torch.zeros(B.select_max_nnz(pb, s), dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.select_workspace_bytes(pb, s), dtype=torch.uint8, device="cuda")
+    B.block_select_pooled(pb, s, qm, km, rp, ci, ws)
+    torch.cuda.synchronize()
+    rp2, ci2, _ = U.gpu_select(w, qo, ko)          # (bf16 routing: gpu_select takes the dtype from its fp8 argument)
+    assert torch.equal(rp, rp2) and torch.equal(ci[: int(rp[-1])], ci2)
