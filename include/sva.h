@@ -106,7 +106,16 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                      size_t workspace_bytes, void* stream);
 
 /*
- * The same routing from block means the caller already holds (sva_qk_norm_rope_pool writes them): the
+ * The pooling step of the routing alone: q_mean, k_mean ([B,H,Nb,d] fp32 contiguous, 16-byte aligned) =
+ * the mean over the valid tokens of each block of Q and K as described by p (e4m3 codes are multiplied
+ * by their block scale).  Together with sva_block_select_pooled it is sva_block_select in two calls,
+ * for callers that want the HBM-bound pooling pass and the latency-bound rest on streams of their own.
+ */
+int sva_pool_qk(const sva_problem_t* p, const void* q, const void* k, const float* q_scale, const float* k_scale,
+                float* q_mean, float* k_mean, void* stream);
+
+/*
+ * The same routing from block means the caller already holds (sva_pool_qk or sva_qk_norm_rope_pool writes them): the
  * pooling pass over Q and K is skipped, everything else is sva_block_select.
  *   q_mean, k_mean : [B,H,Nb,d] fp32 contiguous, 16-byte aligned; the mean over the valid tokens of each block
  * workspace as for sva_block_select (the part that held the means stays unused).

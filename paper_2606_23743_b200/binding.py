@@ -23,7 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
-    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool",
+    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -89,6 +89,8 @@ def lib():
         L.sva_smooth_workspace_bytes.argtypes = [C.POINTER(Problem)]
         L.sva_quantize_qk_fp8_smooth_k.restype = C.c_int
         L.sva_quantize_qk_fp8_smooth_k.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_pool_qk.restype = C.c_int
+        L.sva_pool_qk.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
         L.sva_block_select_pooled.restype = C.c_int
         L.sva_block_select_pooled.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.sva_qk_norm_rope_pool.restype = C.c_int
@@ -266,3 +268,10 @@ def qk_norm_rope_pool(p: Problem, q, k, g_q, g_k, cos_table, sin_table, eps, q_o
                                      _ptr(k_mean), _ptr(q8), _ptr(k8), _ptr(q_scale), _ptr(k_scale), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_qk_norm_rope_pool")
+
+
+def pool_qk(p: Problem, q, k, q_mean, k_mean, q_scale=None, k_scale=None) -> None:
+    rc = lib().sva_pool_qk(C.byref(p), _ptr(q), _ptr(k), _ptr(q_scale), _ptr(k_scale), _ptr(q_mean), _ptr(k_mean),
+                           _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_pool_qk")

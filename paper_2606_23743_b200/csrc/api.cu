@@ -95,6 +95,19 @@ int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* 
                        workspace_bytes, (cudaStream_t)stream);
 }
 
+int sva_pool_qk(const sva_problem_t* p, const void* q, const void* k, const float* q_scale, const float* k_scale,
+                float* q_mean, float* k_mean, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  Dims m = make_dims(p);
+  if (!q || !k || !q_mean || !k_mean) return SVA_ERR_INVALID_ARG;
+  if (m.fp8 && (!q_scale || !k_scale)) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(q_mean) || !aligned16(k_mean)) return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, m.fp8 ? 16 : 8))) return rc;
+  if ((rc = check_strides(p->k_stride, m.fp8 ? 16 : 8))) return rc;
+  return launch_pool(m, p, q, k, q_scale, k_scale, q_mean, k_mean, (cudaStream_t)stream);
+}
+
 int sva_block_select_pooled(const sva_problem_t* p, const sva_select_t* s, const float* q_mean, const float* k_mean,
                             int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* workspace,
                             size_t workspace_bytes, void* stream) {

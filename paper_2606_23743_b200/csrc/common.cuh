@@ -65,6 +65,8 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
                   int32_t* col_idx, float* block_scores, void* ws, size_t ws_bytes,
                   cudaStream_t st);
 size_t select_workspace_bytes(const Dims& m, const sva_select_t* s);
+int launch_pool(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const float* q_scale,
+                const float* k_scale, float* qbar, float* kbar, cudaStream_t st);
 int launch_select_pooled(const Dims& m, const sva_problem_t* p, const sva_select_t* s, const float* qbar,
                          const float* kbar, int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* ws,
                          size_t ws_bytes, cudaStream_t st);

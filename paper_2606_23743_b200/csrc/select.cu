@@ -487,6 +487,27 @@ int launch_select(const Dims& m, const sva_problem_t* p, const sva_select_t* s, 
   return SVA_ERR_UNSUPPORTED;
 }
 
+// Pooling alone: block means of Q and K into the caller's arrays ([B,H,Nb,d] fp32 each).
+int launch_pool(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const float* q_scale,
+                const float* k_scale, float* qbar, float* kbar, cudaStream_t st) {
+  dim3 pg(m.Nb, m.B * m.H, 2);
+  Strides sq = make_strides(p->q_stride), sk = make_strides(p->k_stride);
+#define SVA_POOL_LAUNCH(DD)                                                                                        \
+  do {                                                                                                             \
+    if (m.fp8)                                                                                                     \
+      pool_kernel<DD, 1><<<pg, POOL_THREADS, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, q_scale, k_scale, \
+                                                      m.H, m.N, m.block, m.Nb, qbar, kbar);                       \
+    else                                                                                                           \
+      pool_kernel<DD, 2><<<pg, POOL_THREADS, 0, st>>>((const uint8_t*)q, (const uint8_t*)k, sq, sk, nullptr, nullptr, \
+                                                      m.H, m.N, m.block, m.Nb, qbar, kbar);                       \
+  } while (0)
+  if (m.d == 128) SVA_POOL_LAUNCH(128);
+  else if (m.d == 64) SVA_POOL_LAUNCH(64);
+  else return SVA_ERR_UNSUPPORTED;
+#undef SVA_POOL_LAUNCH
+  return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
+}
+
 // Routing from block means the caller already has (qbar, kbar: [B,H,Nb,d] fp32).
 int launch_select_pooled(const Dims& m, const sva_problem_t* p, const sva_select_t* s, const float* qbar,
                          const float* kbar, int32_t* row_ptr, int32_t* col_idx, float* block_scores, void* ws,

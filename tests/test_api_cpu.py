@@ -124,6 +124,10 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert pro(p, q8=one) == 1 and pro(p, q8=one, k8=one, qs=one) == 1    # codes without all of their scales
     assert pro(p, q=vp(264)) == 5
     assert pro(bad, q8=one, k8=one, qs=one, ks=one) == 5                  # stride 136 is fine for bf16, not for the codes
+    # pooling alone
+    pool = lambda pp, q=one, qm=one: lib.sva_pool_qk(C.byref(pp), q, one, None, None, qm, one, None)
+    assert pool(p, q=None) == 1 and pool(p, qm=None) == 1 and pool(p, qm=vp(260)) == 5
+    assert pool(_problem(qk_dtype=1)) == 1                                # e4m3 codes without their scales
     # routing from given means
     selp = lambda pp, ss, qm=one, km=one, rp=one, ci=one, ws=one, wsb=1 << 30: \
         lib.sva_block_select_pooled(C.byref(pp), C.byref(ss), qm, km, rp, ci, None, ws, C.c_size_t(wsb), None)

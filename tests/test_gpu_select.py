@@ -82,3 +82,37 @@ def test_workspace_too_small_is_rejected():
     with pytest.raises(B.SvaError) as e:
         B.block_select(p, s, qd, kd, rp, ci, ws)
     assert e.value.status == 3
+
+
+@pytest.mark.parametrize("name", ["medium", "large_fp8"])
+def test_routing_in_two_calls_equals_the_one_call(name):
+    """sva_pool_qk + sva_block_select_pooled = sva_block_select (bf16 and e4m3 inputs); the means against
+    the oracle's pooling."""
+    import oracle
+    from paper_2606_23743_b200 import binding as B
+    from paper_2606_23743_b200.workloads import shrink
+    w = shrink(WORKLOADS[name], H=2, T=3)
+    (q, k, _), (qb, kb, _) = U.host_inputs(w)
+    qd, kd = U.dev(q), U.dev(k)
+    qs = ks = None
+    if w.fp8:
+        q8 = torch.zeros(qd.shape, dtype=torch.uint8, device="cuda"); k8 = torch.zeros_like(q8)
+        qs = torch.zeros(w.B, w.H, w.Nb, dtype=torch.float32, device="cuda"); ks = torch.zeros_like(qs)
+        B.quantize_qk_fp8(B.make_problem(qd, kd, None, None, w.N, w.block), qd, kd, q8, k8, qs, ks)
+        qd, kd = q8, k8
+    rp1, ci1, _ = U.gpu_select(w, qd, kd, q_scale=qs, k_scale=ks, fp8=w.fp8)
+    p = B.make_problem(qd, kd, None, None, w.N, w.block, 0.0, w.fp8)
+    s = B.make_select(w.mode, w.k, w.tau, w.win_t, w.win_s, w.blocks_per_frame if w.win_t >= 0 else 0)
+    qm = torch.full((w.B, w.H, w.Nb, w.d), 7.0, dtype=torch.float32, device="cuda"); km = torch.full_like(qm, 7.0)
+    B.pool_qk(p, qd, kd, qm, km, qs, ks)
+    rp2 = torch.zeros(w.R + 1, dtype=torch.int32, device="cuda")
+    ci2 = torch.zeros(B.select_max_nnz(p, s), dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.select_workspace_bytes(p, s), dtype=torch.uint8, device="cuda")
+    B.block_select_pooled(p, s, qm, km, rp2, ci2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(rp1, rp2) and torch.equal(ci1, ci2[: int(rp2[-1])])
+    if w.fp8:
+        qb = oracle.dequantize_e4m3(qd.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+        kb = oracle.dequantize_e4m3(kd.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    np.testing.assert_allclose(qm.cpu().numpy(), oracle.pool(qb, w.N, w.block), rtol=2e-6, atol=2e-7)
+    np.testing.assert_allclose(km.cpu().numpy(), oracle.pool(kb, w.N, w.block), rtol=2e-6, atol=2e-7)
