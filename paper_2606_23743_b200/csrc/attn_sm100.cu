@@ -63,6 +63,7 @@ struct TsParams {
   int32_t* status;
   Strides so;
   int H, N, Nb, R;            // Nb: key blocks per head; R: rows handed out (128-query tiles)
+  int d;                      // head dimension of the tensors: 128, or 64 (computed as 128 with the upper half zero)
   int Nt;                     // 128-query tiles per head (= Nb for 128-token blocks, ceil(Nb/2) for 64-token blocks)
   const int32_t* tile_cnt;    // 64-token blocks only: per tile row, number of 128-key tiles ...
   const int32_t* tile_beg;    // ... and where its descriptors start
@@ -247,7 +248,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (qi >= prm.N) break;
               __nv_bfloat16* orow = prm.o + (long long)(bh0 / prm.H) * prm.so.b + (long long)(bh0 % prm.H) * prm.so.h +
                                     (long long)qi * prm.so.n;
-              for (int cc = 0; cc < D; cc += 8) *reinterpret_cast<uint4*>(orow + cc) = make_uint4(0, 0, 0, 0);
+              for (int cc = 0; cc < prm.d; cc += 8) *reinterpret_cast<uint4*>(orow + cc) = make_uint4(0, 0, 0, 0);
               if (prm.lse) prm.lse[(long long)bh0 * prm.N + qi] = -INFINITY;
             }
           }
@@ -430,7 +431,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int e = 0; e < 32; ++e) qv[e] = 0u;
       if (r >= prm.R) return;
       const int bh = r / Nb, qi = (r % Nb) * BS + row;
-      if (qi >= prm.N) return;
+      if (qi >= prm.N || 64 * w >= prm.d) return;                      // (d = 64: the second group's half of Q is zero)
       const long long eoff = (long long)(bh / prm.H) * prm.sq.b + (long long)(bh % prm.H) * prm.sq.h +
                              (long long)qi * prm.sq.n + 64 * w;           // in elements
       const uint4* src = F8 ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(prm.q) + eoff)
@@ -671,7 +672,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         mbar_arrive(bar_ost + 8 * w);
         if ((threadIdx.x & 127) == 0) {
           // (a wait that runs out has raised the abort flag; the other threads leave at their next wait)
-          if (mbar_wait(bar_ost + 8 * w, rows_done & 1u, abort_flag, prm.status)) {
+          if (mbar_wait(bar_ost + 8 * w, rows_done & 1u, abort_flag, prm.status) && (D / 2) * w < prm.d) {
             tma_store_4d(&tm_o, sbase + OFF_O + w * (TILE / 2), (D / 2) * w, I * BS, hh, bb);
             bulk_commit();
           }
@@ -707,6 +708,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 __global__ void __launch_bounds__(256)
 transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat16* __restrict__ vt, int H, int N,
                    int Nb, int d, int kb, int32_t* __restrict__ row_counter) {
+  // d = 64: the tile still has 128 d-rows; the CTAs of the upper half (d0 >= d) write zeros
   // the attention kernel that follows draws its rows from this counter
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) {
     row_counter[0] = 0;     // next row to hand out
@@ -722,7 +724,7 @@ transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat1
     for (int pass = 0; pass < 2; ++pass) {
       const int key = (threadIdx.x >> 3) + 32 * pass;
       uint4 u = make_uint4(0, 0, 0, 0);
-      if (n0 + key < N) u = __ldg(reinterpret_cast<const uint4*>(src + (long long)(n0 + key) * sv.n + d0) + c8);
+      if (n0 + key < N && d0 < d) u = __ldg(reinterpret_cast<const uint4*>(src + (long long)(n0 + key) * sv.n + d0) + c8);
       const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&u);
 #pragma unroll
       for (int q = 0; q < 8; ++q) tile[c8 * 8 + q][key] = e[q];
@@ -738,7 +740,7 @@ transpose_v_kernel(const __nv_bfloat16* __restrict__ v, Strides sv, __nv_bfloat1
       __align__(16) __nv_bfloat16 e[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) e[q] = tile[dd][k8 * 8 + q];
-      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * d + d0 + dd) * kb + kin) = *reinterpret_cast<uint4*>(e);
+      *reinterpret_cast<uint4*>(vt + (((long long)bh * Nb + J) * ts::D + d0 + dd) * kb + kin) = *reinterpret_cast<uint4*>(e);
     }
   }
 }
@@ -875,7 +877,7 @@ struct TsLayout {
 };
 static TsLayout ts_layout(const Dims& m) {
   TsLayout L;
-  L.vt_bytes = (size_t)m.B * m.H * m.Nb * m.block * m.d * 2;
+  L.vt_bytes = (size_t)m.B * m.H * m.Nb * m.block * ts::D * 2;      // (d = 64: tiles are padded to 128 d-rows)
   L.counter_off = L.vt_bytes;
   L.Nt = m.block == 64 ? (m.Nb + 1) / 2 : m.Nb;
   L.R2 = m.B * m.H * L.Nt;
@@ -892,7 +894,7 @@ static TsLayout ts_layout(const Dims& m) {
 }
 
 bool attn_ts_serves(const Dims& m) {
-  return m.d == 128 && m.Nb <= 16383 && (m.block == BS || m.block == 64);
+  return (m.d == 128 || (m.d == 64 && !m.fp8)) && m.Nb <= 16383 && (m.block == BS || m.block == 64);
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {
@@ -921,7 +923,7 @@ int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, vo
   if (rc) return rc;
   const TsLayout L = ts_layout(m);
   const Strides sv = make_strides(p->v_stride);
-  dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+  dim3 tg((m.Nb * m.block + 63) / 64, ts::D / 64, m.B * m.H);    // every key slot of every tile, also those beyond N (zeros)
   transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
                                          reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + L.counter_off));
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
@@ -953,14 +955,14 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
                         m.block, eb)) != SVA_OK)
     return rc;
   // transposed V: per (b,h) a [Nb*128 rows][block keys] matrix, key block J = rows J*128 .. J*128+127
-  const cuuint64_t vrows = (cuuint64_t)m.Nb * m.d;
+  const cuuint64_t vrows = (cuuint64_t)m.Nb * ts::D;
   if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
                         vrows * m.block * 2 * m.H, BS)) != SVA_OK)
     return rc;
   if (v) {
     // (the transposed copy is laid out for the block size of this launch)
     const Strides sv = make_strides(p->v_stride);
-    dim3 tg((m.N + 63) / 64, m.d / 64, m.B * m.H);
+    dim3 tg((m.Nb * m.block + 63) / 64, ts::D / 64, m.B * m.H);    // every key slot of every tile, also those beyond N (zeros)
     transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
                                            reinterpret_cast<int32_t*>(wsb + L.counter_off));
     if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
@@ -973,7 +975,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   prm.row_ptr = row_ptr; prm.col_idx = col_idx;
   prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
   prm.so = make_strides(p->o_stride);
-  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.Nt = L.Nt; prm.R = L.R2;
+  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.Nt = L.Nt; prm.R = L.R2; prm.d = m.d;
   prm.tile_cnt = reinterpret_cast<const int32_t*>(wsb + L.cnt_off);
   prm.tile_beg = reinterpret_cast<const int32_t*>(wsb + L.beg_off);
   prm.tile_desc = reinterpret_cast<const uint32_t*>(wsb + L.desc_off);

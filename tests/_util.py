@@ -24,7 +24,7 @@ def gpu_select(w: Workload, q, k, N=None, want_scores=False, q_scale=None, k_sca
     s = B.make_select(w.mode, w.k, w.tau, w.win_t, w.win_s, w.blocks_per_frame if w.win_t >= 0 else 0)
     Nb = -(-N // w.block)
     R = q.shape[0] * q.shape[1] * Nb
-    ws = torch.empty(max(B.select_workspace_bytes(p, s), 256), dtype=torch.uint8, device="cuda")
+    ws = torch.full((max(B.select_workspace_bytes(p, s), 256),), 0xFF, dtype=torch.uint8, device="cuda")
     row_ptr = torch.full((R + 1,), -7, dtype=torch.int32, device="cuda")
     col_idx = torch.full((max(B.select_max_nnz(p, s), 1),), -7, dtype=torch.int32, device="cuda")
     scores = torch.empty(q.shape[0], q.shape[1], Nb, Nb, dtype=torch.float32, device="cuda") if want_scores else None
@@ -69,7 +69,8 @@ def gpu_attn(w: Workload, q, k, v, row_ptr, col_idx, N=None, simt=False, dense=F
     lse = torch.full((q.shape[0], q.shape[1], N), 7.0, dtype=torch.float32, device="cuda") if want_lse else None
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(q, k, v, o, N, w.block, 0.0, fp8)
-    ws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device="cuda")
+    # (0xff bytes are NaNs as bf16: whatever the kernels do not write themselves shows up in the output)
+    ws = torch.full((max(B.attn_workspace_bytes(p), 256),), 0xFF, dtype=torch.uint8, device="cuda")
     if dense and not simt:
         B.dense_attn_fwd(p, q, k, v, o, lse, status, q_scale, k_scale, workspace=ws)
     else:

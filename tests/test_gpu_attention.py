@@ -19,7 +19,7 @@ def _setup(w):
 
 
 CASES = {
-    "tiny_block64": (WORKLOADS["tiny"], None),                                   # CUDA-core kernel
+    "tiny_block64": (WORKLOADS["tiny"], None),                                   # d = 64: computed as d = 128 with a zero upper half
     "medium_h4": (shrink(WORKLOADS["medium"], H=4), 10),
     "ragged_tail": (shrink(WORKLOADS["medium"], H=3, T=2, Hg=30, Wg=31, k=5), None),
     "odd_nb": (shrink(WORKLOADS["medium"], H=2, T=1, Hg=30, Wg=30, k=4), None),  # Nb = 8 -> N=900: Nb=8
@@ -34,7 +34,10 @@ CASES = {
     "b64_mass_ragged_rows": (shrink(WORKLOADS["large_ragged"], H=2, T=8, block=64, k=60), 14),
     "b64_k1": (shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=1), 12),
     "b64_single_block": (shrink(WORKLOADS["medium"], H=1, T=1, Hg=5, Wg=8, block=64, k=1), None),   # N = 40 < block
-    "block128_d64": (shrink(WORKLOADS["tiny"], H=2, T=4, block=128, k=3), None),         # CUDA-core kernel
+    "block128_d64": (shrink(WORKLOADS["tiny"], H=2, T=4, block=128, k=3), None),
+    "d64_ragged_tail": (shrink(WORKLOADS["medium"], H=3, T=2, Hg=30, Wg=31, k=5, d=64), None),       # N = 1860, d = 64
+    "d64_mass_ragged_rows": (shrink(WORKLOADS["large_ragged"], H=2, T=8, d=64), 12),
+    "d64_b64_odd_nb": (shrink(WORKLOADS["medium"], H=2, T=1, Hg=30, Wg=30, block=64, k=4, d=64), None),
     "many_rows_few_blocks": (shrink(WORKLOADS["medium"], H=6, T=8, k=2), 12),            # R = 384 > 148 CTAs, 2 blocks per row
     "one_block_rows": (shrink(WORKLOADS["medium"], H=3, T=4, k=1), 10),                  # odd row length 1: only one group has work
 }
@@ -55,7 +58,7 @@ def test_sparse_attention_matches_oracle(name, impl):
         assert (o[:, :, w.N:] == 7.0).all()
 
 
-@pytest.mark.parametrize("name", ["ragged_tail", "medium_h4", "b64_ragged_tail", "b64_odd_nb"])
+@pytest.mark.parametrize("name", ["ragged_tail", "medium_h4", "b64_ragged_tail", "b64_odd_nb", "d64_ragged_tail", "d64_b64_odd_nb"])
 def test_dense_equals_keep_all_and_oracle(name):
     w, _ = CASES[name]
     data, bits, _, _ = _setup(w)
@@ -88,7 +91,7 @@ def test_repeatable_bytes():
         assert torch.equal(od, o2) and torch.equal(ld, l2)
 
 
-@pytest.mark.parametrize("name", ["mass_ragged_rows", "b64_mass_ragged_rows"])
+@pytest.mark.parametrize("name", ["mass_ragged_rows", "b64_mass_ragged_rows", "d64_mass_ragged_rows"])
 def test_two_step_form_matches_the_one_call_form(name):
     """V prepared on a second stream, then the attention kernel alone: same bytes as the one-call entry
     points (sparse and, for 128-token blocks, dense), and the workspace can be prepared again for the next call."""
@@ -99,7 +102,7 @@ def test_two_step_form_matches_the_one_call_form(name):
     o2 = torch.full_like(o1, 3.0); l2 = torch.full_like(l1, 3.0)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(qd, kd, vd, o2, w.N, w.block)
-    ws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    ws = torch.full((B.attn_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
     side = torch.cuda.Stream()
     for sparse in ((True, False, True) if w.block == 128 else (True, True)):
         ready = torch.cuda.Event()
@@ -212,7 +215,7 @@ def test_strided_qkv_and_output():
     o = o_buf.permute(0, 2, 1, 3)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(qv, kv, vv, o, w.N, w.block)
-    ws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    ws = torch.full((B.attn_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
     B.block_sparse_attn_fwd(p, qv, kv, vv, rp, ci, o, None, st, workspace=ws)
     torch.cuda.synchronize()
     assert int(st) == 0

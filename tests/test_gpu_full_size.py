@@ -39,7 +39,7 @@ def test_full_size_select_then_attend(name, nrows):
         o2 = torch.full_like(o, 7.0); lse2 = torch.full_like(lse, 7.0)
         st2 = torch.zeros(1, dtype=torch.int32, device="cuda")
         p = B.make_problem(qd, kd, vd, o2, w.N, w.block)
-        aws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        aws = torch.full((B.attn_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
         side, ready = torch.cuda.Stream(), torch.cuda.Event()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):

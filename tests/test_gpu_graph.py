@@ -29,7 +29,7 @@ def test_capture_and_replay(name):
         p = B.make_problem(qd, kd, vd, o, w.N, w.block)
     s = B.make_select(w.mode, w.k, w.tau)
     ws = torch.empty(B.select_workspace_bytes(p, s), dtype=torch.uint8, device="cuda")
-    aws = torch.empty(B.attn_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    aws = torch.full((B.attn_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
     rp = torch.zeros(w.R + 1, dtype=torch.int32, device="cuda")
     ci = torch.zeros(B.select_max_nnz(p, s), dtype=torch.int32, device="cuda")
     side = torch.cuda.Stream()
