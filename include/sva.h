@@ -180,13 +180,13 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * O is bf16.  A row with an empty list writes zeros and lse = -inf.
  * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
  * (16 for e4m3 Q/K).  Tensor-core kernels (bf16 or e4m3 x e4m3 MMA, fp32 accumulate) serve d = 128:
- * bf16 or e4m3 Q/K with 128- or 64-token blocks; bf16 with d = 64 runs on the same kernels (computed as
- * d = 128 with a zero upper half); e4m3 Q/K with d = 64 runs on a CUDA-core kernel.
+ * bf16 or e4m3 Q/K with 128- or 64-token blocks; d = 64 runs on the same kernels (computed as d = 128 with
+ * a zero upper half).
  * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The tensor-core kernel
  * keeps a tiled, transposed copy of V (2*B*H*Nb*block*128 bytes), its row counter and, for 64-token
  * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
  * GPU need a workspace each);
- * the size is 0 -- and the pointer may be NULL -- for shapes served by the CUDA-core kernel.
+ * 0 only for an unsupported problem.
  */
 size_t sva_attn_workspace_bytes(const sva_problem_t* p);
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,

@@ -55,8 +55,8 @@ static int validate_attn(const sva_problem_t* p, const void* q, const void* k, c
   return SVA_OK;
 }
 
-// The tensor-core kernel (attn_ts_serves: d = 128 with bf16 or e4m3 Q/K, d = 64 with bf16; 128- or 64-token
-// blocks; it needs the transposed-V workspace) or, for the other supported shapes, the CUDA-core kernel.
+// The tensor-core kernel (attn_ts_serves: every shape the library takes today; it needs the transposed-V
+// workspace); the CUDA-core kernel stays behind it for shapes it would not serve.
 
 }  // namespace sva
 

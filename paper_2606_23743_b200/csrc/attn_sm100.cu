@@ -894,7 +894,7 @@ static TsLayout ts_layout(const Dims& m) {
 }
 
 bool attn_ts_serves(const Dims& m) {
-  return (m.d == 128 || (m.d == 64 && !m.fp8)) && m.Nb <= 16383 && (m.block == BS || m.block == 64);
+  return (m.d == 128 || m.d == 64) && m.Nb <= 16383 && (m.block == BS || m.block == 64);
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {

@@ -90,7 +90,7 @@ int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const v
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st);
 size_t attn_ts_workspace_bytes(const Dims& m);
-bool attn_ts_serves(const Dims& m);    // d = 128 (bf16 or e4m3 Q/K) or d = 64 (bf16); 128- or 64-token blocks
+bool attn_ts_serves(const Dims& m);    // d = 128 or 64, bf16 or e4m3 Q/K, 128- or 64-token blocks
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
                         cudaStream_t st);
 

@@ -101,7 +101,7 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert prep(p, ws=vp(4096 + 16)) == 5
     assert prep(_problem(qk_dtype=1)) == 2                                # e4m3 Q/K: one-call entry points only
     assert prep(_problem(d=64), ws=None) == 3                             # d = 64 runs on the same kernel (padded to 128)
-    assert prep(_problem(d=64, qk_dtype=1)) == 2                          # d = 64 with e4m3 Q/K: CUDA-core kernel, one call
+    assert prep(_problem(d=64, qk_dtype=1)) == 2                          # e4m3 Q/K: one-call entry points only
     att2 = lambda pp, q=one, rp=one, ci=one, ws=None: lib.sva_block_sparse_attn_fwd_prepared(
         C.byref(pp), q, one, rp, ci, one, None, None, ws, 0, None)
     assert att2(p, q=None) == 1
@@ -109,7 +109,8 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert att2(p) == 3                                                   # no workspace
     assert att2(_problem(qk_dtype=1)) in (1, 2)
     assert B.attn_workspace_bytes(_problem(d=64)) == 1 * 2 * 8 * 128 * 128 * 2 + 256   # d = 64: V tiles padded to 128 d-rows
-    assert B.attn_workspace_bytes(_problem(d=64, qk_dtype=1)) == 0       # CUDA-core kernel needs none
+    assert B.attn_workspace_bytes(_problem(d=64, qk_dtype=1)) == 1 * 2 * 8 * 128 * 128 * 2 + 256
+    assert B.attn_workspace_bytes(_problem(d=96)) == 0                   # unsupported shape
     # 64-token blocks: transposed V, counter, tile lists (R2 = 16 tile rows, 16 key blocks, 32 CSR rows)
     assert B.attn_workspace_bytes(_problem(block=64)) == 2 * 1024 * 128 * 2 + 256 + 256 + 256 + ((((32 * 16 + 16) // 2 + 2) * 4 + 255) // 256) * 256
     assert B.attn_workspace_bytes(_problem(qk_dtype=1)) == 1 * 2 * 8 * 128 * 128 * 2 + 256   # e4m3 Q/K: V is still bf16

@@ -188,3 +188,21 @@ def test_quantiser_every_bf16_value_under_many_scales():
     np.testing.assert_array_equal(qs.cpu().numpy(), scales)
     np.testing.assert_array_equal(q8.cpu().numpy(), codes)
     np.testing.assert_array_equal(k8.cpu().numpy(), codes)
+
+
+@pytest.mark.parametrize("block", [128, 64])
+def test_fp8_d64(block):
+    """e4m3 Q/K with d = 64 (the tensor-core kernel computes it as d = 128 with a zero upper half)."""
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=3, d=64, block=block, mode=0, k=7)
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8, k8, qs, ks = _quantize(w, qd, kd)
+    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
+    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
+    o, lse, st = U.gpu_attn(w, q8, k8, vd, rp, ci, q_scale=qs, k_scale=ks, fp8=True)
+    assert st == 0
+    rows = U.sample_rows(w.R, w.Nb, 12)
+    r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
+    o2, lse2, st2 = U.gpu_attn(w, q8, k8, vd, rp, ci, simt=True, q_scale=qs, k_scale=ks, fp8=True)
+    print(f"fp8 d64 block {block}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}; vs simt max diff {(o.float() - o2.float()).abs().max().item():.2e}")
