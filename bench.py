@@ -256,8 +256,8 @@ def main():
             B.attn_prepare_v(p, vv, aws)
             v_ready.record()
 
-    # the two-step form serves what the bf16 tensor-core kernel serves; other shapes take the one call
-    two_step = (not w.fp8) and B.attn_workspace_bytes(p) > 0
+    # the two-step form serves what the tensor-core kernel serves (every supported shape today)
+    two_step = B.attn_workspace_bytes(p) > 0
 
     def route(qq, kk, vv):
         if args.prologue:
@@ -269,6 +269,8 @@ def main():
                 B.qk_norm_rope_pool(pq, qq, kk, gq, gk, cos_t, sin_t, 1e-6, qn, kn, qm, km)
             B.block_select_pooled(p, s, qm, km, row_ptr, col_idx, ws)
         elif w.fp8:
+            if two_step:
+                prepare_v(vv)
             B.quantize_qk_fp8(pq, qq, kk, q8, k8, qs, ks)
             B.block_select(p, s, q8, k8, row_ptr, col_idx, ws, qs, ks)
         else:
@@ -279,7 +281,11 @@ def main():
     def attend(qq, kk, vv, oo):
         if args.prologue:
             qq, kk = qn, kn
-        if w.fp8:       # (the two-step form takes bf16 Q/K only: the one call transposes V itself)
+        if w.fp8 and two_step:
+            torch.cuda.current_stream().wait_event(v_ready)
+            B.block_sparse_attn_fwd_prepared(p, q8, k8, row_ptr, col_idx, oo, None, status, workspace=aws,
+                                             q_scale=qs, k_scale=ks)
+        elif w.fp8:
             B.block_sparse_attn_fwd(p, q8, k8, vv, row_ptr, col_idx, oo, None, status, qs, ks, workspace=aws)
         elif two_step:
             torch.cuda.current_stream().wait_event(v_ready)
@@ -398,8 +404,8 @@ def main():
         "select_gbs": sel_bytes / (sel_ms * 1e-3) / 1e9,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
-                     "kernel": "attn_ts_kernel" + (" with the V transpose in front of it" if w.fp8 else
-                                                  " (the V transpose runs beside routing on a second stream)"),
+                     "kernel": "attn_ts_kernel" + (" (the V transpose runs beside routing on a second stream)" if two_step
+                                                  else " with the V transpose in front of it"),
                      "mixed_precision_ceiling": peak * 4.0 / 3.0 if w.fp8 else None,
                      "peak_source": f"{peak_kind} bf16 burst",
                      "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"])

@@ -200,7 +200,7 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * The bf16 tensor-core path in two steps (bf16 Q/K only), for callers that can prepare V early -- on another stream
+ * The tensor-core path in two steps, for callers that can prepare V early -- on another stream
  * while routing runs (routing never reads V), or because the producer of V can be made to write
  * the prepared layout itself.  sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
  * and key block one contiguous tile [d][block keys], keys >= N zero) and resets the row counter in
@@ -208,15 +208,16 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
  * NULL means dense).  A prepared workspace serves any number of attention calls on that V that do
  * not overlap on the GPU (after a call that reported SVA_DEV_TIMEOUT, prepare again); the caller
  * orders prepare and attention (same stream, or an event).  Together they do exactly what
- * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call.  SVA_ERR_UNSUPPORTED for problems
- * the bf16 tensor-core kernel does not serve (e4m3 Q/K, d other than 128) and for the dense form with
- * 64-token blocks: use the one-call entry points there.
+ * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call (q_scale, k_scale: as there, NULL for
+ * bf16 Q/K).  SVA_ERR_UNSUPPORTED for the dense form of bf16 Q/K with 64-token blocks (it runs as
+ * 128-token blocks, which a workspace prepared for 64-token blocks does not fit): use the one-call
+ * entry point there.
  */
 int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, size_t workspace_bytes,
                        void* stream);
-int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k,
-                                       const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
-                                       int32_t* device_status, void* workspace, size_t workspace_bytes,
+int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k, const float* q_scale,
+                                       const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o,
+                                       float* lse, int32_t* device_status, void* workspace, size_t workspace_bytes,
                                        void* stream);
 
 /*

@@ -78,7 +78,7 @@ def lib():
         L.sva_attn_prepare_v.restype = C.c_int
         L.sva_attn_prepare_v.argtypes = [C.POINTER(Problem), vp, vp, C.c_size_t, vp]
         L.sva_block_sparse_attn_fwd_prepared.restype = C.c_int
-        L.sva_block_sparse_attn_fwd_prepared.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_block_sparse_attn_fwd_prepared.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         for fn in (L.sva_gather_tokens, L.sva_scatter_tokens):
             fn.restype = C.c_int
             fn.argtypes = [vp, C.POINTER(C.c_int64), vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -206,11 +206,11 @@ def attn_prepare_v(p: Problem, v, workspace) -> None:
 
 
 def block_sparse_attn_fwd_prepared(p: Problem, q, k, row_ptr, col_idx, o, lse=None, status=None,
-                                   workspace=None) -> None:
+                                   workspace=None, q_scale=None, k_scale=None) -> None:
     """Second half: the attention kernel alone on a workspace that attn_prepare_v filled (row_ptr None = dense)."""
-    rc = lib().sva_block_sparse_attn_fwd_prepared(C.byref(p), _ptr(q), _ptr(k), _ptr(row_ptr), _ptr(col_idx),
-                                                  _ptr(o), _ptr(lse), _ptr(status), _ptr(workspace),
-                                                  _ws_bytes(workspace), _stream())
+    rc = lib().sva_block_sparse_attn_fwd_prepared(C.byref(p), _ptr(q), _ptr(k), _ptr(q_scale), _ptr(k_scale),
+                                                  _ptr(row_ptr), _ptr(col_idx), _ptr(o), _ptr(lse), _ptr(status),
+                                                  _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_fwd_prepared")
 

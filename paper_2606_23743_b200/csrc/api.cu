@@ -205,22 +205,22 @@ int sva_attn_prepare_v(const sva_problem_t* p, const void* v, void* workspace, s
   if ((rc = check_strides(p->v_stride, 8))) return rc;
   if (p->v_stride[2] < p->d) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!attn_ts_serves(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
   return launch_prepare_v_ts(m, p, v, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
-int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k,
-                                       const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
-                                       int32_t* device_status, void* workspace, size_t workspace_bytes,
+int sva_block_sparse_attn_fwd_prepared(const sva_problem_t* p, const void* q, const void* k, const float* q_scale,
+                                       const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o,
+                                       float* lse, int32_t* device_status, void* workspace, size_t workspace_bytes,
                                        void* stream) {
   // (q stands in for v in the shared checks: the prepared call takes no V pointer; the v strides of p are still checked)
-  int rc = validate_attn(p, q, k, q, nullptr, nullptr, o);
+  int rc = validate_attn(p, q, k, q, q_scale, k_scale, o);
   if (rc) return rc;
   if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!attn_ts_serves(m) || m.fp8) return SVA_ERR_UNSUPPORTED;
-  return launch_attn_ts(m, p, q, k, nullptr, nullptr, nullptr, row_ptr, col_idx, o, lse, device_status, workspace, workspace_bytes,
-                        (cudaStream_t)stream);
+  if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
+  return launch_attn_ts(m, p, q, k, nullptr, q_scale, k_scale, row_ptr, col_idx, o, lse, device_status, workspace,
+                        workspace_bytes, (cudaStream_t)stream);
 }
 
 int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const void* k,

@@ -99,15 +99,15 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert prep(p, ws=None) == 3
     assert prep(p, nb=16) == 3
     assert prep(p, ws=vp(4096 + 16)) == 5
-    assert prep(_problem(qk_dtype=1)) == 2                                # e4m3 Q/K: one-call entry points only
+    assert prep(_problem(d=96)) == 2
     assert prep(_problem(d=64), ws=None) == 3                             # d = 64 runs on the same kernel (padded to 128)
-    assert prep(_problem(d=64, qk_dtype=1)) == 2                          # e4m3 Q/K: one-call entry points only
-    att2 = lambda pp, q=one, rp=one, ci=one, ws=None: lib.sva_block_sparse_attn_fwd_prepared(
-        C.byref(pp), q, one, rp, ci, one, None, None, ws, 0, None)
+    att2 = lambda pp, q=one, rp=one, ci=one, ws=None, qs=None: lib.sva_block_sparse_attn_fwd_prepared(
+        C.byref(pp), q, one, qs, qs, rp, ci, one, None, None, ws, 0, None)
     assert att2(p, q=None) == 1
     assert att2(p, ci=None) == 1
     assert att2(p) == 3                                                   # no workspace
-    assert att2(_problem(qk_dtype=1)) in (1, 2)
+    assert att2(_problem(qk_dtype=1)) == 1                                # e4m3 Q/K without their scales
+    assert att2(_problem(qk_dtype=1), qs=one) == 3                        # ... with them: next complaint is the workspace
     assert B.attn_workspace_bytes(_problem(d=64)) == 1 * 2 * 8 * 128 * 128 * 2 + 256   # d = 64: V tiles padded to 128 d-rows
     assert B.attn_workspace_bytes(_problem(d=64, qk_dtype=1)) == 1 * 2 * 8 * 128 * 128 * 2 + 256
     assert B.attn_workspace_bytes(_problem(d=96)) == 0                   # unsupported shape

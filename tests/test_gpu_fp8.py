@@ -206,3 +206,23 @@ def test_fp8_d64(block):
     r = U.check_attn_vs_oracle(w, qh, kh, vb, rp, ci, o, lse, rows, rel_tol=U.FP8_REL_L2, abs_tol=5e-2)
     o2, lse2, st2 = U.gpu_attn(w, q8, k8, vd, rp, ci, simt=True, q_scale=qs, k_scale=ks, fp8=True)
     print(f"fp8 d64 block {block}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e}; vs simt max diff {(o.float() - o2.float()).abs().max().item():.2e}")
+
+
+def test_fp8_two_step_form_matches_the_one_call_form():
+    w = shrink(WORKLOADS["large_fp8"], H=2, T=4)
+    (q, k, v), _ = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    q8, k8, qs, ks = _quantize(w, qd, kd)
+    rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
+    o1, l1, st = U.gpu_attn(w, q8, k8, vd, rp, ci, q_scale=qs, k_scale=ks, fp8=True)
+    o2 = torch.full_like(o1, 3.0); l2 = torch.full_like(l1, 3.0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p = B.make_problem(q8, k8, vd, o2, w.N, w.block, 0.0, True)
+    ws = torch.full((B.attn_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
+    B.attn_prepare_v(p, vd, ws)
+    for _ in range(2):                                    # the prepared workspace serves repeated calls
+        o2.fill_(3.0); l2.fill_(3.0)
+        B.block_sparse_attn_fwd_prepared(p, q8, k8, rp, ci, o2, l2, status, workspace=ws, q_scale=qs, k_scale=ks)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(o2[:, :, :w.N], o1[:, :, :w.N]) and torch.equal(l2, l1)
