@@ -175,16 +175,23 @@ def _ws_bytes(ws):
     return ws.numel() * ws.element_size() if ws is not None else 0
 
 
+def block_sparse_attn_fwd_simt(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, q_scale=None,
+                               k_scale=None) -> None:
+    """The diagnostic CUDA-core twin (row_ptr None = dense)."""
+    rc = lib().sva_block_sparse_attn_fwd_simt(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
+                                              _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o),
+                                              _ptr(lse), _ptr(status), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_sparse_attn_fwd_simt")
+
+
 def block_sparse_attn_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, q_scale=None,
                           k_scale=None, simt: bool = False, workspace=None) -> None:
     if simt:
-        rc = lib().sva_block_sparse_attn_fwd_simt(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
-                                                  _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o),
-                                                  _ptr(lse), _ptr(status), _stream())
-    else:
-        rc = lib().sva_block_sparse_attn_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
-                                             _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o), _ptr(lse),
-                                             _ptr(status), _ptr(workspace), _ws_bytes(workspace), _stream())
+        return block_sparse_attn_fwd_simt(p, q, k, v, row_ptr, col_idx, o, lse, status, q_scale, k_scale)
+    rc = lib().sva_block_sparse_attn_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(q_scale),
+                                         _ptr(k_scale), _ptr(row_ptr), _ptr(col_idx), _ptr(o), _ptr(lse),
+                                         _ptr(status), _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_fwd")
 

@@ -25,6 +25,7 @@ def test_header_symbols_exported(lib):
     assert names >= set(B.EXPORTS) and len(names) >= 8
     for n in names:
         assert hasattr(lib, n), n
+        assert callable(getattr(B, n[len("sva_"):], None)), f"no binding function of the same name for {n}"
 
 
 def _problem(**kw):
