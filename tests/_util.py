@@ -131,3 +131,16 @@ def check_attn_vs_oracle(w, qb, kb, vb, row_ptr, col_idx, o_gpu, lse_gpu, rows, 
 def host_inputs(w: Workload, seed=None):
     q, k, v = make_qkv(w, seed)
     return (q, k, v), (bf16_bits(q), bf16_bits(k), bf16_bits(v))
+
+
+def oracle_fp8_inputs(w: Workload, qb, kb, q8, k8, qs, ks):
+    """What the oracle is run on in the FP8 tests: its own codes and scales, made from the bf16 inputs and
+    dequantised in fp64.  The GPU quantiser's bytes must equal them, so the two sides see the same Q, K and
+    nothing the oracle consumes comes from the CUDA path."""
+    out = []
+    for bits, g8, gs in ((qb, q8, qs), (kb, k8, ks)):
+        codes, scales = oracle.quantize_e4m3(bits, w.N, w.block)
+        np.testing.assert_array_equal(gs.cpu().numpy(), scales)
+        assert np.array_equal(g8.cpu().numpy()[:, :, :w.N], codes[:, :, :w.N])
+        out.append(oracle.dequantize_e4m3(codes, scales, w.N, w.block))
+    return out

@@ -69,8 +69,7 @@ def test_full_size_fp8():
         codes, scales = oracle.quantize_e4m3(bits, w.N, w.block)
         np.testing.assert_array_equal(gs.cpu().numpy(), scales)
         assert np.array_equal(g8.cpu().numpy()[:, :, :w.N], codes[:, :, :w.N])
-    qh = oracle.dequantize_e4m3(q8.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
-    kh = oracle.dequantize_e4m3(k8.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+    qh, kh = U.oracle_fp8_inputs(w, qb, kb, q8, k8, qs, ks)
     rp, ci, _ = U.gpu_select(w, q8, k8, q_scale=qs, k_scale=ks, fp8=True)
     sel, _ = U.oracle_select(w, qh, kh)
     n_diff, n_near = U.compare_selection(sel, rp, ci)

@@ -112,7 +112,6 @@ def test_routing_in_two_calls_equals_the_one_call(name):
     torch.cuda.synchronize()
     assert torch.equal(rp1, rp2) and torch.equal(ci1, ci2[: int(rp2[-1])])
     if w.fp8:
-        qb = oracle.dequantize_e4m3(qd.cpu().numpy(), qs.cpu().numpy(), w.N, w.block)
-        kb = oracle.dequantize_e4m3(kd.cpu().numpy(), ks.cpu().numpy(), w.N, w.block)
+        qb, kb = U.oracle_fp8_inputs(w, qb, kb, qd, kd, qs, ks)
     np.testing.assert_allclose(qm.cpu().numpy(), oracle.pool(qb, w.N, w.block), rtol=2e-6, atol=2e-7)
     np.testing.assert_allclose(km.cpu().numpy(), oracle.pool(kb, w.N, w.block), rtol=2e-6, atol=2e-7)
