@@ -84,7 +84,7 @@ typedef struct {
  * where the per-row cap is max(min(k,Nb), window size). */
 int64_t sva_select_max_nnz(const sva_problem_t* p, const sva_select_t* s);
 
-/* Bytes of scratch sva_block_select needs (pooled means, per-row staging). 0 on bad input. */
+/* Bytes of scratch sva_block_select needs (pooled means, the score matrix, per-row staging). 0 on bad input. */
 size_t sva_select_workspace_bytes(const sva_problem_t* p, const sva_select_t* s);
 
 /*
@@ -98,7 +98,9 @@ size_t sva_select_workspace_bytes(const sva_problem_t* p, const sva_select_t* s)
  * order = forced window first, then score descending, ties to the LOWER block index;
  * mode 0 keeps min(k,Nb) blocks, mode 1 the shortest prefix whose softmax mass (over all
  * Nb blocks of the row) reaches `mass`, at least one block, at most k; the forced window is
- * always kept.  Arithmetic is fp32 with a fixed summation order (deterministic).
+ * always kept.  Arithmetic is fp32 with a fixed summation order; the kept mass of mode 1 is summed in
+ * units of 2^-31 (order-independent), which can move a decision only where the mass is within ~1e-7 of
+ * `mass`.  Results are deterministic.
  */
 int sva_block_select(const sva_problem_t* p, const sva_select_t* s, const void* q, const void* k,
                      const float* q_scale, const float* k_scale, int32_t* row_ptr,
@@ -159,7 +161,8 @@ int sva_qk_norm_rope_pool(const sva_problem_t* p, const void* q, const void* k, 
  * those of sva_block_select minus workspace/workspace_bytes.
  *   - Limit: sva_select_workspace_bytes(p, s) must be <= SVA_NOALLOC_SCRATCH_BYTES, otherwise
  *     SVA_ERR_SCRATCH_LIMIT is returned and nothing is launched (B*H*Nb*d*8 bytes of pooled
- *     means dominate: e.g. 24 heads x 256 blocks x d=128 fits, 64 heads x 372 blocks does not).
+ *     means and B*H*Nb*Nb*4 of scores dominate: e.g. 24 heads x 256 blocks x d=128 fits,
+ *     64 heads x 372 blocks does not).
  *   - The first call on each device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls share the one array and it keeps the previous call's contents; every value
@@ -179,9 +182,9 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  *   lse_i = log sum_j exp(scale*<q_i,k_j>)       (optional, [B,H,N] fp32 contiguous)
  * O is bf16.  A row with an empty list writes zeros and lse = -inf.
  * q, k, v, o must be 16-byte aligned and every stride a multiple of 8 elements
- * (16 for e4m3 Q/K).  Tensor-core kernels (bf16 or e4m3 x e4m3 MMA, fp32 accumulate) serve d = 128:
- * bf16 or e4m3 Q/K with 128- or 64-token blocks; d = 64 runs on the same kernels (computed as d = 128 with
- * a zero upper half).
+ * (16 for e4m3 Q/K).  One tensor-core kernel (bf16 x bf16 or e4m3 x e4m3 MMA for Q K^T, bf16 for P V,
+ * fp32 accumulate) serves every supported shape: d = 128 or 64 (64 is computed as 128 with a zero upper
+ * half), bf16 or e4m3 Q/K, 128- or 64-token blocks.
  * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The tensor-core kernel
  * keeps a tiled, transposed copy of V (2*B*H*Nb*block*128 bytes), its row counter and, for 64-token
  * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
