@@ -240,12 +240,14 @@ int svo_select(const double *s, int R, int Nb, int mode, int k, double tau, int 
         cum += exp(key[m - 1].s - mx) / z;
         if (cum >= tau) { n = m; break; }
       }
-      /* near-boundary report: only the prefixes next to the crossing, and only
-         those shorter than the cap, can change the final count */
+      /* near-boundary report: a prefix shorter than the cap whose mass is close to tau is
+         where an implementation in lower precision may stop instead (below the crossing the
+         mass only grows, so the closest one is the longest such prefix; when the crossing
+         lies beyond the cap -- tau = 1 -- that is prefix k-1, not n-1) */
       cum = 0.0;
-      for (int m = 1; m <= n; ++m) {
+      for (int m = 1; m <= n && m <= k - 1; ++m) {
         cum += exp(key[m - 1].s - mx) / z;
-        if ((m == n - 1 || m == n) && m <= k - 1 && fabs(cum - tau) < margin) margin = fabs(cum - tau);
+        if (fabs(cum - tau) < margin) margin = fabs(cum - tau);
       }
       if (n > k) n = k;
     }

@@ -109,9 +109,27 @@ def test_mass_rule_brute_force_and_margin():
         n = int(np.argmax(cum >= tau)) + 1
         assert sel.counts[r] == min(n, cap)
         assert sel.kept(r).tolist() == sorted(order[:min(n, cap)])
-        cands = [abs(cum[m - 1] - tau) for m in (n - 1, n) if 1 <= m <= cap - 1]
+        # the margin: how close the mass comes to tau at any prefix shorter than the cap (up to the crossing)
+        cands = [abs(cum[m - 1] - tau) for m in range(1, min(n, cap - 1) + 1)]
         exp_margin = min(cands) if cands else np.inf
         assert sel.mass_margin[r] == pytest.approx(exp_margin, rel=1e-9)
+
+
+def test_mass_margin_when_the_crossing_lies_beyond_the_cap():
+    """tau = 1 is only reached by all blocks together, so the cap decides the count -- but a peaked row gets
+    within rounding of 1 after two blocks, which is where an fp32 implementation stops: the row must be
+    reported as a near-tie."""
+    Nb, cap = 8, 5
+    row = np.array([30.0, 29.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0])
+    s = np.tile(row, (1, 1, Nb, 1))
+    sel = oracle.select(s, 1, cap, 1.0)
+    assert (sel.counts == cap).all()                       # the rule itself: mass < 1 until the last block, capped at 5
+    p = np.exp(row - row.max()); p /= p.sum()
+    assert sel.mass_margin[0] == pytest.approx(1.0 - np.cumsum(p)[cap - 2], rel=1e-6)
+    assert sel.mass_margin[0] < 1e-10
+    # a flat row is nowhere near tau before the cap
+    sel2 = oracle.select(np.zeros((1, 1, Nb, Nb)), 1, cap, 1.0)
+    assert (sel2.counts == cap).all() and (sel2.mass_margin > 0.4).all()
 
 
 def test_forced_window_hand_enumerated():
