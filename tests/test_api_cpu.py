@@ -77,6 +77,7 @@ def test_rejects_bad_arguments_before_launch(lib):
     assert sel(p, B.make_select(1, 4, 0.0)) == 1
     assert sel(p, B.make_select(0, 4, 1.0, 1, 1, 3)) == 1            # Nb not a multiple of strips/frame
     assert sel(p, s, q=None) == 1
+    assert sel(_problem(N=64 * 1025, block=64), s) == 2                # more than 1024 blocks per head
     assert sel(p, s, ws=None) == 3
     assert sel(p, s, wsb=16) == 3
     assert sel(p, s, q=vp(8)) == 5

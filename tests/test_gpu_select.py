@@ -115,3 +115,20 @@ def test_routing_in_two_calls_equals_the_one_call(name):
         qb, kb = U.oracle_fp8_inputs(w, qb, kb, qd, kd, qs, ks)
     np.testing.assert_allclose(qm.cpu().numpy(), oracle.pool(qb, w.N, w.block), rtol=2e-6, atol=2e-7)
     np.testing.assert_allclose(km.cpu().numpy(), oracle.pool(kb, w.N, w.block), rtol=2e-6, atol=2e-7)
+
+
+@pytest.mark.parametrize("T,Hg,Wg,mode,k,tau,d", [(25, 40, 40, 0, 20, 1.0, 128), (16, 64, 64, 1, 30, 0.95, 64)])
+def test_many_blocks_per_head(T, Hg, Wg, mode, k, tau, d):
+    """625 and 1024 (the maximum) 64-token blocks per head: every lane of the selection warp holds up to 32
+    scores of its row; routing against the oracle, attention on sampled rows."""
+    w = shrink(WORKLOADS["medium"], B=1, H=1, T=T, Hg=Hg, Wg=Wg, block=64, mode=mode, k=k, tau=tau, d=d, win_t=-1, win_s=-1)
+    (q, kk, v), (qb, kb, vb) = U.host_inputs(w, seed=5)
+    qd, kd, vd = U.dev(q), U.dev(kk), U.dev(v)
+    rp, ci, sc = U.gpu_select(w, qd, kd, want_scores=True)
+    sel, s_ref = U.oracle_select(w, qb, kb)
+    assert np.abs(sc.cpu().numpy() - s_ref).max() < 2e-5
+    n_diff, n_near = U.compare_selection(sel, rp, ci)
+    assert n_diff <= n_near
+    o, lse, st = U.gpu_attn(w, qd, kd, vd, rp, ci)
+    assert st == 0
+    U.check_attn_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, U.sample_rows(w.R, w.Nb, 6))
