@@ -33,9 +33,12 @@ from paper_2606_23743_b200.workloads import SEED_BASE, WORKLOADS, bf16_bits, mak
 METRIC = "block-sparse attn fwd effective TFLOPS (selected blocks)"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_ts_kernel launch on the "large" workload,
-# from the ncu capture summarised in profiles/attn_ts_kernel_large.md (other workloads: not captured)
-ATTN_TRAFFIC_BYTES = {"large": 796.0e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, constants copied from one ncu capture each
+# (`ncu --set full --clock-control none -k regex:<kernel> -c 1` of this script on the "large" workload);
+# they are not measured by this run.  Other workloads: not captured (null).
+ATTN_TRAFFIC_BYTES = {"large": 796.0e6}           # attn_ts_kernel alone
+TRANSPOSE_TRAFFIC_BYTES = {"large": 355.9e6}      # transpose_v_kernel (201.3 MB read + 154.6 MB written)
+SM_COUNT_FALLBACK = 148
 
 
 def load_peaks():
@@ -50,8 +53,9 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, device_index: int):
+    def __init__(self, device_index: int, period_s: float = 0.002):
         self.samples, self.reasons, self.max_mhz, self.power = [], set(), None, []
+        self.period_s = period_s
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -90,7 +94,7 @@ class ClockSampler:
                 self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(self.period_s)
 
     def start(self):
         if self._nv is not None:
@@ -102,8 +106,12 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.join()
         med = float(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples), "power_w_max": max(self.power) if self.power else None}
+        # NVML's clock and power readings lag by tens of milliseconds: a record of fewer than ~100 samples
+        # (a burst of a few dozen ms) describes the idle GPU before the burst, not the burst
+        return {"sm_mhz": med, "sm_mhz_min": float(min(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples), "power_w_max": max(self.power) if self.power else None,
+                "reliable": len(self.samples) >= 100}
 
 
 def flops_per_tile(w):
@@ -192,6 +200,8 @@ def main():
     ap.add_argument("--workload", default="large", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=2.5,
+                    help="length of the second, back-to-back leg whose clocks NVML can follow (0 = skip)")
     ap.add_argument("--prologue", action="store_true",
                     help="extended step: the fused QK-norm + RoPE prologue in front (it also writes the block means, "
                          "and the e4m3 codes of an FP8 workload, so routing skips its pooling pass and the quantiser)")
@@ -332,6 +342,73 @@ def main():
     value = job_flops / (ms_per_step * 1e-3) / 1e12
     assert int(status.item()) == 0, "device status set during the timed region"
 
+    # ---- the same step back to back for seconds: the regime a denoising loop lives in (the part is
+    # power-limited, so the SM clock settles below its burst value) and the only one NVML's readings can
+    # follow.  Same work per step as above; nothing of it enters `value`.
+    sms = torch.cuda.get_device_properties(local_rank).multi_processor_count or SM_COUNT_FALLBACK
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / ms_per_step) + 1)
+        s_att = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_sus)]
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sus_sampler = ClockSampler(local_rank, period_s=0.005)
+        D.barrier()
+        torch.cuda.synchronize()
+        s0.record()
+        for i in range(n_sus):
+            route(q, k, v)
+            s_att[i][0].record()
+            attend(q, k, v, o)
+            s_att[i][1].record()
+            if i == n_sus // 5:
+                sus_sampler.start()               # sample the settled part only (the first fifth ramps down)
+        s1.record()
+        torch.cuda.synchronize()
+        sus_clocks = sus_sampler.stop()
+        D.barrier()
+        sus_ms = D.max_over_ranks(s0.elapsed_time(s1)) / n_sus
+        tail = s_att[n_sus // 5:]
+        sus_attn_ms = float(np.mean([a.elapsed_time(b) for a, b in tail]))
+        mhz = sus_clocks["sm_mhz"]
+        sustained = {"seconds": sus_ms * n_sus * 1e-3, "steps": n_sus, "ms_per_step": sus_ms,
+                     "value": job_flops / (sus_ms * 1e-3) / 1e12, "attention_ms": sus_attn_ms,
+                     "attention_tflops": step_flops / (sus_attn_ms * 1e-3) / 1e12,
+                     "sm_mhz_median": mhz, "sm_mhz_min": sus_clocks["sm_mhz_min"],
+                     "power_w_max": sus_clocks["power_w_max"], "reasons": sus_clocks["reasons"],
+                     "clock_samples": sus_clocks["samples"],
+                     "cycles_per_tile": sus_attn_ms * 1e-3 * mhz * 1e6 * sms / nnz if mhz else None,
+                     "note": "attention_ms, clocks and power over the last four fifths of the leg"}
+        assert int(status.item()) == 0, "device status set during the sustained leg"
+
+    # ---- the kernel's own cycle counter (one extra launch): cycles do not depend on the SM clock, so
+    # cycles / measured time is the clock each regime really ran at -- the record NVML cannot give for a burst
+    kernel_cycles = None
+    if two_step:
+        prof = torch.zeros(320, dtype=torch.int64, device=dev)
+        B.debug_set_prof_buffer(prof)
+        try:
+            route(q, k, v)
+            attend(q, k, v, o)
+            torch.cuda.synchronize()
+        finally:
+            B.debug_set_prof_buffer(None)
+        kernel_cycles = int(prof[319].item())
+
+    # ---- attention with its V preparation in line (the one-call entry point: transpose, then the kernel)
+    inline_ms = None
+    if two_step and not w.fp8 and not args.prologue:
+        n_in = max(5, min(args.steps, 20))
+        route(q, k, v)
+        torch.cuda.current_stream().wait_event(v_ready)
+        i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(n_in + 3):
+            if i == 3:
+                i0.record()
+            B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status, workspace=aws)
+        i1.record()
+        torch.cuda.synchronize()
+        inline_ms = i0.elapsed_time(i1) / n_in
+
     # ---- end to end: pinned host -> device, path, device -> pinned host, every step
     e2e = None
     if not args.no_e2e:
@@ -404,6 +481,19 @@ def main():
         "select_gbs": sel_bytes / (sel_ms * 1e-3) / 1e9,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
+                     "traffic_source": "constant from one ncu capture of attn_ts_kernel on this workload, not measured by this run",
+                     "traffic_with_v_transpose": (ATTN_TRAFFIC_BYTES[w.name] + TRANSPOSE_TRAFFIC_BYTES[w.name])
+                     if w.name in ATTN_TRAFFIC_BYTES and w.name in TRANSPOSE_TRAFFIC_BYTES else None,
+                     "algorithmic_bytes": 8.0 * w.B * w.H * w.N * w.d,
+                     "frac_with_prepare": (step_flops / (inline_ms * 1e-3) / 1e12 / peak) if inline_ms else None,
+                     "attention_with_prepare_ms": inline_ms,
+                     "frac_whole_step": value / world / peak,
+                     "kernel_cycles": kernel_cycles,
+                     "cycles_per_tile": kernel_cycles * min(sms, w.R) / nnz if kernel_cycles else None,
+                     "cycles_source": "clock64 of the longest CTA of one extra launch (sva_debug_set_prof_buffer)",
+                     "sm_mhz_implied_burst": kernel_cycles / (attn_ms * 1e3) if kernel_cycles else None,
+                     "sm_mhz_implied_sustained": kernel_cycles / (sustained["attention_ms"] * 1e3)
+                     if kernel_cycles and sustained else None,
                      "kernel": "attn_ts_kernel" + (" (the V transpose runs beside routing on a second stream)" if two_step
                                                   else " with the V transpose in front of it"),
                      "mixed_precision_ceiling": peak * 4.0 / 3.0 if w.fp8 else None,
@@ -411,7 +501,7 @@ def main():
                      "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"])
                      if "bf16_tflops_sustained" in peaks else None,
                      "frac_of_nominal_2250": achieved / 2250.0},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks, "sustained": sustained, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline and not args.prologue:   # (the oracle leg times the plain step)

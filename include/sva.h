@@ -23,7 +23,17 @@
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*), never
  *     synchronise the device and may be issued back to back on one stream.
  *   - The library allocates no device memory; scratch is the caller's `workspace`
- *     (routing and attention each state their size).
+ *     (routing and attention each state their size).  One exception, by design:
+ *     sva_block_select_noalloc takes its scratch from a 16 MiB device array that is part of
+ *     the library image.  The library keeps no state between calls apart from per-device
+ *     caches of constants (SM count, function attributes, that array's address) and the
+ *     process-global test switches of sva_debug.h.
+ *   - Three things differ from the boundary as first drafted for this path and are deliberate:
+ *     (i) the attention calls take `workspace, workspace_bytes` (the tensor-core kernel reads V
+ *     from a tiled transposed copy, and the library does not allocate); (ii) faults found on
+ *     the device are bits in *device_status (SVA_DEV_*), not return codes: the calls are
+ *     asynchronous, so the host cannot know at return time; (iii) "no forced window" is a
+ *     NEGATIVE half-width; win_t = win_s = 0 is a window of one block, the diagonal.
  *   - Every call validates its arguments on the host first and returns a non-zero
  *     sva_status_t WITHOUT launching anything when they are bad.  No exception
  *     crosses the ABI.  Non-finite inputs give undefined (but memory-safe) results.
@@ -80,8 +90,10 @@ typedef struct {
   int32_t blocks_per_frame;  /* strips per frame; Nb must be a multiple when a window is set */
 } sva_select_t;
 
-/* Capacity (in entries) that col_idx must have for sva_block_select: R * per-row cap,
- * where the per-row cap is max(min(k,Nb), window size). */
+/* Size queries for the routing call below (the routing step of the paper's sparse attention; they
+ * compute nothing).  Capacity (in entries) that col_idx must have for sva_block_select: R * per-row cap,
+ * where the per-row cap is max(min(k,Nb), window size).  0 on bad input, for more than 1024 blocks per
+ * head (the routing kernels' limit) and when R * cap would not fit the CSR's int32 offsets. */
 int64_t sva_select_max_nnz(const sva_problem_t* p, const sva_select_t* s);
 
 /* Bytes of scratch sva_block_select needs (pooled means, the score matrix, per-row staging). 0 on bad input. */
@@ -234,7 +246,9 @@ int sva_block_sparse_attn_fwd_simt(const sva_problem_t* p, const void* q, const 
                                    float* lse, int32_t* device_status, void* stream);
 
 /*
- * FP8 variant's quantiser: per (b,h,block) absmax a over the valid tokens, scale s = a/448
+ * FP8 variant's quantiser (the problem statement's "FP8 QK^T variant for the paper's quantization
+ * technique"; the paper's Quantization section cites the 8-bit attention line of work for it and prints no
+ * formula): per (b,h,block) absmax a over the valid tokens, scale s = a/448
  * (s = 1 when a = 0), y = x/s in fp32, round-to-nearest-even saturating cast to OCP e4m3.
  * q8/k8 use the strides of p (in elements = bytes); scales are [B,H,Nb] fp32.
  */

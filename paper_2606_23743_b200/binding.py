@@ -25,6 +25,7 @@ EXPORTS = [
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
     "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
 ]
+DEBUG_EXPORTS = ["sva_debug_set_prof_buffer", "sva_debug_set_mode", "sva_debug_set_wait_limit"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
 
@@ -96,6 +97,13 @@ def lib():
         L.sva_qk_norm_rope_pool.restype = C.c_int
         L.sva_qk_norm_rope_pool.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp, vp, vp,
                                             vp, vp, vp]
+        # test and tuning aids (include/sva_debug.h): process-global settings
+        L.sva_debug_set_prof_buffer.restype = None
+        L.sva_debug_set_prof_buffer.argtypes = [vp]
+        L.sva_debug_set_mode.restype = None
+        L.sva_debug_set_mode.argtypes = [C.c_int]
+        L.sva_debug_set_wait_limit.restype = C.c_int
+        L.sva_debug_set_wait_limit.argtypes = [C.c_longlong]
         L.sva_status_string.restype = C.c_char_p
         L.sva_status_string.argtypes = [C.c_int]
         _lib = L
@@ -256,14 +264,14 @@ def smooth_workspace_bytes(p: Problem) -> int:
 def quantize_qk_fp8_smooth_k(p: Problem, q, k, q8, k8, q_scale, k_scale, k_mean, lse_shift, workspace) -> None:
     rc = lib().sva_quantize_qk_fp8_smooth_k(C.byref(p), _ptr(q), _ptr(k), _ptr(q8), _ptr(k8), _ptr(q_scale),
                                             _ptr(k_scale), _ptr(k_mean), _ptr(lse_shift), _ptr(workspace),
-                                            C.c_size_t(workspace.numel() if workspace is not None else 0), _stream())
+                                            C.c_size_t(_ws_bytes(workspace)), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_quantize_qk_fp8_smooth_k")
 
 
 def block_select_pooled(p: Problem, s: Select, q_mean, k_mean, row_ptr, col_idx, workspace, block_scores=None) -> None:
     rc = lib().sva_block_select_pooled(C.byref(p), C.byref(s), _ptr(q_mean), _ptr(k_mean), _ptr(row_ptr), _ptr(col_idx),
-                                       _ptr(block_scores), _ptr(workspace), C.c_size_t(workspace.numel()), _stream())
+                                       _ptr(block_scores), _ptr(workspace), C.c_size_t(_ws_bytes(workspace)), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_select_pooled")
 
@@ -282,3 +290,20 @@ def pool_qk(p: Problem, q, k, q_mean, k_mean, q_scale=None, k_scale=None) -> Non
                            _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_pool_qk")
+
+
+def debug_set_prof_buffer(buf) -> None:
+    """Cycle counter of the attention kernel (include/sva_debug.h): a zeroed device int64 tensor of >= 320
+    entries, entry 319 receives the cycle count of the longest CTA of later launches; None switches it off."""
+    lib().sva_debug_set_prof_buffer(_ptr(buf))
+
+
+def debug_set_mode(bits: int) -> None:
+    """Kernel behaviour switches of later attention launches (include/sva_debug.h); 0 = normal."""
+    lib().sva_debug_set_mode(int(bits))
+
+
+def debug_set_wait_limit(cycles: int) -> None:
+    """SM cycles a device-side wait may last before its CTA gives up; <= 0 restores the default."""
+    if lib().sva_debug_set_wait_limit(C.c_longlong(int(cycles))) != 0:
+        raise RuntimeError("sva_debug_set_wait_limit failed")

@@ -27,6 +27,12 @@ static int check_strides(const int64_t s[3], int mult) {
   return SVA_OK;
 }
 
+// What the routing kernels cannot take: more than 1024 blocks per head (a lane holds at most 32 scores of
+// a row), or a CSR whose capacity R * cap would overflow its int32 offsets.
+static bool select_fits(const Dims& m, const sva_select_t* s) {
+  return m.Nb <= 1024 && (long long)m.R * select_row_cap(m, s) <= 0x7fffffffLL;
+}
+
 static int validate_select(const Dims& m, const sva_select_t* s) {
   if (!s) return SVA_ERR_INVALID_ARG;
   if (s->mode != 0 && s->mode != 1) return SVA_ERR_INVALID_ARG;
@@ -35,6 +41,7 @@ static int validate_select(const Dims& m, const sva_select_t* s) {
   if (s->win_t >= 0 && s->win_s >= 0) {
     if (s->blocks_per_frame <= 0 || m.Nb % s->blocks_per_frame != 0) return SVA_ERR_INVALID_ARG;
   }
+  if (!select_fits(m, s)) return SVA_ERR_UNSUPPORTED;
   return SVA_OK;
 }
 
@@ -55,8 +62,9 @@ static int validate_attn(const sva_problem_t* p, const void* q, const void* k, c
   return SVA_OK;
 }
 
-// The tensor-core kernel (attn_ts_serves: every shape the library takes today; it needs the transposed-V
-// workspace); the CUDA-core kernel stays behind it for shapes it would not serve.
+// The tensor-core kernel serves every shape validate_problem lets through except more than 16383 key
+// blocks per head (its 64-token-block tile descriptors hold 14-bit block indices); only there do the
+// public attention calls run the CUDA-core kernel instead.
 
 }  // namespace sva
 
@@ -67,12 +75,14 @@ extern "C" {
 int64_t sva_select_max_nnz(const sva_problem_t* p, const sva_select_t* s) {
   if (validate_problem(p) || !s || s->k < 1) return 0;
   Dims m = make_dims(p);
+  if (!select_fits(m, s)) return 0;
   return (int64_t)m.R * select_row_cap(m, s);
 }
 
 size_t sva_select_workspace_bytes(const sva_problem_t* p, const sva_select_t* s) {
   if (validate_problem(p) || !s || s->k < 1) return 0;
   Dims m = make_dims(p);
+  if (!select_fits(m, s)) return 0;
   return select_workspace_bytes(m, s);
 }
 

@@ -45,7 +45,9 @@ attn_simt_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ k,
 
   int beg, end;
   if (row_ptr) { beg = row_ptr[r]; end = row_ptr[r + 1]; } else { beg = 0; end = Nb; }
-  if (end < beg || end - beg > Nb) {       // corrupt row: report, write the empty-row result
+  if (beg < 0 || end < beg || end - beg > Nb || (row_ptr && end > row_ptr[gridDim.x])) {
+    // corrupt row (not monotone, too long, or reaching beyond the row_ptr[R] entries the CSR says it has):
+    // report, read no entry, write the empty-row result
     if (threadIdx.x == 0 && status) atomicOr(status, SVA_DEV_BAD_INDEX);
     end = beg;
   }

@@ -47,6 +47,8 @@
 // Every wait is bounded: when one expires the CTA sets SVA_DEV_TIMEOUT, all roles leave their
 // loops, TMEM is released and the kernel returns.  Parity waits never run a whole phase ahead of
 // their barrier (each wait on a barrier is preceded by a wait on its previous phase).
+#include <mutex>
+
 #include "tc_ptx.cuh"
 
 namespace sva {
@@ -101,21 +103,25 @@ constexpr float LAZY_LOG2 = 32.0f;
 //   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
 //   3328 row queue: QD entries {row, count, start, first entry, second entry, -, -, -} | 3456 rq_full[QD] | 3488 rq_empty[QD]
 
-// Work list of row r (a 128-query tile): count and start.  128-token blocks: the CSR row itself (a corrupt
-// row_ptr pair gives an empty row).  64-token blocks: the tile row's list of 128-key tiles that
-// pair_lists_kernel built from the two CSR rows of the tile.  Every role calls this with the same
-// inputs and so reaches the same answer.
+// Work list of row r (a 128-query tile): count and start; returns false for a corrupt row_ptr pair.
+// 128-token blocks: the CSR row itself.  A pair that is not monotone, longer than Nb, negative or that
+// reaches beyond nnz_bound (= row_ptr[R], the number of entries the CSR says it has) gives an empty row,
+// so no col_idx entry outside [0, row_ptr[R]) is ever read.  64-token blocks: the tile row's list of
+// 128-key tiles that pair_lists_kernel built (and checked) from the two CSR rows of the tile.
+// Only the K producer calls this; the other roles take its answer from the row queue.
 template <bool B64>
-__device__ __forceinline__ void row_list(const TsParams& prm, int r, int& n, int& beg) {
+__device__ __forceinline__ bool row_list(const TsParams& prm, int r, int nnz_bound, int& n, int& beg) {
   if (B64) {
-    if (prm.row_ptr == nullptr) { n = (prm.Nb + 1) >> 1; beg = 0; return; }     // dense: every pair of key blocks
+    if (prm.row_ptr == nullptr) { n = (prm.Nb + 1) >> 1; beg = 0; return true; }     // dense: every pair of key blocks
     n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r);
-    return;
+    return true;
   }
-  if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return; }
+  if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return true; }
   beg = __ldg(prm.row_ptr + r);
-  n = __ldg(prm.row_ptr + r + 1) - beg;
-  if (n < 0 || n > prm.Nb || beg < 0) n = 0;
+  const int end = __ldg(prm.row_ptr + r + 1);
+  n = end - beg;
+  if (beg < 0 || end < beg || n > prm.Nb || end > nnz_bound) { n = 0; beg = 0; return false; }
+  return true;
 }
 // Entry j of a work list.  128-token blocks: the key block (an out-of-range entry is replaced by block 0;
 // the producer reports it).  64-token blocks: the tile descriptor.
@@ -231,6 +237,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int s = 0;
         uint32_t ph = 0;
         bool ok = true;
+        const int nnz_bound = (!B64 && prm.row_ptr) ? __ldg(prm.row_ptr + prm.R) : 0;
         for (uint32_t i = 0; ok; ++i) {
           // ---- row scheduling: draw the next row with a non-empty list and publish it
           const uint32_t slot = i % QD;
@@ -239,7 +246,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (;;) {
             r = atomicAdd(prm.next_row, 1);
             if (r >= prm.R) break;
-            row_list<B64>(prm, r, n, beg);
+            if (!row_list<B64>(prm, r, nnz_bound, n, beg) && prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX);
             if (n > 0) break;
             // nothing kept (or a corrupt row_ptr pair): zeros and lse = -inf; rare, so this one lane does it
             const int I = r % Nb, bh0 = r / Nb;
@@ -771,7 +778,8 @@ pair_lists_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict
   __syncwarp();
   const int begA = __ldg(row_ptr + rA), endA = __ldg(row_ptr + rA + 1);
   const int endB = hasB ? __ldg(row_ptr + rA + 2) : endA;
-  const bool bad = begA < 0 || endA < begA || endB < endA || endA - begA > Nb || endB - endA > Nb;
+  const int nnz_bound = __ldg(row_ptr + (R2 / Nt) * Nb);      // row_ptr[R]: the entries the CSR says it has
+  const bool bad = begA < 0 || endA < begA || endB < endA || endA - begA > Nb || endB - endA > Nb || endB > nnz_bound;
   bool bad_idx = false;
   if (!bad) {
     for (int e = begA + lane; e < endB; e += 32) {
@@ -853,16 +861,32 @@ static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuui
 static long long* g_prof_ts = nullptr;
 static int g_debug_ts = 0;
 
+// Per-device constants looked up once (the SM count, and the shared-memory opt-in of each kernel variant):
+// a cache, not state -- every call would find the same values.
+static constexpr int TS_MAX_DEVICES = 64;
+static std::mutex g_ts_mutex;
+static int g_ts_sms[TS_MAX_DEVICES];
+static bool g_ts_attr[TS_MAX_DEVICES][4];
+
 template <bool B64, bool F8>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                      const TsParams& prm, cudaStream_t st) {
   auto kern = attn_ts_kernel<B64, F8>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
-    return SVA_ERR_CUDA;
   int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-    return SVA_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lock(g_ts_mutex);
+    constexpr int variant = (B64 ? 2 : 0) + (F8 ? 1 : 0);
+    if (!g_ts_attr[dev][variant]) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
+        return SVA_ERR_CUDA;
+      g_ts_attr[dev][variant] = true;
+    }
+    if (g_ts_sms[dev] <= 0 &&
+        (cudaDeviceGetAttribute(&g_ts_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_ts_sms[dev] <= 0))
+      return SVA_ERR_CUDA;
+    sms = g_ts_sms[dev];
+  }
   const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
   kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;

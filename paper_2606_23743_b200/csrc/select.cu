@@ -3,11 +3,13 @@
 // window, CSR assembly.  (Paper: "score-based routing" of the critical blocks; block-wise
 // similarity metric of the sparse-attention section.)
 //
-// Kernel 1 (pool) streams Q and K once from HBM: 128-bit loads, fp32 accumulation in a fixed
-// order, one CTA per (block, head, tensor).  Kernel 2 (score+select) is one warp per query
-// block row with the head's pooled K staged through shared memory.  When the per-row count is
-// not a compile-time constant of the call (mass rule, or a window larger than k), rows are
-// staged and kernels 3/4 (scan, compact) build the CSR.
+// pool_kernel streams Q and K once from HBM: 128-bit loads, fp32 accumulation in a fixed order, one
+// CTA per (block, head, tensor).  block_scores_kernel computes a head's score matrix as a small fp32
+// GEMM (64 x 64 tiles from two shared-memory panels, fixed summation order).  select_rows_kernel is one
+// warp per query-block row: it reads the row's scores from that matrix (no shared memory), finds the
+// threshold of the rule by bisection on order-preserving integer keys and emits the kept blocks in
+// ascending order.  When the per-row count is known on the host (top-k with no window larger than k)
+// rows go straight into the CSR; otherwise they are staged and scan_kernel + compact_kernel build it.
 #include <mutex>
 
 #include "common.cuh"

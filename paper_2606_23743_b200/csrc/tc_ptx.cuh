@@ -37,15 +37,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(SVA_SUSPEND_HINT_NS) : "memory");
   return ok;
 }
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {      // non-blocking
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok;
-}
 // Bounded wait.  Returns false when the CTA is aborting.  SLEEP_NS > 0 backs off between polls
 // (for roles whose wake-up latency is not on the critical path).  The first poll is marked as the
 // likely exit so that the polling loop is laid out away from the hot instruction stream
@@ -99,19 +90,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t elected) {
   asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
                "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
                ::"r"(bar), "r"(elected) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-template <bool F8>
-__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc,
-                                          uint32_t elected) {
-  if (F8)
-    asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
-                 "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
-  else
-    asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
-                 "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]; F8: 8-bit operands (kind::f8f6f4, K = 32 per instruction)
 template <bool F8 = false>
@@ -194,7 +172,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
-// 2^x for x <= ~8 on the FMA pipe: round-to-nearest split x = n + f, |f| <= 0.5, cubic minimax
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

@@ -93,9 +93,12 @@ def sequence_parallel_attention(q_local: torch.Tensor, k_local: torch.Tensor, v_
     return head_to_seq_shard(attend(q, k, v), shard_sizes, group)
 
 
-def sparse_attend(select, block: int = 128):
+def sparse_attend(select, block: int = 128, status=None):
     """The library's routing + block-sparse attention as an `attend` callable for CUDA bf16 tensors
-    (select: a `binding.Select`).  Buffers are allocated per call; a serving loop would keep them."""
+    (select: a `binding.Select`).  Buffers are allocated per call; a serving loop would keep them.
+    `status`: optional caller-owned device int32[1] that the kernels OR their SVA_DEV_* bits into (zero it
+    first); without one the callable allocates its own.  Either way the word the last call used is
+    `attend.status` -- read it after a synchronisation; a non-zero value means the output is not valid."""
     from . import binding as B
 
     def attend(q, k, v):
@@ -108,10 +111,12 @@ def sparse_attend(select, block: int = 128):
         ws = torch.empty(max(B.select_workspace_bytes(p, select), 256), dtype=torch.uint8, device=q.device)
         row_ptr = torch.zeros(R + 1, dtype=torch.int32, device=q.device)
         col_idx = torch.zeros(max(B.select_max_nnz(p, select), 1), dtype=torch.int32, device=q.device)
-        status = torch.zeros(1, dtype=torch.int32, device=q.device)
+        st = status if status is not None else torch.zeros(1, dtype=torch.int32, device=q.device)
+        attend.status = st
         aws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device=q.device)
         B.block_select(p, select, q, k, row_ptr, col_idx, ws)
-        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, status, workspace=aws)
+        B.block_sparse_attn_fwd(p, q, k, v, row_ptr, col_idx, o, None, st, workspace=aws)
         return o
 
+    attend.status = status
     return attend

@@ -89,11 +89,28 @@ def sample_rows(R: int, Nb: int, n: int, seed: int = 0):
     return sorted(rows)
 
 
+def sample_rows_per_head(BH: int, Nb: int, n_random: int = 8, seed: int = 0):
+    """The full-size sample: for EVERY (b, h) query block 0, the last (ragged) query block and
+    `n_random` seeded random ones, as row indices r = bh * Nb + I."""
+    rng = np.random.default_rng(seed)
+    rows = []
+    for bh in range(BH):
+        mine = {0, Nb - 1}
+        while len(mine) < min(n_random + 2, Nb):
+            mine.add(int(rng.integers(0, Nb)))
+        rows += [bh * Nb + I for I in sorted(mine)]
+    return rows
+
+
 def attn_errors(o_gpu, lse_gpu, o_ref, lse_ref, rows, N, block, H):
     """o_gpu [B,H,n_alloc,d] bf16 device; o_ref [n_rows, block, d] f64 with NaN for absent queries."""
     Bq, Hq, n_alloc, d = o_gpu.shape
     Nb = -(-N // block)
-    og = o_gpu.float().cpu().numpy().astype(np.float64)
+    # only the sampled query blocks leave the device (a full-size tensor in fp64 would be gigabytes)
+    rt = torch.as_tensor(rows, device=o_gpu.device, dtype=torch.int64)
+    tok = ((rt % Nb) * block)[:, None] + torch.arange(block, device=o_gpu.device)[None, :]
+    flat = o_gpu.reshape(Bq * Hq, n_alloc, d)
+    og_rows = flat[(rt // Nb)[:, None], tok.clamp_(max=n_alloc - 1)].float().cpu().numpy().astype(np.float64)
     num = den = 0.0
     max_abs = 0.0
     lse_err = 0.0
@@ -101,7 +118,7 @@ def attn_errors(o_gpu, lse_gpu, o_ref, lse_ref, rows, N, block, H):
         bh, I = divmod(r, Nb)
         lo, hi = I * block, min((I + 1) * block, N)
         ref = o_ref[t, : hi - lo]
-        got = og[bh // Hq, bh % Hq, lo:hi]
+        got = og_rows[t, : hi - lo]
         assert not np.isnan(ref).any()
         diff = got - ref
         num += (diff ** 2).sum(); den += (ref ** 2).sum()

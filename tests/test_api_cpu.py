@@ -19,10 +19,12 @@ def lib():
 
 
 def test_header_symbols_exported(lib):
-    text = open(os.path.join(ROOT, "include", "sva.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = set(re.findall(r"\b(sva_[a-z0-9_]+)\s*\(", text))
-    assert names >= set(B.EXPORTS) and len(names) >= 8
+    names = set()
+    for header in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        text = open(os.path.join(ROOT, "include", header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(sva_[a-z0-9_]+)\s*\(", text))
+    assert names == set(B.EXPORTS) | set(B.DEBUG_EXPORTS), names ^ (set(B.EXPORTS) | set(B.DEBUG_EXPORTS))
     for n in names:
         assert hasattr(lib, n), n
         assert callable(getattr(B, n[len("sva_"):], None)), f"no binding function of the same name for {n}"
@@ -171,3 +173,21 @@ def test_token_move_rejects_bad_arguments_before_launch(lib):
         assert mv(fn, dst=C.c_void_p(8)) == 5
         assert mv(fn, ss=(C.c_int64 * 3)(0, 0, 132)) == 5
         assert mv(fn, ss=(C.c_int64 * 3)(0, 0, 64)) == 1  # row stride shorter than a row
+
+
+def test_routing_limits_are_refused_on_the_host(lib):
+    """More than 1024 blocks per head, or a CSR capacity R * cap beyond int32: size queries answer 0 and the
+    routing calls return UNSUPPORTED before any launch (no silent wrap of the int32 offsets)."""
+    big_nb = _problem(N=128 * 1025)                       # Nb = 1025
+    s = B.make_select(0, 4)
+    assert B.select_max_nnz(big_nb, s) == 0 and B.select_workspace_bytes(big_nb, s) == 0
+    many = _problem(B=32, H=512, N=128 * 1024)            # R = 2^24 rows, k = 128 -> 2^31 entries
+    s64 = B.make_select(0, 128)
+    assert B.select_max_nnz(many, s64) == 0 and B.select_workspace_bytes(many, s64) == 0
+    assert B.select_max_nnz(many, B.make_select(0, 127)) == (32 * 512 * 1024) * 127
+    fake = C.c_void_p(256)
+    for p, sel in ((big_nb, s), (many, s64)):
+        for fn, args in ((lib.sva_block_select, (fake, fake, None, None, fake, fake, None, fake, C.c_size_t(1 << 40), None)),
+                         (lib.sva_block_select_pooled, (fake, fake, fake, fake, None, fake, C.c_size_t(1 << 40), None)),
+                         (lib.sva_block_select_noalloc, (fake, fake, None, None, fake, fake, None, None))):
+            assert fn(C.byref(p), C.byref(sel), *args) == 2, fn

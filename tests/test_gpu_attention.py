@@ -147,6 +147,46 @@ def test_empty_rows_and_bad_indices_are_reported_not_trapped():
         U.check_attn_vs_oracle(w, *bits, rp, ci, o, lse, [0, 4, 6, 15])
 
 
+@pytest.mark.parametrize("block", [128, 64])
+def test_corrupt_row_ptr_is_reported_and_no_entry_outside_the_csr_is_read(block):
+    """row_ptr pairs that are not monotone, longer than Nb, or that point far beyond the CSR's row_ptr[R]
+    entries: the flag is set, the rows that own a bad pair come out empty (zeros, lse = -inf; with 64-token
+    blocks the query block that shares the tile too), no col_idx entry at or beyond row_ptr[R] is read (the
+    kernels bound every pair by it), and every other row is still right."""
+    w = shrink(WORKLOADS["medium"], H=2, T=2, k=3, block=block)
+    data, bits, rp, ci = _setup(w)
+    rp_h = rp.cpu().clone()
+    nnz, Nb = int(rp_h[-1]), w.Nb
+    r0 = 5
+    cases = {
+        "not monotone": lambda x: x.__setitem__(r0 + 1, int(x[r0]) - 2),
+        "longer than Nb": lambda x: x.__setitem__(r0 + 1, int(x[r0]) + Nb + 3),
+        "far beyond the CSR": lambda x: (x.__setitem__(r0, 1 << 30), x.__setitem__(r0 + 1, (1 << 30) + 2)),
+        "negative": lambda x: x.__setitem__(r0, -4),
+    }
+    for name, corrupt in cases.items():
+        rp2 = rp_h.clone(); corrupt(rp2)
+        d = torch.diff(rp2)
+        bad = [r for r in range(w.R) if rp2[r] < 0 or d[r] < 0 or d[r] > Nb or rp2[r + 1] > nnz]
+        assert bad, name
+        touched = set()
+        for r in range(w.R):                       # rows whose pair differs from the intact CSR
+            if rp2[r] != rp_h[r] or rp2[r + 1] != rp_h[r + 1]:
+                touched.add(r)
+                if block == 64:
+                    touched.add(r ^ 1)             # the other query block of its tile row
+        for simt in (False, True):
+            o, lse, st = U.gpu_attn(w, *data, rp2.cuda(), ci, simt=simt)
+            assert st & B.SVA_DEV_BAD_INDEX, (name, simt)
+            assert not (st & B.SVA_DEV_TIMEOUT)
+            for r in bad:
+                bh, I = divmod(r, Nb)
+                sl = (bh // w.H, bh % w.H, slice(I * block, min((I + 1) * block, w.N)))
+                assert (o[sl] == 0).all() and torch.isinf(lse[sl]).all(), (name, simt, r)
+            rows = [r for r in range(w.R) if r not in touched]
+            U.check_attn_vs_oracle(w, *bits, rp_h, ci, o, lse, rows[:6] + rows[-6:])
+
+
 def test_block64_tile_with_one_empty_query_block():
     """64-token blocks: a tile row whose two query blocks keep different key blocks, down to one of them
     keeping nothing, against the CUDA-core kernel and the oracle."""

@@ -22,8 +22,10 @@ def test_one_rank_group_matches_the_direct_path_and_the_oracle():
         (q, k, v), (qb, kb, vb) = U.host_inputs(w)
         qd, kd, vd = (U.dev(x)[:, :, :w.N].contiguous() for x in (q, k, v))
         sel = B.make_select(w.mode, w.k, w.tau)
-        o = SP.sequence_parallel_attention(qd, kd, vd, SP.even_shards(w.N, 1), SP.sparse_attend(sel, w.block))
+        attend = SP.sparse_attend(sel, w.block)
+        o = SP.sequence_parallel_attention(qd, kd, vd, SP.even_shards(w.N, 1), attend)
         torch.cuda.synchronize()
+        assert int(attend.status.item()) == 0                 # what the kernels reported is not dropped
         rp, ci, _ = U.gpu_select(w, U.dev(q), U.dev(k))
         o_direct, _, st = U.gpu_attn(w, U.dev(q), U.dev(k), U.dev(v), rp, ci)
         assert st == 0 and torch.equal(o, o_direct[:, :, :w.N])

@@ -2,7 +2,7 @@
 
 Some users of this library run where cudaMalloc is not theirs to call (a plugin that only
 gets input and output buffers, a step inside a region that must not touch the allocator), so
-sva_block_select_noalloc takes its scratch from an 8 MiB device array built into the library.
+sva_block_select_noalloc takes its scratch from a 16 MiB device array built into the library.
 It runs the same kernels as sva_block_select, so its CSR and scores must be identical -- on a
 first call and again on a second call that finds the previous call's bytes in the scratch.
 This file sorts last on purpose: a run that stops at the first failure has then already run
