@@ -268,3 +268,6 @@ def qk_norm_rope(x: np.ndarray, g: np.ndarray, cos: np.ndarray, sin: np.ndarray,
             out[b, h, :N, 0::2] = ue * cos - uo * sin
             out[b, h, :N, 1::2] = uo * cos + ue * sin
     return out
+
+
+from .remainder import attn_remainder_rows, block_stats, merge as merge_lse, remainder_rows  # noqa: E402,F401

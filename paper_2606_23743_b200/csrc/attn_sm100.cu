@@ -51,6 +51,21 @@
 
 #include "tc_ptx.cuh"
 
+// Timeline stamps for tuning builds only (-DSVA_TIMELINE; never in the shipped library): CTA 0 appends
+// {cycle << 20 | role << 16 | row << 12 | tile << 4 | event} to prof[512..] for its rows 2..4.
+#ifdef SVA_TIMELINE
+#define SVA_STAMP(role, row, j, ev)                                                                       \
+  do {                                                                                                    \
+    if (blockIdx.x == 0 && (row) >= 2 && (row) <= 4 && stamp_n < 800u) {                                  \
+      stamp_buf[(role) * 800 + stamp_n++] = ((unsigned long long)(unsigned)clock() << 20) |               \
+          ((unsigned long long)(role) << 16) | ((unsigned long long)((row) & 15) << 12) |                 \
+          ((unsigned long long)((j) & 255) << 4) | (unsigned long long)(ev);                              \
+    }                                                                                                     \
+  } while (0)
+#else
+#define SVA_STAMP(role, row, j, ev) do { } while (0)
+#endif
+
 namespace sva {
 
 struct TsParams {
@@ -89,7 +104,11 @@ constexpr int OFF_V = OFF_K + KS * TILE;
 constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][128 B] panels (one per softmax group)
 constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
 constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers, reference exponents, row sums (two rows), row queue
+#ifdef SVA_TIMELINE
+constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024 + 3200 * 8;
+#else
 constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;      // + alignment slack
+#endif
 constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
 // The reference exponent of a row is raised only when a block's maximum exceeds it by more than this
 // many powers of two.  P then reaches at most 2^32 and a row sum 2^32 * N: far inside fp32 (and bf16
@@ -171,6 +190,12 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   // ---------------------------------------------------------------- set-up
   const long long t_cta0 = prm.prof ? clock64() : 0;
+#ifdef SVA_TIMELINE
+  uint32_t stamp_n = 0;
+  unsigned long long* stamp_buf = reinterpret_cast<unsigned long long*>(smem + OFF_CTRL + CTRL_BYTES);   // 3200 entries
+  if (blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 3200; i_ += THREADS) stamp_buf[i_] = 0ull;
+  __syncthreads();
+#endif
   if (threadIdx.x == 0) {
     mbar_init(bar_q_ready, 256);
     mbar_init(bar_o_free, 256);
@@ -356,8 +381,10 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               ok = mbar_wait(bar_s_free + 8 * w, (cs[w] - 1u) & 1u, abort_flag, prm.status);
               if (!ok) break;
             }
+            SVA_STAMP(2, i, j, 0);
             ok = mbar_wait(bar_k_full + 8 * s, ph, abort_flag, prm.status);
             if (!ok) break;
+            SVA_STAMP(2, i, j, 1);
             tc_fence_after();
             const uint64_t kd = kd0 + (uint64_t)(s * (TILE >> 4));
             if (F8) {
@@ -373,6 +400,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               }
             }
             tc_commit(bar_k_empty + 8 * s, 1u);
+            SVA_STAMP(2, i, j, 2);
             tc_commit(bar_s_full + 8 * w, 1u);
             ++cs[w];
             if (++s == KS) { s = 0; ph ^= 1u; }
@@ -396,15 +424,18 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
             const uint64_t vd = vd0 + (uint64_t)(s * (TILE >> 4));
-            ok = mbar_wait(bar_p_full + 8 * w, cp[w] & 1u, abort_flag, prm.status) &&
-                 mbar_wait(bar_v_full + 8 * s, ph, abort_flag, prm.status);
+            ok = mbar_wait(bar_p_full + 8 * w, cp[w] & 1u, abort_flag, prm.status);
+            SVA_STAMP(3, i, j, 0);
+            ok = ok && mbar_wait(bar_v_full + 8 * s, ph, abort_flag, prm.status);
             if (!ok) break;
+            SVA_STAMP(3, i, j, 1);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < BS / 16; ++kk) {
               const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
               tc_mma_ts(tmem_base + COL_O, tmem_base + COL_P + 8 * kk, vd + off, IDESC, (j > 0 || kk > 0) ? 1u : 0u, 1u);
             }
+            SVA_STAMP(3, i, j, 2);
             tc_commit(bar_v_empty + 8 * s, 1u);
             tc_commit(bar_pv_done + 8 * w, 1u);
             if (!ok) break;
@@ -513,7 +544,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           J = list_block<B64>(prm, lbeg, j + 2);
           if (F8) load_ks(J);
         }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 0);
         if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 1);
         tc_fence_after();
         if (B64 ? (v0 + v1 < BS) : (v0 < BS)) {
           // Keys that do not exist (ragged last key block) become -inf in TMEM before S is read: a short
@@ -542,6 +575,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 2);
         float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
         float mx0, mx1;
         if (B64) {                                           // a, b: keys 0..63; c, d: keys 64..127
@@ -574,6 +608,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (!mbar_wait(bar_ref + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
           m_prev = ref[(w ^ 1) * 128 + row];
         }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 3);
         // lazy rule: raise the reference only when the row maximum outgrows it by more than 2^LAZY_LOG2
         const float m_new = (mx > m_prev + LAZY_LOG2) ? mx : m_prev;
         ref[w * 128 + row] = m_new;
@@ -623,18 +658,22 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           unpack2(sum2, sum_a, sum_b);
           l += sum_a + sum_b;
         }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 4);
         // the P columns are free once P V(j-1) has completed (block 0: the previous row's last P V
         // was waited for in that row's epilogue)
         if (j > 0 && !pv_waited &&
             !mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 5);
         tc_fence_after();
         tmem_st32(p_tmem, sv);
         tmem_st32(p_tmem + 32, sv + 32);
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p_full + 8 * w);
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 6);
       }
       if (!ok) break;
+      if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 7);
       // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
       // normalise and store (each group half of d)
       if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
@@ -651,7 +690,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
       // both groups have seen all their S tiles: no MMA reads Q any more
       if (r_next < prm.R) store_q(qn);
+      if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
       if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+      if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 9);
       tc_fence_after();
       const float lt = l + lxr[(w ^ 1) * 128 + row];
       // (64-token blocks: a query block with an empty list beside one with work has lt = 0 -> zeros, lse = -inf)
@@ -686,6 +727,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         if (qi < prm.N && prm.lse && w == 0) prm.lse[(long long)bh * prm.N + qi] = (m_fin + log2f(lt)) * 0.6931471805599453f;
       }
+      if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 10);
       cnt[0] += (uint32_t)((n + 1) >> 1);
       cnt[1] += (uint32_t)(n >> 1);
     }
@@ -695,6 +737,10 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // ---------------------------------------------------------------- tear-down
   if (prm.prof && threadIdx.x == 0)
     atomicMax(reinterpret_cast<unsigned long long*>(prm.prof + 319), (unsigned long long)(clock64() - t_cta0));
+#ifdef SVA_TIMELINE
+  __syncthreads();
+  if (prm.prof && blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 3200; i_ += THREADS) prm.prof[512 + i_] = (long long)stamp_buf[i_];
+#endif
   if (*abort_flag) {
     // give copies and MMAs still in flight time to land before shared memory and TMEM go away
     const long long t0 = clock64();
