@@ -209,6 +209,32 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Piecewise attention: exact over the kept blocks, approximate remainder for the dropped ones (the paper's
+ * sparse-attention section: non-critical blocks "compensated with first-order Taylor approximation"; its
+ * LTX-2.3 pipeline runs with the "approximate remainder enabled").  The paper prints no formula; this is the
+ * expansion of exp(scale <q_i, k_j>) about the mean key of each dropped block J (n_J keys, mean key kbar_J,
+ * mean value vbar_J; a_iJ = scale <q_i, kbar_J>):
+ *     Z_i = sum_{j kept} exp(s_ij)     + sum_{J dropped} n_J exp(a_iJ)              (the first-order term cancels)
+ *     N_i = sum_{j kept} exp(s_ij) v_j + sum_{J dropped} n_J exp(a_iJ) vbar_J  [+ the first-order term]
+ *     o_i = N_i / Z_i,   lse_i = ln Z_i            (exact part and remainder share one online softmax)
+ * order 0 stops there: a dropped block acts as n_J copies of its mean key carrying its mean value.  On the
+ * device the dropped blocks cost ceil(Nb/128) extra tiles per query block, whose "keys" and "values" are the
+ * bf16-rounded block means (written into the workspace by this call), the kept blocks masked out.
+ * order 1 adds scale * exp(sbar_IJ) * C_J^T q_i per dropped block, C_J = sum_j (k_j - kbar_J) v_j^T weighted at
+ * the query block's mean query so that the dropped blocks collapse into one d x d matrix per query block: not
+ * built on the device yet (SVA_ERR_UNSUPPORTED).
+ * Supported: bf16 Q/K, d = 128, 128- or 64-token blocks; otherwise SVA_ERR_UNSUPPORTED.  A query block that
+ * drops nothing gets exactly the result of sva_block_sparse_attn_fwd.  workspace: >=
+ * sva_attn_remainder_workspace_bytes(p), 256-byte aligned, rewritten by every call.  Everything else as for
+ * sva_block_sparse_attn_fwd.
+ */
+size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p);
+int sva_block_sparse_attn_remainder_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                                        const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                        int32_t* device_status, int32_t order, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+
 /* The dense fallback: every block kept, no CSR read. */
 int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                        const float* q_scale, const float* k_scale, void* o, float* lse,

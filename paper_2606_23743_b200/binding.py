@@ -23,7 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
-    "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
+    "sva_attn_remainder_workspace_bytes", "sva_block_sparse_attn_remainder_fwd", "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
 ]
 DEBUG_EXPORTS = ["sva_debug_set_prof_buffer", "sva_debug_set_mode", "sva_debug_set_wait_limit"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -76,6 +76,11 @@ def lib():
         L.sva_block_sparse_attn_fwd_simt.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.sva_dense_attn_fwd.restype = C.c_int
         L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_attn_remainder_workspace_bytes.restype = C.c_size_t
+        L.sva_attn_remainder_workspace_bytes.argtypes = [C.POINTER(Problem)]
+        L.sva_block_sparse_attn_remainder_fwd.restype = C.c_int
+        L.sva_block_sparse_attn_remainder_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp,
+                                                          C.c_size_t, vp]
         L.sva_attn_prepare_v.restype = C.c_int
         L.sva_attn_prepare_v.argtypes = [C.POINTER(Problem), vp, vp, C.c_size_t, vp]
         L.sva_block_sparse_attn_fwd_prepared.restype = C.c_int
@@ -307,3 +312,17 @@ def debug_set_wait_limit(cycles: int) -> None:
     """SM cycles a device-side wait may last before its CTA gives up; <= 0 restores the default."""
     if lib().sva_debug_set_wait_limit(C.c_longlong(int(cycles))) != 0:
         raise RuntimeError("sva_debug_set_wait_limit failed")
+
+
+def attn_remainder_workspace_bytes(p: Problem) -> int:
+    return int(lib().sva_attn_remainder_workspace_bytes(C.byref(p)))
+
+
+def block_sparse_attn_remainder_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, order: int = 0,
+                                    workspace=None) -> None:
+    """Exact attention over the kept blocks plus the approximate remainder of the dropped ones (order 0)."""
+    rc = lib().sva_block_sparse_attn_remainder_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(row_ptr), _ptr(col_idx),
+                                                   _ptr(o), _ptr(lse), _ptr(status), int(order), _ptr(workspace),
+                                                   _ws_bytes(workspace), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_sparse_attn_remainder_fwd")

@@ -193,6 +193,25 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
                           (cudaStream_t)stream);
 }
 
+size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p) {
+  if (validate_problem(p)) return 0;
+  return attn_ts_remainder_workspace_bytes(make_dims(p));
+}
+
+int sva_block_sparse_attn_remainder_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
+                                        const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                        int32_t* device_status, int32_t order, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
+  int rc = validate_attn(p, q, k, v, nullptr, nullptr, o);
+  if (rc) return rc;
+  if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
+  if (order != 0 && order != 1) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  if (!attn_ts_remainder_serves(m) || order != 0) return SVA_ERR_UNSUPPORTED;
+  return launch_attn_ts(m, p, q, k, v, nullptr, nullptr, row_ptr, col_idx, o, lse, device_status, workspace,
+                        workspace_bytes, (cudaStream_t)stream, order);
+}
+
 int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                        const float* q_scale, const float* k_scale, void* o, float* lse,
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream) {

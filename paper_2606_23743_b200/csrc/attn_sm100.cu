@@ -87,6 +87,11 @@ struct TsParams {
   const uint32_t* tile_desc;  // two 16-bit halves {key block (14 bits), kept by query block A, kept by B}
   float scale_log2;           // softmax_scale * log2(e)
   int32_t* next_row;          // two device counters (both start at 0): the next row to hand out, CTAs done drawing
+  // approximate remainder (REM kernels): every row's list is followed by np tiles whose "keys" are the
+  // block means of K (and whose "values" the block means of V), 128 blocks per tile
+  int np;                     // pooled tiles per head = ceil(Nb / 128); 0 = no remainder
+  float log2_block;           // log2(tokens per block): a block mean stands for that many keys
+  float tail_bias;            // (log2(keys of the last block) - log2_block) / scale_log2: added to the last block's pooled logit
   long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
   int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
                               // bit4: starve the pipeline so that a wait runs out (test aid)
@@ -128,24 +133,33 @@ constexpr float LAZY_LOG2 = 32.0f;
 // so no col_idx entry outside [0, row_ptr[R]) is ever read.  64-token blocks: the tile row's list of
 // 128-key tiles that pair_lists_kernel built (and checked) from the two CSR rows of the tile.
 // Only the K producer calls this; the other roles take its answer from the row queue.
-template <bool B64>
+// (REM: the count includes the np pooled tiles that follow the row's own entries.)
+template <bool B64, bool REM = false>
 __device__ __forceinline__ bool row_list(const TsParams& prm, int r, int nnz_bound, int& n, int& beg) {
   if (B64) {
     if (prm.row_ptr == nullptr) { n = (prm.Nb + 1) >> 1; beg = 0; return true; }     // dense: every pair of key blocks
-    n = __ldg(prm.tile_cnt + r); beg = __ldg(prm.tile_beg + r);
+    n = __ldg(prm.tile_cnt + r) + (REM ? prm.np : 0); beg = __ldg(prm.tile_beg + r);
     return true;
   }
   if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return true; }
   beg = __ldg(prm.row_ptr + r);
   const int end = __ldg(prm.row_ptr + r + 1);
   n = end - beg;
-  if (beg < 0 || end < beg || n > prm.Nb || end > nnz_bound) { n = 0; beg = 0; return false; }
+  if (beg < 0 || end < beg || n > prm.Nb || end > nnz_bound) { n = REM ? prm.np : 0; beg = 0; return false; }
+  if (REM) n += prm.np;
   return true;
+}
+// Pooled tiles (REM) are marked in their list entry: bit 31 (128-token blocks) resp. an upper half of
+// 0xffff (64-token blocks: block index 0x3fff cannot occur, Nb <= 16383); the low 16 bits are the chunk.
+template <bool B64>
+__device__ __forceinline__ bool entry_is_pooled(uint32_t e) {
+  return B64 ? (e >> 16) == 0xffffu : (e >> 31) != 0u;
 }
 // Entry j of a work list.  128-token blocks: the key block (an out-of-range entry is replaced by block 0;
 // the producer reports it).  64-token blocks: the tile descriptor.
-template <bool B64>
-__device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j) {
+template <bool B64, bool REM = false>
+__device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j, int n_own = 0) {
+  if (REM && j >= n_own) return (B64 ? 0xffff0000u : 0x80000000u) | (uint32_t)(j - n_own);
   if (B64) {
     if (prm.row_ptr == nullptr) {        // dense: key blocks 2j and 2j+1 (if it exists), kept by both query blocks
       const uint32_t u0 = 2u * (uint32_t)j, u1 = u0 + 1u;
@@ -164,10 +178,11 @@ __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int
 // zero-fills it if its list is empty, and otherwise publishes {row, count, start, first two entries}
 // in a small shared-memory queue that every other role reads in the same order.  All barriers keep running across rows, so the producers and the S
 // issuer run ahead into the next row while the softmax groups finish the current one.
-template <bool B64, bool F8>
+template <bool B64, bool F8, bool REM>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
-               const __grid_constant__ CUtensorMap tm_o, const TsParams prm) {
+               const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_kp,
+               const __grid_constant__ CUtensorMap tm_vtp, const TsParams prm) {
   using namespace ts;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -222,8 +237,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 8 && lane == 0) prefetch_tmap(&tm_k);
-  if (warp == 11 && lane == 0) prefetch_tmap(&tm_vt);
+  if (warp == 8 && lane == 0) { prefetch_tmap(&tm_k); if (REM) prefetch_tmap(&tm_kp); }
+  if (warp == 11 && lane == 0) { prefetch_tmap(&tm_vt); if (REM) prefetch_tmap(&tm_vtp); }
   if (warp == 0 && lane == 0) prefetch_tmap(&tm_o);
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -271,7 +286,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (;;) {
             r = atomicAdd(prm.next_row, 1);
             if (r >= prm.R) break;
-            if (!row_list<B64>(prm, r, nnz_bound, n, beg) && prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX);
+            if (!row_list<B64, REM>(prm, r, nnz_bound, n, beg) && prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX);
             if (n > 0) break;
             // nothing kept (or a corrupt row_ptr pair): zeros and lse = -inf; rare, so this one lane does it
             const int I = r % Nb, bh0 = r / Nb;
@@ -285,7 +300,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
           }
           uint32_t e0 = 0u, e1 = 0u;
-          if (r < prm.R) { e0 = list_block<B64>(prm, beg, 0); if (n > 1) e1 = list_block<B64>(prm, beg, 1); }
+          const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);        // entries of the row's own list
+          if (r < prm.R) { e0 = list_block<B64, REM>(prm, beg, 0, n_own); if (n > 1) e1 = list_block<B64, REM>(prm, beg, 1, n_own); }
           rowq[8 * slot] = r;
           rowq[8 * slot + 1] = n;
           rowq[8 * slot + 2] = beg;
@@ -308,10 +324,15 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
             const uint32_t dst = sbase + OFF_K + s * TILE;
             mbar_expect_tx(bar_k_full + 8 * s, KTILE);
-            if (B64) {
+            if (REM && j >= n_own) {
+              // pooled tile: 128 block means of K (rows beyond Nb are zero in the pooled tensor)
+              const int c = j - n_own;
+              tma_load_4d(dst, &tm_kp, bar_k_full + 8 * s, 0, c * BS, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_kp, bar_k_full + 8 * s, 64, c * BS, hh, bb);
+            } else if (B64) {
               // two 64-key blocks side by side: rows 0..63 and 64..127 of both d-panels
               // (e4m3: one 128-byte panel, so one load per key block)
-              const uint32_t dsc = list_block<B64>(prm, beg, j);
+              const uint32_t dsc = list_block<B64>(prm, beg, j);      // (an own entry: j < n_own)
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
                 const int J = (int)((dsc >> (16 * h)) & 0x3fffu);
@@ -343,12 +364,18 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           uint32_t e0, e1;
           if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);
           for (int j = 0; j < n; ++j) {
             if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-            const uint32_t e = list_block<B64>(prm, beg, j);
+            const uint32_t e = list_block<B64, REM>(prm, beg, j, n_own);
             const uint32_t dst = sbase + OFF_V + s * TILE;
             mbar_expect_tx(bar_v_full + 8 * s, TILE);
-            if (B64) {
+            if (REM && j >= n_own) {
+              // pooled tile: the block means of V, transposed ([128 d rows][128 blocks]; blocks beyond Nb zero)
+              const int c = j - n_own;
+              tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
+              tma_load_4d(dst + TILE / 2, &tm_vtp, bar_v_full + 8 * s, 64, c * BS, hh, bb);
+            } else if (B64) {
               // each 64-key panel of the tile is one key block's transposed V: [128 d rows][64 keys]
               tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)(e & 0x3fffu) * D, hh, bb);
               tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 0, (int)((e >> 16) & 0x3fffu) * D, hh, bb);
@@ -456,6 +483,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t p_tmem = tmem_base + lane_addr + COL_P;
     const uint32_t q_tmem = tmem_base + lane_addr + COL_Q + (F8 ? 16 : 32) * w;
     const int tail_keys = prm.N - (prm.Nb - 1) * KB;         // valid keys of the last key block
+    const int nnz_total = (REM && prm.row_ptr) ? __ldg(prm.row_ptr + (prm.R / prm.Nt) * prm.Nb) : 0;   // row_ptr[R of the CSR]
     const int qh = row >> 6;                                 // 64-token blocks: which query block of the tile I am in
     float c = prm.scale_log2;      // e4m3 variant: times the scales of the query block and of the key block, per block
     float c1 = prm.scale_log2;     // e4m3 with 64-token blocks: the same for the tile's second key block
@@ -525,13 +553,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + qb) * prm.scale_log2;
         if (w < n) load_ks(J);
       }
+      const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);      // entries of the row's own list
       for (int j = w; j < n; j += 2) {
         const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
         const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
         // valid keys of the tile's two 64-key halves (64-token blocks: a half whose key block this
         // thread's query block does not keep counts as 0; uniform over a warp)
         int v0, v1;
-        if (B64) {
+        const bool pooled = REM && entry_is_pooled<B64>(J);          // a tile of block means (the remainder)
+        const int pc = (int)(J & 0xffffu);                            // ... and which 128 blocks it holds
+        if (pooled) {
+          const int vn = min(BS, prm.Nb - BS * pc);                   // blocks that exist in this tile
+          v0 = B64 ? min(64, vn) : vn;
+          v1 = B64 ? max(vn - 64, 0) : 0;
+        } else if (B64) {
           const int u0 = (int)(J & 0x3fffu), u1 = (int)((J >> 16) & 0x3fffu);
           v0 = ((J >> (14 + qh)) & 1u) ? (u0 == prm.Nb - 1 ? tail_keys : 64) : 0;
           v1 = ((J >> (30 + qh)) & 1u) ? (u1 == prm.Nb - 1 ? tail_keys : 64) : 0;
@@ -541,7 +576,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         if (F8) { c = qs_row * ks_next; if (B64) c1 = qs_row * ks_next1; }
         if (j + 2 < n) {                                               // one entry ahead
-          J = list_block<B64>(prm, lbeg, j + 2);
+          J = list_block<B64, REM>(prm, lbeg, j + 2, n_own);
           if (F8) load_ks(J);
         }
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 0);
@@ -564,6 +599,27 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           } else {
 #pragma unroll 1
             for (int e = v0; e < BS; ++e) tmem_st1(s_tmem + e, 0xff800000u);
+          }
+          tc_wait_st();
+        }
+        if (REM && pooled) {
+          // The remainder stands for the DROPPED blocks only: the blocks this thread's query block keeps become
+          // -inf (one warp-wide TMEM store each; the row's CSR entries are the same for a whole warp), and the
+          // ragged last block's mean stands for fewer keys than the others.
+          const int rq = B64 ? bh * prm.Nb + min(2 * I + qh, prm.Nb - 1) : r;      // my query block's CSR row
+          int cb = __ldg(prm.row_ptr + rq), ce = __ldg(prm.row_ptr + rq + 1);
+          if (cb < 0 || ce < cb || ce - cb > prm.Nb || ce > nnz_total) ce = cb;      // corrupt pair (reported elsewhere)
+#pragma unroll 1
+          for (int t = cb; t < ce; ++t) {
+            const int Jk = __ldg(prm.col_idx + t);
+            if (Jk >= 0 && Jk < prm.Nb && (Jk >> 7) == pc) tmem_st1(s_tmem + (Jk & 127), 0xff800000u);
+          }
+          if (tail_keys < KB && ((prm.Nb - 1) >> 7) == pc) {
+            tc_wait_st();
+            const uint32_t col = s_tmem + ((prm.Nb - 1) & 127);
+            const float x = __uint_as_float(tmem_ld1(col));
+            tc_wait_ld();
+            tmem_st1(col, __float_as_uint(x + prm.tail_bias));          // (-inf stays -inf)
           }
           tc_wait_st();
         }
@@ -600,8 +656,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           mx1 = fmaxf(mxc, mxd);
         }
         // (e4m3 with 64-token blocks: each half has its own scale; a half that is not kept stays -inf)
+        // (a pooled logit carries + log2(keys per block): a block mean stands for that many keys)
         const float mx = (B64 && F8) ? fmaxf(v0 > 0 ? mx0 * c : -INFINITY, v1 > 0 ? mx1 * c1 : -INFINITY)
-                                     : fmaxf(mx0, mx1) * c;
+                                     : fmaxf(mx0, mx1) * c + ((REM && pooled) ? prm.log2_block : 0.f);
         // reference exponent left by block j-1 (other group)
         float m_prev = -INFINITY;
         if (j > 0) {
@@ -636,6 +693,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // (64-token blocks: -inf instead of -m for a half that is not kept, or while the row has seen no
         // kept key yet, makes those P exactly 0 at no cost)
         float nm = -m_new, nmh1 = -m_new;
+        if (REM && pooled) { nm += prm.log2_block; nmh1 = nm; }
         if (B64) {
           if (m_new == -INFINITY || v0 == 0) nm = -INFINITY;
           if (m_new == -INFINITY || v1 == 0) nmh1 = -INFINITY;
@@ -864,6 +922,45 @@ pair_lists_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict
   }
 }
 
+// ------------------------------------------------------------------ remainder: block means of K and V
+// One CTA per (block J, head, tensor): the mean over the existing tokens of the block, fp32 accumulation in a
+// fixed order, rounded to bf16.  K means go to kp [B*H][Nbp][128] (rows >= Nb stay zero: the launcher clears the
+// buffer), V means transposed to vtp [B*H][np][128 d][128 blocks], the layout of a V^T tile.
+__global__ void __launch_bounds__(256)
+pool_kv_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, Strides sk, Strides sv,
+               int H, int N, int block, int Nb, int Nbp, __nv_bfloat16* __restrict__ kp,
+               __nv_bfloat16* __restrict__ vtp) {
+  __shared__ float part[16][ts::D + 1];
+  const int J = blockIdx.x, bh = blockIdx.y, which = blockIdx.z;
+  const int b = bh / H, h = bh % H;
+  const Strides s = which ? sv : sk;
+  const __nv_bfloat16* base = (which ? v : k) + (long long)b * s.b + (long long)h * s.h;
+  const int lo = J * block, cnt = min(block, N - lo);
+  const int vec = threadIdx.x & 15, grp = threadIdx.x >> 4;          // 16 vectors of 8 elements per row, 16 rows at a time
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  for (int t = grp; t < cnt; t += 16) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(base + (long long)(lo + t) * s.n) + vec);
+    const uint32_t wd[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { acc[2 * e] += bf16lo(wd[e]); acc[2 * e + 1] += bf16hi(wd[e]); }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) part[grp][vec * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < ts::D) {
+    float sum = 0.f;
+#pragma unroll
+    for (int g = 0; g < 16; ++g) sum += part[g][threadIdx.x];
+    const __nv_bfloat16 mean = __float2bfloat16_rn(sum / (float)cnt);
+    if (which == 0)
+      kp[((long long)bh * Nbp + J) * ts::D + threadIdx.x] = mean;
+    else
+      vtp[(((long long)bh * (Nbp >> 7) + (J >> 7)) * ts::D + threadIdx.x) * BS + (J & 127)] = mean;
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -912,17 +1009,17 @@ static int g_debug_ts = 0;
 static constexpr int TS_MAX_DEVICES = 64;
 static std::mutex g_ts_mutex;
 static int g_ts_sms[TS_MAX_DEVICES];
-static bool g_ts_attr[TS_MAX_DEVICES][4];
+static bool g_ts_attr[TS_MAX_DEVICES][8];
 
-template <bool B64, bool F8>
+template <bool B64, bool F8, bool REM = false>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                     const TsParams& prm, cudaStream_t st) {
-  auto kern = attn_ts_kernel<B64, F8>;
+                     const CUtensorMap& tkp, const CUtensorMap& tvp, const TsParams& prm, cudaStream_t st) {
+  auto kern = attn_ts_kernel<B64, F8, REM>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
   {
     std::lock_guard<std::mutex> lock(g_ts_mutex);
-    constexpr int variant = (B64 ? 2 : 0) + (F8 ? 1 : 0);
+    constexpr int variant = (REM ? 4 : 0) + (B64 ? 2 : 0) + (F8 ? 1 : 0);
     if (!g_ts_attr[dev][variant]) {
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
         return SVA_ERR_CUDA;
@@ -934,7 +1031,7 @@ static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, con
     sms = g_ts_sms[dev];
   }
   const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
-  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, prm);
+  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, tkp, tvp, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
@@ -942,6 +1039,8 @@ static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, con
 // tile_beg[R2], tile_desc[cap] with R2 = B*H*ceil(Nb/2) tile rows and cap the bound for a dense CSR.
 struct TsLayout {
   size_t vt_bytes, counter_off, cnt_off, beg_off, desc_off, total;
+  size_t kp_off, vtp_off, pooled_bytes, total_rem;      // remainder: bf16 block means of K, and of V transposed
+  int np, Nbp;
   long long cap;
   int R2, Nt;
 };
@@ -960,11 +1059,23 @@ static TsLayout ts_layout(const Dims& m) {
     L.cap = ((long long)m.R * m.Nb + L.R2) / 2 + 2;
     L.total = L.desc_off + (((size_t)L.cap * 4 + 255) & ~(size_t)255);
   }
+  L.np = (m.Nb + BS - 1) / BS;
+  L.Nbp = L.np * BS;
+  L.pooled_bytes = (size_t)m.B * m.H * L.Nbp * ts::D * 2;
+  L.kp_off = L.total;
+  L.vtp_off = L.kp_off + L.pooled_bytes;
+  L.total_rem = L.vtp_off + L.pooled_bytes;
   return L;
 }
 
 bool attn_ts_serves(const Dims& m) {
   return (m.d == 128 || m.d == 64) && m.Nb <= 16383 && (m.block == BS || m.block == 64);
+}
+
+// The remainder variant: bf16 Q/K, d = 128, a CSR (the dense form drops nothing).
+bool attn_ts_remainder_serves(const Dims& m) { return attn_ts_serves(m) && m.d == ts::D && !m.fp8; }
+size_t attn_ts_remainder_workspace_bytes(const Dims& m) {
+  return attn_ts_remainder_serves(m) ? ts_layout(m).total_rem : 0;
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {
@@ -1000,11 +1111,18 @@ int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, vo
 }
 
 // v == nullptr: the workspace has been prepared by launch_prepare_v_ts (once per attention call).
+// remainder_order < 0: exact attention over the kept blocks only.  0: plus the block-mean remainder of the
+// dropped blocks (needs v, a CSR and the larger workspace of attn_ts_remainder_workspace_bytes).
 int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                   void* ws, size_t ws_bytes, cudaStream_t st) {
+                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order) {
   int rc = check_ts_workspace(m_in, ws, ws_bytes);
   if (rc) return rc;
+  const bool rem = remainder_order >= 0;
+  if (rem) {
+    if (remainder_order != 0 || !attn_ts_remainder_serves(m_in) || !row_ptr || !v) return SVA_ERR_UNSUPPORTED;
+    if (ws_bytes < attn_ts_remainder_workspace_bytes(m_in)) return SVA_ERR_WORKSPACE;
+  }
   // dense attention does not depend on the block size: 64-token blocks run as 128-token blocks
   Dims m = m_in;
   if (m.block == 64 && row_ptr == nullptr && !m.fp8) {     // (e4m3 scales are per 64-token block: that stays as it is)
@@ -1017,7 +1135,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
-  CUtensorMap tk, tv, to;
+  CUtensorMap tk, tv, to, tkp, tvp;
   if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2, BS)) != SVA_OK)
     return rc;
   const int eb = m.fp8 ? 1 : 2;
@@ -1029,6 +1147,22 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
                         vrows * m.block * 2 * m.H, BS)) != SVA_OK)
     return rc;
+  tkp = tk; tvp = tv;            // (placeholders when there is no remainder: the kernel never touches them)
+  if (rem) {
+    // block means of K ([Nbp rows][128], rows >= Nb zero) and of V (transposed tiles), then their maps
+    __nv_bfloat16* kp = reinterpret_cast<__nv_bfloat16*>(wsb + L.kp_off);
+    __nv_bfloat16* vtp = reinterpret_cast<__nv_bfloat16*>(wsb + L.vtp_off);
+    if (cudaMemsetAsync(kp, 0, 2 * L.pooled_bytes, st) != cudaSuccess) return SVA_ERR_CUDA;
+    pool_kv_kernel<<<dim3(m.Nb, m.B * m.H, 2), 256, 0, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, sk,
+                                                            make_strides(p->v_stride), m.H, m.N, m.block, m.Nb, L.Nbp, kp, vtp);
+    if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+    const cuuint64_t prow = (cuuint64_t)L.Nbp;
+    if ((rc = make_map_ts(&tkp, kp, ts::D, prow, m.H, m.B, (cuuint64_t)ts::D * 2, prow * ts::D * 2,
+                          prow * ts::D * 2 * m.H, BS)) != SVA_OK)
+      return rc;
+    if ((rc = make_map_ts(&tvp, vtp, BS, prow, m.H, m.B, (cuuint64_t)BS * 2, prow * BS * 2, prow * BS * 2 * m.H, BS)) != SVA_OK)
+      return rc;
+  }
   if (v) {
     // (the transposed copy is laid out for the block size of this launch)
     const Strides sv = make_strides(p->v_stride);
@@ -1051,6 +1185,12 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   prm.tile_desc = reinterpret_cast<const uint32_t*>(wsb + L.desc_off);
   prm.scale_log2 = m.scale * 1.4426950408889634f;
   prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
+  prm.np = rem ? L.np : 0;
+  prm.log2_block = log2f((float)m.block);
+  {
+    const int tail = m.N - (m.Nb - 1) * m.block;
+    prm.tail_bias = (log2f((float)tail) - prm.log2_block) / prm.scale_log2;
+  }
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
   if (b64) {
@@ -1060,10 +1200,13 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
           reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
       if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     }
-    return m.fp8 ? launch_ts<true, true>(L.R2, tk, tv, to, prm, st) : launch_ts<true, false>(L.R2, tk, tv, to, prm, st);
+    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+    return m.fp8 ? launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
+                 : launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
   }
-  if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, prm, st);
-  return launch_ts<false, false>(L.R2, tk, tv, to, prm, st);
+  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+  if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+  return launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }

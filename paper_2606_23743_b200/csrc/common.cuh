@@ -88,8 +88,10 @@ int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const
                      const int32_t* col_idx, void* o, float* lse, int32_t* status, cudaStream_t st);
 int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                   void* ws, size_t ws_bytes, cudaStream_t st);
+                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order = -1);
 size_t attn_ts_workspace_bytes(const Dims& m);
+size_t attn_ts_remainder_workspace_bytes(const Dims& m);
+bool attn_ts_remainder_serves(const Dims& m);
 bool attn_ts_serves(const Dims& m);    // d = 128 or 64, bf16 or e4m3 Q/K, 128- or 64-token blocks
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,
                         cudaStream_t st);

@@ -1,0 +1,109 @@
+"""Piecewise attention with the approximate remainder (order 0) through the C ABI against the oracle's
+remainder formula with bf16-rounded block statistics, the same CSR on both sides.  bf16 tolerances."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import _util as U
+from paper_2606_23743_b200 import binding as B
+from paper_2606_23743_b200.workloads import WORKLOADS, shrink
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_remainder(w, q, k, v, rp, ci, order=0, N=None):
+    N = w.N if N is None else N
+    o = torch.full(v.shape, 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((q.shape[0], q.shape[1], N), 7.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p = B.make_problem(q, k, v, o, N, w.block)
+    ws = torch.full((B.attn_remainder_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
+    B.block_sparse_attn_remainder_fwd(p, q, k, v, rp, ci, o, lse, status, order, ws)
+    torch.cuda.synchronize()
+    return o, lse, int(status.item())
+
+
+def check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows, order=0):
+    o_ref, l_ref = oracle.attn_remainder_rows(qb, kb, vb, w.N, w.block, w.scale, rp.cpu().numpy(), ci.cpu().numpy(),
+                                              rows, order=order, stats="bf16")
+    max_abs, rel, lse_err = U.attn_errors(o, lse, o_ref, l_ref, rows, w.N, w.block, o.shape[1])
+    assert max_abs <= U.BF16_MAX_ABS and rel <= U.BF16_REL_L2 and lse_err <= 2e-3, (max_abs, rel, lse_err)
+    return max_abs, rel, lse_err
+
+
+CASES = {
+    "medium_h2": shrink(WORKLOADS["medium"], H=2),                                   # Nb = 64: one pooled tile
+    "ragged_tail": shrink(WORKLOADS["medium"], H=3, T=2, Hg=30, Wg=31, k=5),         # N = 1860: last block of 68 keys
+    "two_pooled_tiles": shrink(WORKLOADS["large"], H=2, T=14, k=20),                 # Nb = 171 > 128
+    "mass_ragged_rows": shrink(WORKLOADS["large_ragged"], H=2, T=8),
+    "window": shrink(WORKLOADS["xl"], B=2, H=2, T=5),
+    "single_block": shrink(WORKLOADS["medium"], H=1, T=1, Hg=8, Wg=16, k=1),         # nothing dropped
+    "b64": shrink(WORKLOADS["medium"], H=2, T=2, block=64, k=8),
+    "b64_ragged_tail": shrink(WORKLOADS["medium"], H=3, T=2, Hg=30, Wg=31, block=64, k=7),   # 30 blocks, 4-key tail
+    "b64_odd_nb": shrink(WORKLOADS["medium"], H=2, T=1, Hg=30, Wg=30, block=64, k=4),        # 15 blocks
+    "b64_three_pooled_tiles": shrink(WORKLOADS["large_b64"], H=1, T=11, k=30),               # Nb = 269
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_remainder_matches_oracle(name):
+    w = CASES[name]
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w, qd, kd)
+    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci)
+    assert st == 0
+    rows = list(range(w.R)) if w.R <= 160 else U.sample_rows_per_head(w.B * w.H, w.Nb, 6, seed=1)
+    r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
+    print(f"{name}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
+    if w.n_alloc > w.N:
+        assert (o[:, :, w.N:] == 7.0).all()
+
+
+def test_rows_that_drop_nothing_equal_the_exact_call_and_empty_rows_are_all_remainder():
+    w = shrink(WORKLOADS["medium"], H=2, T=2, k=3)           # Nb = 16
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w, qd, kd)
+    rp_h, ci_h = rp.cpu(), ci.cpu()
+    kept = [ci_h[rp_h[r]:rp_h[r + 1]].tolist() for r in range(w.R)]
+    kept[2] = list(range(w.Nb))                              # keeps everything: no remainder
+    kept[5] = []                                             # keeps nothing: the remainder is the whole answer
+    kept[w.R - 1] = list(range(w.Nb))
+    rp2 = torch.zeros(w.R + 1, dtype=torch.int32); rp2[1:] = torch.cumsum(torch.tensor([len(x) for x in kept]), 0)
+    ci2 = torch.tensor([j for x in kept for j in x], dtype=torch.int32)
+    o, lse, st = gpu_remainder(w, qd, kd, vd, rp2.cuda(), ci2.cuda())
+    assert st == 0
+    check_vs_oracle(w, qb, kb, vb, rp2, ci2, o, lse, list(range(w.R)))
+    o_e, lse_e, _ = U.gpu_attn(w, qd, kd, vd, rp2.cuda(), ci2.cuda())
+    for r in (2, w.R - 1):
+        bh, I = divmod(r, w.Nb)
+        sl = (bh // w.H, bh % w.H, slice(I * w.block, min((I + 1) * w.block, w.N)))
+        assert torch.equal(o[sl], o_e[sl]) and torch.equal(lse[sl], lse_e[sl])
+
+
+def test_unsupported_forms_are_refused_on_the_host():
+    w = shrink(WORKLOADS["tiny"], H=2)                        # d = 64
+    (q, k, v), _ = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w, qd, kd)
+    p = B.make_problem(qd, kd, vd, torch.empty_like(vd), w.N, w.block)
+    assert B.attn_remainder_workspace_bytes(p) == 0
+    with pytest.raises(B.SvaError) as e:
+        B.block_sparse_attn_remainder_fwd(p, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 0,
+                                          torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 2
+    w2 = shrink(WORKLOADS["medium"], H=1, T=2)
+    (q, k, v), _ = U.host_inputs(w2)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w2, qd, kd)
+    p2 = B.make_problem(qd, kd, vd, torch.empty_like(vd), w2.N, w2.block)
+    ws = torch.empty(B.attn_remainder_workspace_bytes(p2), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SvaError) as e:                      # first-order term: not built on the device
+        B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 1, ws)
+    assert e.value.status == 2
+    with pytest.raises(B.SvaError) as e:                      # the exact call's workspace is too small
+        B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 0,
+                                          ws[: B.attn_workspace_bytes(p2)])
+    assert e.value.status == 3
