@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--workload", default="large", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--remainder", action="store_true",
+                    help="extended step: attention with the approximate remainder of the dropped blocks (order 0) "
+                         "instead of exact-only attention; `value` still counts the selected blocks' FLOPs only")
     ap.add_argument("--sustained-seconds", type=float, default=2.5,
                     help="length of the second, back-to-back leg whose clocks NVML can follow (0 = skip)")
     ap.add_argument("--prologue", action="store_true",
@@ -243,13 +246,18 @@ def main():
     row_ptr = torch.zeros(w.R + 1, dtype=torch.int32, device=dev)
     col_idx = torch.zeros(B.select_max_nnz(p, s), dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    aws = torch.empty(max(B.attn_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
+    if args.remainder and (w.fp8 or args.prologue):
+        raise SystemExit("--remainder runs on the plain bf16 step")
+    aws = torch.empty(max(B.attn_remainder_workspace_bytes(p) if args.remainder else B.attn_workspace_bytes(p), 256),
+                      dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
     # routing kernels (pooling, scores, selection; scan and compaction when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
     launches_per_step = (5 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
+    if args.remainder:      # + the block means of K and V (the memset before it is not a kernel of this library)
+        launches_per_step += 1
 
     # V is prepared (tiled transposed copy) on a second stream while routing, which never reads V, runs
     # (lower priority: its CTAs fill the SMs that the latency-bound selection kernel leaves idle instead of
@@ -267,7 +275,7 @@ def main():
             v_ready.record()
 
     # the two-step form serves what the tensor-core kernel serves (every supported shape today)
-    two_step = B.attn_workspace_bytes(p) > 0
+    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder     # (the remainder call prepares V itself)
 
     def route(qq, kk, vv):
         if args.prologue:
@@ -291,7 +299,9 @@ def main():
     def attend(qq, kk, vv, oo):
         if args.prologue:
             qq, kk = qn, kn
-        if w.fp8 and two_step:
+        if args.remainder:
+            B.block_sparse_attn_remainder_fwd(p, qq, kk, vv, row_ptr, col_idx, oo, None, status, 0, aws)
+        elif w.fp8 and two_step:
             torch.cuda.current_stream().wait_event(v_ready)
             B.block_sparse_attn_fwd_prepared(p, q8, k8, row_ptr, col_idx, oo, None, status, workspace=aws,
                                              q_scale=qs, k_scale=ks)
@@ -396,7 +406,7 @@ def main():
 
     # ---- attention with its V preparation in line (the one-call entry point: transpose, then the kernel)
     inline_ms = None
-    if two_step and not w.fp8 and not args.prologue:
+    if two_step and not w.fp8 and not args.prologue and not args.remainder:
         n_in = max(5, min(args.steps, 20))
         route(q, k, v)
         torch.cuda.current_stream().wait_event(v_ready)
@@ -474,6 +484,7 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
                    "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
                    "nnz_tiles": nnz, "parallelism": f"replicas x{world}", "prologue": bool(args.prologue),
+                   "remainder": "order 0: +%d pooled tiles per query-block row" % (-(-w.Nb // 128)) if args.remainder else None,
                    "l2": "inputs (%.0f MB) larger than L2; no flush" % (3 * sel_bytes / 2 / 1e6)},
         "tokens_per_s": world * w.B * w.N / (ms_per_step * 1e-3),
         "attention_ms": attn_ms, "select_ms": sel_ms,
@@ -504,7 +515,7 @@ def main():
         "clocks": clocks, "sustained": sustained, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline and not args.prologue:   # (the oracle leg times the plain step)
+        if world == 1 and not args.no_cpu_baseline and not args.prologue and not args.remainder:   # (the oracle leg times the plain step)
             import oracle
             oracle.build()
             line["cpu_baseline"] = cpu_baseline(w, bf16_bits(qh), bf16_bits(kh), bf16_bits(vh))

@@ -610,9 +610,14 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           int cb = __ldg(prm.row_ptr + rq), ce = __ldg(prm.row_ptr + rq + 1);
           if (cb < 0 || ce < cb || ce - cb > prm.Nb || ce > nnz_total) ce = cb;      // corrupt pair (reported elsewhere)
 #pragma unroll 1
-          for (int t = cb; t < ce; ++t) {
-            const int Jk = __ldg(prm.col_idx + t);
-            if (Jk >= 0 && Jk < prm.Nb && (Jk >> 7) == pc) tmem_st1(s_tmem + (Jk & 127), 0xff800000u);
+          for (int t0 = cb; t0 < ce; t0 += 32) {                       // 32 entries at a time, one per lane
+            const int Jl = t0 + lane < ce ? __ldg(prm.col_idx + t0 + lane) : -1;
+            uint32_t hit = __ballot_sync(0xffffffffu, Jl >= 0 && Jl < prm.Nb && (Jl >> 7) == pc);
+            while (hit) {
+              const int Jk = __shfl_sync(0xffffffffu, Jl, __ffs(hit) - 1);
+              hit &= hit - 1;
+              tmem_st1(s_tmem + (Jk & 127), 0xff800000u);
+            }
           }
           if (tail_keys < KB && ((prm.Nb - 1) >> 7) == pc) {
             tc_wait_st();

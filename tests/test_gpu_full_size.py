@@ -146,3 +146,22 @@ def test_full_size_prologue():
     torch.cuda.synchronize()
     rp2, ci2, _ = U.gpu_select(w, qo, ko)          # (bf16 routing: gpu_select takes the dtype from its fp8 argument)
     assert torch.equal(rp, rp2) and torch.equal(ci[: int(rp[-1])], ci2)
+
+
+@pytest.mark.parametrize("name", ["large", "large_b64"])
+def test_full_size_remainder(name):
+    """Piecewise attention with the order-0 remainder at full size in the launch configuration
+    `bench.py --remainder` times: per head, block 0, the ragged last block and 3 random ones against the oracle."""
+    from test_gpu_remainder import check_vs_oracle, gpu_remainder
+    w = WORKLOADS[name]
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, _ = U.gpu_select(w, qd, kd)
+    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci)
+    assert st == 0
+    rows = U.sample_rows_per_head(w.B * w.H, w.Nb, 3, seed=w.cfg)
+    r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
+    print(f"{name} + remainder: oracle sample {len(rows)} of {w.R} query blocks: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
+    assert torch.isfinite(o[:, :, :w.N].float()).all() and torch.isfinite(lse).all()
+    if w.n_alloc > w.N:
+        assert (o[:, :, w.N:] == 7.0).all()
