@@ -251,9 +251,9 @@ def main():
     aws = torch.empty(max(B.attn_remainder_workspace_bytes(p) if args.remainder else B.attn_workspace_bytes(p), 256),
                       dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
-    # routing kernels (pooling, scores, selection; scan and compaction when rows vary in length) + V transpose
+    # routing kernels (pooling, scores, selection; CSR assembly when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
-    launches_per_step = (5 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
+    launches_per_step = (4 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
     if args.remainder:      # + the block means of K and V (the memset before it is not a kernel of this library)

@@ -9,7 +9,7 @@
 // warp per query-block row: it reads the row's scores from that matrix (no shared memory), finds the
 // threshold of the rule by bisection on order-preserving integer keys and emits the kept blocks in
 // ascending order.  When the per-row count is known on the host (top-k with no window larger than k)
-// rows go straight into the CSR; otherwise they are staged and scan_kernel + compact_kernel build it.
+// rows go straight into the CSR; otherwise they are staged and csr_kernel builds it in one launch.
 #include <mutex>
 
 #include "common.cuh"
@@ -332,52 +332,44 @@ select_rows_kernel(const float* __restrict__ scores, SelParams p, int32_t* __res
   select_and_emit<ITEMS>(key, I, bh, lane, p, row_ptr, col_idx, tmp_idx, counts, R);
 }
 
-// Exclusive scan of counts[R] -> row_ptr[R+1]; one CTA, chunks of 1024 with a running carry.
-__global__ void __launch_bounds__(1024) scan_kernel(const int32_t* __restrict__ counts, int R,
-                                                     int32_t* __restrict__ row_ptr) {
+// CSR assembly for rows of varying length, one launch: a CTA owns 32 consecutive rows (one warp each).  It
+// first adds up the counts of all rows before its own (every thread a strided share, then a block
+// reduction: at most R counts = a few KB from the L2 per CTA, which is cheaper than a scan kernel of its
+// own plus its launch), then scans its 32 counts, writes row_ptr and copies the staged indices.
+static constexpr int CSR_ROWS = 32;
+__global__ void __launch_bounds__(CSR_ROWS * 32)
+csr_kernel(const int32_t* __restrict__ tmp_idx, const int32_t* __restrict__ counts, int cap, int R,
+           int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx) {
   __shared__ int warp_sum[32];
-  __shared__ int carry_s;
+  __shared__ int row_off[CSR_ROWS + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) carry_s = 0;
+  const int r0 = blockIdx.x * CSR_ROWS;
+  int part = 0;
+  for (int i = threadIdx.x; i < r0; i += CSR_ROWS * 32) part += __ldg(counts + i);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+  if (lane == 0) warp_sum[warp] = part;
   __syncthreads();
-  for (int base = 0; base < R; base += 1024) {
-    int i = base + threadIdx.x;
-    int v = i < R ? counts[i] : 0;
-    int x = v;
+  if (warp == 0) {
+    int base = warp_sum[lane];
+#pragma unroll
+    for (int o = 16; o; o >>= 1) base += __shfl_xor_sync(0xffffffffu, base, o);   // rows before this CTA
+    const int r = r0 + lane;
+    const int c = r < R ? __ldg(counts + r) : 0;
+    int incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= o) x += y;
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
     }
-    if (lane == 31) warp_sum[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      int w = warp_sum[lane];
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, w, o);
-        if (lane >= o) w += y;
-      }
-      warp_sum[lane] = w;
-    }
-    __syncthreads();
-    int incl = x + (warp ? warp_sum[warp - 1] : 0) + carry_s;
-    if (i < R) row_ptr[i] = incl - v;
-    __syncthreads();
-    if (threadIdx.x == 1023) carry_s = incl;
-    __syncthreads();
+    row_off[lane] = base + incl - c;
+    if (r < R) row_ptr[r] = base + incl - c;
+    if (r == R - 1) row_ptr[R] = base + incl;
   }
-  if (threadIdx.x == 0) row_ptr[R] = carry_s;
-}
-
-// One warp per row copies its staged indices to their CSR position.
-__global__ void compact_kernel(const int32_t* __restrict__ tmp_idx, const int32_t* __restrict__ counts,
-                               const int32_t* __restrict__ row_ptr, int cap, int R,
-                               int32_t* __restrict__ col_idx) {
-  int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  int lane = threadIdx.x & 31;
+  __syncthreads();
+  const int r = r0 + warp;
   if (r >= R) return;
-  int n = counts[r], dst = row_ptr[r];
+  const int n = __ldg(counts + r), dst = row_off[warp];
   for (int t = lane; t < n; t += 32) col_idx[dst + t] = tmp_idx[(long long)r * cap + t];
 }
 
@@ -470,8 +462,7 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   else SVA_SEL_LAUNCH(32);
 #undef SVA_SEL_LAUNCH
   if (!fixed_n) {
-    scan_kernel<<<1, 1024, 0, st>>>(counts, m.R, row_ptr);
-    compact_kernel<<<(m.R * 32 + 255) / 256, 256, 0, st>>>(tmp_idx, counts, row_ptr, cap, m.R, col_idx);
+    csr_kernel<<<(m.R + CSR_ROWS - 1) / CSR_ROWS, CSR_ROWS * 32, 0, st>>>(tmp_idx, counts, cap, m.R, row_ptr, col_idx);
   }
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
