@@ -282,6 +282,26 @@ int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* 
                         void* k8, float* q_scale, float* k_scale, void* stream);
 
 /*
+ * Block-scaled 4-bit quantiser for Q and K (NVFP4 is the paper's quantisation format -- its Quantization section
+ * and the per-model appendix paragraphs -- and the low-bit attention work it cites quantises Q K^T; the paper
+ * prints no formula).  As read here, every scalar step one fp32 operation rounded to nearest:
+ *   per (b,h)            g  = amax / (6 * 448) over the existing tokens (1 if amax = 0)
+ *   per token, 16 elems  sf = e4m3((amax_block / 6) / g), round-to-nearest-even, saturating at 448
+ *   per element          code = e2m1(x / (value(sf) * g)), round-to-nearest-even, saturating at +-6
+ *                        (e2m1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6; code = sign << 3 | index; all 0 where sf = 0)
+ *   x ~= value(code) * value(sf) * g
+ * Outputs (device, 16-byte aligned), in the layout the block-scaled tensor-core MMA takes:
+ *   q4, k4     : [B*H][Nb*128 tokens][64] bytes, two codes per byte (even element in the low nibble), rows >= N zero
+ *   q_sf, k_sf : [B*H][Nb][2][32][4][4] bytes: for 128-token block I and half c of the head dimension, the scale of
+ *                token t (within the block) and scale block kb (within the half) is byte (t%32)*16 + (t/32)*4 + kb
+ *   q_g, k_g   : [B*H] fp32
+ * d = 128 and block = 128 only (SVA_ERR_UNSUPPORTED otherwise).  workspace: >= 8*B*H bytes, 16-byte aligned.
+ */
+int sva_quantize_qk_fp4(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q4, void* k4,
+                        void* q_sf, void* k_sf, float* q_g, float* k_g, void* workspace, size_t workspace_bytes,
+                        void* stream);
+
+/*
  * The same quantiser with K smoothing, the step the 8-bit attention work cited in the paper's related
  * work on quantised attention puts before the cast: per (b,h) the mean key over the N tokens,
  *   k_mean[b,h,:] = (1/N) sum_j k[b,h,j,:]        (fp32; per-block sums in a fixed order, then the blocks in

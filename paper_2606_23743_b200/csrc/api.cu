@@ -276,6 +276,23 @@ int sva_quantize_qk_fp8(const sva_problem_t* p, const void* q_bf16, const void* 
   return launch_quantize(m, p, q_bf16, k_bf16, q8, k8, q_scale, k_scale, nullptr, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+int sva_quantize_qk_fp4(const sva_problem_t* p, const void* q_bf16, const void* k_bf16, void* q4, void* k4,
+                        void* q_sf, void* k_sf, float* q_g, float* k_g, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q_bf16 || !k_bf16 || !q4 || !k4 || !q_sf || !k_sf || !q_g || !k_g) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q_bf16) || !aligned16(k_bf16) || !aligned16(q4) || !aligned16(k4) || !aligned16(q_sf) || !aligned16(k_sf))
+    return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->q_stride, 16))) return rc;
+  if ((rc = check_strides(p->k_stride, 16))) return rc;
+  Dims m = make_dims(p);
+  if (m.d != 128 || m.block != 128) return SVA_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < (size_t)8 * m.B * m.H) return SVA_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return SVA_ERR_ALIGNMENT;
+  return launch_quantize4(m, p, q_bf16, k_bf16, q4, k4, q_sf, k_sf, q_g, k_g, workspace, (cudaStream_t)stream);
+}
+
 size_t sva_smooth_workspace_bytes(const sva_problem_t* p) {
   if (validate_problem(p)) return 0;
   return smooth_workspace_bytes(make_dims(p));

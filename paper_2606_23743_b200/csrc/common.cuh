@@ -80,6 +80,8 @@ int select_row_cap(const Dims& m, const sva_select_t* s);
 size_t smooth_workspace_bytes(const Dims& m);
 int launch_quantize(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q8,
                     void* k8, float* qs, float* ks, float* k_mean, float* lse_shift, void* ws, cudaStream_t st);
+int launch_quantize4(const Dims& m, const sva_problem_t* p, const void* q, const void* k, void* q4, void* k4,
+                     void* q_sf, void* k_sf, float* q_g, float* k_g, void* ws, cudaStream_t st);
 int launch_token_move(bool scatter, const void* src, const int64_t ss[3], void* dst, const int64_t sd[3],
                       const int32_t* idx, int B, int H, int M, int n_full, int d, int elem_bytes,
                       int32_t* status, cudaStream_t st);
