@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--workload", default="large", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--fp4", action="store_true",
+                    help="extended step: Q and K quantised to 4-bit block-scaled codes inside every step, Q K^T as a "
+                         "block-scaled 4-bit MMA (routing stays on the bf16 Q, K); 128-token blocks only")
     ap.add_argument("--remainder", action="store_true",
                     help="extended step: attention with the approximate remainder of the dropped blocks (order 0) "
                          "instead of exact-only attention; `value` still counts the selected blocks' FLOPs only")
@@ -248,6 +251,14 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     if args.remainder and (w.fp8 or args.prologue):
         raise SystemExit("--remainder runs on the plain bf16 step")
+    if args.fp4:
+        if w.fp8 or args.prologue or args.remainder or w.block != 128 or w.d != 128:
+            raise SystemExit("--fp4 runs on a bf16 workload with 128-token blocks and d = 128")
+        BH = w.B * w.H
+        q4 = torch.zeros(BH, w.Nb * 128, 64, dtype=torch.uint8, device=dev); k4 = torch.zeros_like(q4)
+        qsf = torch.zeros(BH, w.Nb, 1024, dtype=torch.uint8, device=dev); ksf = torch.zeros_like(qsf)
+        qg = torch.zeros(BH, dtype=torch.float32, device=dev); kg = torch.zeros_like(qg)
+        ws4 = torch.zeros(max(8 * BH, 256), dtype=torch.uint8, device=dev)
     aws = torch.empty(max(B.attn_remainder_workspace_bytes(p) if args.remainder else B.attn_workspace_bytes(p), 256),
                       dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
@@ -256,6 +267,8 @@ def main():
     launches_per_step = (4 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
+    if args.fp4:            # + amax and cast kernels of the 4-bit quantiser
+        launches_per_step += 2
     if args.remainder:      # + the block means of K and V (the memset before it is not a kernel of this library)
         launches_per_step += 1
 
@@ -275,7 +288,7 @@ def main():
             v_ready.record()
 
     # the two-step form serves what the tensor-core kernel serves (every supported shape today)
-    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder     # (the remainder call prepares V itself)
+    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder and not args.fp4     # (those calls prepare V themselves)
 
     def route(qq, kk, vv):
         if args.prologue:
@@ -299,7 +312,10 @@ def main():
     def attend(qq, kk, vv, oo):
         if args.prologue:
             qq, kk = qn, kn
-        if args.remainder:
+        if args.fp4:
+            B.quantize_qk_fp4(pq, qq, kk, q4, k4, qsf, ksf, qg, kg, ws4)
+            B.block_sparse_attn_fwd_fp4(p, q4, k4, qsf, ksf, qg, kg, vv, row_ptr, col_idx, oo, None, status, aws)
+        elif args.remainder:
             B.block_sparse_attn_remainder_fwd(p, qq, kk, vv, row_ptr, col_idx, oo, None, status, 0, aws)
         elif w.fp8 and two_step:
             torch.cuda.current_stream().wait_event(v_ready)
@@ -406,7 +422,7 @@ def main():
 
     # ---- attention with its V preparation in line (the one-call entry point: transpose, then the kernel)
     inline_ms = None
-    if two_step and not w.fp8 and not args.prologue and not args.remainder:
+    if two_step and not w.fp8 and not args.prologue:
         n_in = max(5, min(args.steps, 20))
         route(q, k, v)
         torch.cuda.current_stream().wait_event(v_ready)
@@ -480,7 +496,8 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "e4m3 QK^T, bf16 PV" if w.fp8 else "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": "e4m3 QK^T, bf16 PV" if w.fp8 else ("e2m1 block-scaled QK^T, bf16 PV" if args.fp4 else "bf16"),
+        "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
                    "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
                    "nnz_tiles": nnz, "parallelism": f"replicas x{world}", "prologue": bool(args.prologue),
@@ -515,7 +532,7 @@ def main():
         "clocks": clocks, "sustained": sustained, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline and not args.prologue and not args.remainder:   # (the oracle leg times the plain step)
+        if world == 1 and not args.no_cpu_baseline and not args.prologue and not args.remainder and not args.fp4:   # (the oracle leg times the plain step)
             import oracle
             oracle.build()
             line["cpu_baseline"] = cpu_baseline(w, bf16_bits(qh), bf16_bits(kh), bf16_bits(vh))

@@ -302,6 +302,20 @@ int sva_quantize_qk_fp4(const sva_problem_t* p, const void* q_bf16, const void* 
                         void* stream);
 
 /*
+ * Attention with 4-bit Q and K (the block-scaled low-bit Q K^T of the paper's quantisation direction): q4, k4,
+ * q_sf, k_sf, q_g, k_g as sva_quantize_qk_fp4 writes them; V, P V, O and the softmax as in
+ * sva_block_sparse_attn_fwd.  S = Q K^T runs as a block-scaled e2m1 x e2m1 tensor-core MMA with fp32 accumulation
+ * (the e4m3 scale factors are applied by the MMA, the two fp32 tensor scales are folded into the softmax scale),
+ * so the result is attention over the DEQUANTISED Q and K.  row_ptr == NULL means dense.  d = 128, block = 128
+ * only; p's q/k strides and qk_dtype are ignored (the code tensors have their own fixed layout).  workspace: >=
+ * sva_attn_workspace_bytes(p), as for the bf16 call.
+ */
+int sva_block_sparse_attn_fwd_fp4(const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
+                                  const void* k_sf, const float* q_g, const float* k_g, const void* v,
+                                  const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                  int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The same quantiser with K smoothing, the step the 8-bit attention work cited in the paper's related
  * work on quantised attention puts before the cast: per (b,h) the mean key over the N tokens,
  *   k_mean[b,h,:] = (1/N) sum_j k[b,h,j,:]        (fp32; per-block sums in a fixed order, then the blocks in

@@ -23,7 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
-    "sva_quantize_qk_fp4", "sva_attn_remainder_workspace_bytes", "sva_block_sparse_attn_remainder_fwd", "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
+    "sva_quantize_qk_fp4", "sva_block_sparse_attn_fwd_fp4", "sva_attn_remainder_workspace_bytes", "sva_block_sparse_attn_remainder_fwd", "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
 ]
 DEBUG_EXPORTS = ["sva_debug_set_prof_buffer", "sva_debug_set_mode", "sva_debug_set_wait_limit"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -93,6 +93,8 @@ def lib():
         L.sva_quantize_qk_fp8.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp]
         L.sva_quantize_qk_fp4.restype = C.c_int
         L.sva_quantize_qk_fp4.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sva_block_sparse_attn_fwd_fp4.restype = C.c_int
+        L.sva_block_sparse_attn_fwd_fp4.argtypes = [C.POINTER(Problem)] + [vp] * 13 + [C.c_size_t, vp]
         L.sva_smooth_workspace_bytes.restype = C.c_size_t
         L.sva_smooth_workspace_bytes.argtypes = [C.POINTER(Problem)]
         L.sva_quantize_qk_fp8_smooth_k.restype = C.c_int
@@ -336,3 +338,13 @@ def quantize_qk_fp4(p: Problem, q, k, q4, k4, q_sf, k_sf, q_g, k_g, workspace) -
                                    _ptr(k_g), _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_quantize_qk_fp4")
+
+
+def block_sparse_attn_fwd_fp4(p: Problem, q4, k4, q_sf, k_sf, q_g, k_g, v, row_ptr, col_idx, o, lse=None, status=None,
+                              workspace=None) -> None:
+    """Attention over 4-bit block-scaled Q and K (row_ptr None = dense)."""
+    rc = lib().sva_block_sparse_attn_fwd_fp4(C.byref(p), _ptr(q4), _ptr(k4), _ptr(q_sf), _ptr(k_sf), _ptr(q_g), _ptr(k_g),
+                                             _ptr(v), _ptr(row_ptr), _ptr(col_idx), _ptr(o), _ptr(lse), _ptr(status),
+                                             _ptr(workspace), _ws_bytes(workspace), _stream())
+    if rc != SVA_OK:
+        raise SvaError(rc, "sva_block_sparse_attn_fwd_fp4")

@@ -212,6 +212,25 @@ int sva_block_sparse_attn_remainder_fwd(const sva_problem_t* p, const void* q, c
                         workspace_bytes, (cudaStream_t)stream, order);
 }
 
+int sva_block_sparse_attn_fwd_fp4(const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
+                                  const void* k_sf, const float* q_g, const float* k_g, const void* v,
+                                  const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
+                                  int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = validate_problem(p);
+  if (rc) return rc;
+  if (!q4 || !k4 || !q_sf || !k_sf || !q_g || !k_g || !v || !o) return SVA_ERR_INVALID_ARG;
+  if (row_ptr && !col_idx) return SVA_ERR_INVALID_ARG;
+  if (!aligned16(q4) || !aligned16(k4) || !aligned16(q_sf) || !aligned16(k_sf) || !aligned16(v) || !aligned16(o))
+    return SVA_ERR_ALIGNMENT;
+  if ((rc = check_strides(p->v_stride, 8))) return rc;
+  if ((rc = check_strides(p->o_stride, 8))) return rc;
+  if (p->v_stride[2] < p->d || p->o_stride[2] < p->d) return SVA_ERR_INVALID_ARG;
+  Dims m = make_dims(p);
+  m.fp8 = false;
+  return launch_attn_ts_fp4(m, p, q4, k4, q_sf, k_sf, q_g, k_g, v, row_ptr, col_idx, o, lse, device_status, workspace,
+                            workspace_bytes, (cudaStream_t)stream);
+}
+
 int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                        const float* q_scale, const float* k_scale, void* o, float* lse,
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream) {

@@ -71,8 +71,10 @@ namespace sva {
 struct TsParams {
   const __nv_bfloat16* q;     // e4m3 variant: bytes (strides in elements either way)
   Strides sq;
-  const float* q_scale;       // e4m3 variant: one scale per (b, h, block) for Q and for K
+  const float* q_scale;       // e4m3 variant: one scale per (b, h, block) for Q and for K; 4-bit variant: one per (b, h)
   const float* k_scale;
+  const uint8_t* q_sf;        // 4-bit variant: e4m3 scale factors, 1024 bytes per (b, h, 128-token block), tile order
+  const uint8_t* k_sf;
   const int32_t* row_ptr;     // null = dense
   const int32_t* col_idx;
   __nv_bfloat16* o;
@@ -109,11 +111,13 @@ constexpr int OFF_V = OFF_K + KS * TILE;
 constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][128 B] panels (one per softmax group)
 constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
 constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers, reference exponents, row sums (two rows), row queue
+constexpr int OFF_Q4 = OFF_CTRL + 4096;     // 4-bit variant: the row's Q codes (8 KB) and their scale factors (1 KB)
 #ifdef SVA_TIMELINE
 constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024 + 3200 * 8;
 #else
-constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024;      // + alignment slack
+constexpr int SMEM_BYTES = OFF_Q4 + 8192 + 1024 + 1024;      // + alignment slack
 #endif
+constexpr uint32_t COL_SFA = 384, COL_SFB = 392;              // 4-bit variant: scale factors in the Q columns (8 + 2 x 8)
 constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
 // The reference exponent of a row is raised only when a block's maximum exceeds it by more than this
 // many powers of two.  P then reaches at most 2^32 and a row sum 2^32 * N: far inside fp32 (and bf16
@@ -178,7 +182,11 @@ __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int
 // zero-fills it if its list is empty, and otherwise publishes {row, count, start, first two entries}
 // in a small shared-memory queue that every other role reads in the same order.  All barriers keep running across rows, so the producers and the S
 // issuer run ahead into the next row while the softmax groups finish the current one.
-template <bool B64, bool F8, bool REM>
+// F4: Q and K as packed e2m1 codes with e4m3 scales per 16 elements and one fp32 scale per (b,h).  S is then a
+// block-scaled 4-bit MMA whose operands both come from shared memory (the Q tile is fetched by TMA once per row
+// instead of being written to tensor memory; tm_kp is the map of the Q codes), with the scale factors copied
+// into the tensor-memory columns the bf16 Q would have used.  128-token blocks, d = 128 only.
+template <bool B64, bool F8, bool REM, bool F4 = false>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_kp,
@@ -323,8 +331,17 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
             if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
             const uint32_t dst = sbase + OFF_K + s * TILE;
-            mbar_expect_tx(bar_k_full + 8 * s, KTILE);
-            if (REM && j >= n_own) {
+            mbar_expect_tx(bar_k_full + 8 * s, F4 ? 8192 + 1024 : KTILE);
+            if (F4) {
+              // packed codes of the key block (128 rows x 64 bytes, 64-byte swizzle) and its 1 KB of scale factors
+              int J = j;
+              if (prm.row_ptr) {
+                J = __ldg(prm.col_idx + beg + j);
+                if (J < 0 || J >= prm.Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
+              }
+              tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);
+              bulk_load(dst + 8192, prm.k_sf + ((long long)bh * prm.Nb + J) * 1024, 1024, bar_k_full + 8 * s);
+            } else if (REM && j >= n_own) {
               // pooled tile: 128 block means of K (rows beyond Nb are zero in the pooled tensor)
               const int c = j - n_own;
               tma_load_4d(dst, &tm_kp, bar_k_full + 8 * s, 0, c * BS, hh, bb);
@@ -414,7 +431,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             SVA_STAMP(2, i, j, 1);
             tc_fence_after();
             const uint64_t kd = kd0 + (uint64_t)(s * (TILE >> 4));
-            if (F8) {
+            if (F4) {
+              const uint32_t kslot = sbase + OFF_K + s * TILE;
+              if (j == 0) {                                    // the row's Q scale factors (q_ready: they are in shared memory)
+                tc_cp_sf(tmem_base + COL_SFA, smem_desc_plain(sbase + OFF_Q4 + 8192), 1u);
+                tc_cp_sf(tmem_base + COL_SFA + 4, smem_desc_plain(sbase + OFF_Q4 + 8192 + 512), 1u);
+              }
+              tc_cp_sf(tmem_base + COL_SFB + 8 * s, smem_desc_plain(kslot + 8192), 1u);
+              tc_cp_sf(tmem_base + COL_SFB + 8 * s + 4, smem_desc_plain(kslot + 8192 + 512), 1u);
+              const uint64_t qd4 = smem_desc_sw64(sbase + OFF_Q4), kd4 = smem_desc_sw64(kslot);
+#pragma unroll
+              for (int kk = 0; kk < 2; ++kk)                    // 64 elements (32 bytes) of d per instruction
+                tc_mma_bs4_ss(tmem_base + 128 * w, qd4 + (uint64_t)(kk * 2), kd4 + (uint64_t)(kk * 2), instr_desc_bs4(128, 128),
+                              tmem_base + COL_SFA + 4 * kk, tmem_base + COL_SFB + 8 * s + 4 * kk, kk > 0 ? 1u : 0u, 1u);
+            } else if (F8) {
 #pragma unroll
               for (int kk = 0; kk < D / 32; ++kk)               // 32 e4m3 values (32 bytes, 8 TMEM columns) per step
                 tc_mma_ts<true>(tmem_base + 128 * w, tmem_base + COL_Q + 8 * kk, kd + (uint64_t)(kk * 2), IDESC_QK,
@@ -495,7 +525,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     auto load_q = [&](int r, uint32_t* qv) {
 #pragma unroll
       for (int e = 0; e < 32; ++e) qv[e] = 0u;
-      if (r >= prm.R) return;
+      if (F4 || r >= prm.R) return;                                     // (4-bit variant: the Q tile goes to shared memory by TMA)
       const int bh = r / Nb, qi = (r % Nb) * BS + row;
       if (qi >= prm.N || 64 * w >= prm.d) return;                      // (d = 64: the second group's half of Q is zero)
       const long long eoff = (long long)(bh / prm.H) * prm.sq.b + (long long)(bh % prm.H) * prm.sq.h +
@@ -508,7 +538,19 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
       }
     };
-    auto store_q = [&](const uint32_t* qv) {
+    auto store_q = [&](const uint32_t* qv, int r) {
+      if (F4) {
+        // one thread fetches the row's Q codes and scale factors; the barrier completes when every softmax thread
+        // has arrived (none of them reads the previous row's Q any more) and the bytes have landed
+        if (threadIdx.x == 0) {
+          const int bh = r / Nb, I = r % Nb;
+          mbar_expect_tx_only(bar_q_ready, 8192 + 1024);
+          tma_load_4d(sbase + OFF_Q4, &tm_kp, bar_q_ready, 0, I * BS, bh % prm.H, bh / prm.H);
+          bulk_load(sbase + OFF_Q4 + 8192, prm.q_sf + ((long long)bh * prm.Nb + I) * 1024, 1024, bar_q_ready);
+        }
+        mbar_arrive(bar_q_ready);
+        return;
+      }
       if (F8) tmem_st16(q_tmem, qv); else tmem_st32(q_tmem, qv);
       tc_wait_st();
       tc_fence_before();
@@ -526,7 +568,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // first row: its Q goes in right away
       uint32_t qv[32];
       load_q(r_c, qv);
-      store_q(qv);
+      store_q(qv, r_c);
     }
     for (; ok && r_c < prm.R; ++rows_done) {
       const int r = r_c, n = n_c, lbeg = beg_c;
@@ -548,6 +590,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           ks_next = __ldg(ks + (int)e);
         }
       };
+      if (F4) c = prm.scale_log2 * __ldg(prm.q_scale + bh) * __ldg(prm.k_scale + bh);     // the two tensor scales
       if (F8) {
         const int qb = B64 ? min(2 * I + qh, prm.Nb - 1) : I;         // my query block
         qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + qb) * prm.scale_log2;
@@ -752,7 +795,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_arrive(bar_xch);
       if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
       // both groups have seen all their S tiles: no MMA reads Q any more
-      if (r_next < prm.R) store_q(qn);
+      if (r_next < prm.R) store_q(qn, r_next);
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
       if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 9);
@@ -986,9 +1029,10 @@ static encode_fn_t get_encode_ts() {
 }
 
 // 4-D map (inner, rows, H, B) of bf16 (or bytes) with byte strides; box = 128 bytes x box_rows, 128-byte swizzle.
+// (box_bytes = 64: rows of 64 bytes with the 64-byte swizzle, the packed 4-bit tiles)
 static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuuint64_t rows, int H, int B,
                        cuuint64_t row_stride, cuuint64_t h_stride, cuuint64_t b_stride, int box_rows,
-                       int elem_bytes = 2) {
+                       int elem_bytes = 2, int box_bytes = 128) {
   encode_fn_t enc = get_encode_ts();
   if (!enc) return SVA_ERR_CUDA;
   cuuint64_t dims[4] = {inner, rows, (cuuint64_t)H, (cuuint64_t)B};
@@ -998,10 +1042,11 @@ static int make_map_ts(CUtensorMap* map, const void* ptr, cuuint64_t inner, cuui
   if (B == 1) strides[2] = strides[1] * (cuuint64_t)H;
   for (int i = 0; i < 3; ++i)
     if (strides[i] % 16 != 0 || strides[i] == 0) return SVA_ERR_ALIGNMENT;
-  cuuint32_t box[4] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows, 1, 1};   // 128 bytes per row
+  cuuint32_t box[4] = {(cuuint32_t)(box_bytes / elem_bytes), (cuuint32_t)box_rows, 1, 1};   // 128 (or 64) bytes per row
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult rc = enc(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? SVA_OK : SVA_ERR_CUDA;
 }
@@ -1014,17 +1059,17 @@ static int g_debug_ts = 0;
 static constexpr int TS_MAX_DEVICES = 64;
 static std::mutex g_ts_mutex;
 static int g_ts_sms[TS_MAX_DEVICES];
-static bool g_ts_attr[TS_MAX_DEVICES][8];
+static bool g_ts_attr[TS_MAX_DEVICES][9];
 
-template <bool B64, bool F8, bool REM = false>
+template <bool B64, bool F8, bool REM = false, bool F4 = false>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                      const CUtensorMap& tkp, const CUtensorMap& tvp, const TsParams& prm, cudaStream_t st) {
-  auto kern = attn_ts_kernel<B64, F8, REM>;
+  auto kern = attn_ts_kernel<B64, F8, REM, F4>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
   {
     std::lock_guard<std::mutex> lock(g_ts_mutex);
-    constexpr int variant = (REM ? 4 : 0) + (B64 ? 2 : 0) + (F8 ? 1 : 0);
+    constexpr int variant = F4 ? 8 : (REM ? 4 : 0) + (B64 ? 2 : 0) + (F8 ? 1 : 0);
     if (!g_ts_attr[dev][variant]) {
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
         return SVA_ERR_CUDA;
@@ -1181,6 +1226,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   TsParams prm;
   prm.q = (const __nv_bfloat16*)q; prm.sq = make_strides(p->q_stride);
   prm.q_scale = q_scale; prm.k_scale = k_scale;
+  prm.q_sf = nullptr; prm.k_sf = nullptr;
   prm.row_ptr = row_ptr; prm.col_idx = col_idx;
   prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
   prm.so = make_strides(p->o_stride);
@@ -1212,6 +1258,51 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
   if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
   return launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+}
+
+// 4-bit Q/K: packed codes [B*H][Nb*128][64], tiled scale factors, one fp32 scale per (b,h); V bf16 as always.
+bool attn_ts_fp4_serves(const Dims& m) { return m.d == ts::D && m.block == BS && !m.fp8 && m.Nb <= 16383; }
+
+int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
+                       const void* k_sf, const float* q_g, const float* k_g, const void* v, const int32_t* row_ptr,
+                       const int32_t* col_idx, void* o, float* lse, int32_t* status, void* ws, size_t ws_bytes,
+                       cudaStream_t st) {
+  if (!attn_ts_fp4_serves(m)) return SVA_ERR_UNSUPPORTED;
+  int rc = check_ts_workspace(m, ws, ws_bytes);
+  if (rc) return rc;
+  const TsLayout L = ts_layout(m);
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  const Strides so = make_strides(p->o_stride);
+  CUtensorMap tk, tv, to, tq;
+  if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2, BS)) != SVA_OK)
+    return rc;
+  const cuuint64_t crow = (cuuint64_t)m.Nb * BS;              // token rows of the code tensors (padded to whole blocks)
+  if ((rc = make_map_ts(&tk, k4, 64, crow, m.H, m.B, 64, crow * 64, crow * 64 * m.H, BS, 1, 64)) != SVA_OK) return rc;
+  if ((rc = make_map_ts(&tq, q4, 64, crow, m.H, m.B, 64, crow * 64, crow * 64 * m.H, BS, 1, 64)) != SVA_OK) return rc;
+  const cuuint64_t vrows = (cuuint64_t)m.Nb * ts::D;
+  if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
+                        vrows * m.block * 2 * m.H, BS)) != SVA_OK)
+    return rc;
+  const Strides sv = make_strides(p->v_stride);
+  dim3 tg((m.Nb * m.block + 63) / 64, ts::D / 64, m.B * m.H);
+  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
+                                         reinterpret_cast<int32_t*>(wsb + L.counter_off));
+  if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+  TsParams prm = {};
+  prm.q = nullptr; prm.sq = Strides{0, 0, 0};
+  prm.q_scale = q_g; prm.k_scale = k_g;
+  prm.q_sf = static_cast<const uint8_t*>(q_sf); prm.k_sf = static_cast<const uint8_t*>(k_sf);
+  prm.row_ptr = row_ptr; prm.col_idx = col_idx;
+  prm.o = (__nv_bfloat16*)o; prm.lse = lse; prm.status = status;
+  prm.so = so;
+  prm.H = m.H; prm.N = m.N; prm.Nb = m.Nb; prm.Nt = L.Nt; prm.R = L.R2; prm.d = m.d;
+  prm.tile_cnt = nullptr; prm.tile_beg = nullptr; prm.tile_desc = nullptr;
+  prm.scale_log2 = m.scale * 1.4426950408889634f;
+  prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
+  prm.np = 0; prm.log2_block = 7.f; prm.tail_bias = 0.f;
+  prm.prof = g_prof_ts;
+  prm.debug = g_debug_ts;
+  return launch_ts<false, false, false, true>(L.R2, tk, tv, to, tq, tv, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }

@@ -91,6 +91,11 @@ int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const
 int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order = -1);
+int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
+                       const void* k_sf, const float* q_g, const float* k_g, const void* v, const int32_t* row_ptr,
+                       const int32_t* col_idx, void* o, float* lse, int32_t* status, void* ws, size_t ws_bytes,
+                       cudaStream_t st);
+bool attn_ts_fp4_serves(const Dims& m);
 size_t attn_ts_workspace_bytes(const Dims& m);
 size_t attn_ts_remainder_workspace_bytes(const Dims& m);
 bool attn_ts_remainder_serves(const Dims& m);

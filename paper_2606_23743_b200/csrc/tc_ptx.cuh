@@ -105,6 +105,31 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t b, ui
                  ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc), "r"(elected) : "memory");
 }
 
+// Block-scaled 4-bit MMA (e2m1 operands packed two per byte in shared memory, one e4m3 scale per 16
+// elements along K, K = 64 per instruction): D[tmem] (+)= (A .* SFA)[smem] * (B .* SFB)[smem]^T with the
+// scale factors in tensor memory (4 columns per operand and instruction, see tc_cp_sf).
+__device__ __forceinline__ void tc_mma_bs4_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t sfa,
+                                              uint32_t sfb, uint32_t acc, uint32_t elected) {
+  asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %6, 0;\nsetp.ne.b32 q, %7, 0;\n"
+               "@q tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%4], [%5], p;\n}"
+               ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(sfa), "r"(sfb), "r"(acc), "r"(elected) : "memory");
+}
+// Scale factors shared -> tensor memory: 32 rows x 16 bytes (512 contiguous bytes: the scales of 128 rows x 4
+// scale blocks, byte (r % 32) * 16 + (r / 32) * 4 + kb), replicated into the four 32-lane quarters; 4 columns.
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc, uint32_t elected) {
+  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n"
+               "@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;\n}" ::"r"(taddr), "l"(sdesc), "r"(elected) : "memory");
+}
+// plain bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// raises the transaction count a barrier's current phase waits for, without arriving
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
 #define SVA_R4(v, i) "=r"(v[i]), "=r"(v[i + 1]), "=r"(v[i + 2]), "=r"(v[i + 3])
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
   asm volatile(
@@ -188,6 +213,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
          ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// The same with a 64-byte swizzle (tiles whose rows are 64 bytes: 128 packed 4-bit values) and without swizzle
+// (8-row x 16-byte core matrices stored one after the other: the scale-factor groups).
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
+}
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(128 >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor of the block-scaled 4-bit MMA: e2m1 x e2m1 (format code 1 in both fields), e4m3
+// scales (bit 23 clear), A and B K-major, N, M, K = 64 (bit 31 clear); fp32 accumulation is implied.
+__host__ __device__ constexpr uint32_t instr_desc_bs4(int M, int N) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 // Instruction descriptor: fp32 accumulate, A/B format code, B major, N, M.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int fmt, bool b_mn_major) {
