@@ -259,12 +259,16 @@ def main():
         qsf = torch.zeros(BH, w.Nb, 1024, dtype=torch.uint8, device=dev); ksf = torch.zeros_like(qsf)
         qg = torch.zeros(BH, dtype=torch.float32, device=dev); kg = torch.zeros_like(qg)
         ws4 = torch.zeros(max(8 * BH, 256), dtype=torch.uint8, device=dev)
-    aws = torch.empty(max(B.attn_remainder_workspace_bytes(p) if args.remainder else B.attn_workspace_bytes(p), 256),
-                      dtype=torch.uint8, device=dev)
+    # e4m3 and 4-bit Q/K: the kernel reads V where it lies, the one-call entry point needs only its row counters
+    aws_bytes = (B.attn_remainder_workspace_bytes(p) if args.remainder else 256 if args.fp4 else
+                 B.attn_one_call_workspace_bytes(p) if w.fp8 else B.attn_workspace_bytes(p))
+    aws = torch.empty(max(aws_bytes, 256), dtype=torch.uint8, device=dev)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
     # routing kernels (pooling, scores, selection; CSR assembly when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
     launches_per_step = (4 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
+    if w.fp8 or args.fp4:   # no V transpose: V is read where it lies
+        launches_per_step -= 1
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
     if args.fp4:            # + amax and cast kernels of the 4-bit quantiser
@@ -288,7 +292,8 @@ def main():
             v_ready.record()
 
     # the two-step form serves what the tensor-core kernel serves (every supported shape today)
-    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder and not args.fp4     # (those calls prepare V themselves)
+    # bf16: V is prepared (tiled transposed copy) beside routing; the other forms have no such step
+    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder and not args.fp4 and not w.fp8
 
     def route(qq, kk, vv):
         if args.prologue:
@@ -409,7 +414,7 @@ def main():
     # ---- the kernel's own cycle counter (one extra launch): cycles do not depend on the SM clock, so
     # cycles / measured time is the clock each regime really ran at -- the record NVML cannot give for a burst
     kernel_cycles = None
-    if two_step:
+    if B.attn_workspace_bytes(p) > 0:
         prof = torch.zeros(320, dtype=torch.int64, device=dev)
         B.debug_set_prof_buffer(prof)
         try:

@@ -202,8 +202,13 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
  * GPU need a workspace each);
  * 0 only for an unsupported problem.
+ * sva_attn_one_call_workspace_bytes(p) is what sva_block_sparse_attn_fwd and sva_dense_attn_fwd themselves need (the
+ * larger figure also serves the two-step form below): the same for bf16 Q/K; for e4m3 Q/K -- whose kernel reads V
+ * where it lies, S and P V being different MMA kinds anyway -- only the row counters and, for 64-token blocks, the
+ * tile lists (a few KB to a few MB).  sva_block_sparse_attn_fwd_fp4 needs 256 bytes (its row counters).
  */
 size_t sva_attn_workspace_bytes(const sva_problem_t* p);
+size_t sva_attn_one_call_workspace_bytes(const sva_problem_t* p);
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                               const float* q_scale, const float* k_scale, const int32_t* row_ptr,
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,
@@ -307,8 +312,8 @@ int sva_quantize_qk_fp4(const sva_problem_t* p, const void* q_bf16, const void* 
  * sva_block_sparse_attn_fwd.  S = Q K^T runs as a block-scaled e2m1 x e2m1 tensor-core MMA with fp32 accumulation
  * (the e4m3 scale factors are applied by the MMA, the two fp32 tensor scales are folded into the softmax scale),
  * so the result is attention over the DEQUANTISED Q and K.  row_ptr == NULL means dense.  d = 128, block = 128
- * only; p's q/k strides and qk_dtype are ignored (the code tensors have their own fixed layout).  workspace: >=
- * sva_attn_workspace_bytes(p), as for the bf16 call.
+ * only; p's q/k strides and qk_dtype are ignored (the code tensors have their own fixed layout).  V is read where
+ * it lies (no transposed copy): workspace >= 256 bytes (the row counters), 256-byte aligned.
  */
 int sva_block_sparse_attn_fwd_fp4(const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
                                   const void* k_sf, const float* q_g, const float* k_g, const void* v,

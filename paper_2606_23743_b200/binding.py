@@ -23,7 +23,7 @@ EXPORTS = [
     "sva_block_sparse_attn_fwd", "sva_dense_attn_fwd", "sva_block_sparse_attn_fwd_simt",
     "sva_quantize_qk_fp8", "sva_status_string", "sva_block_select_noalloc", "sva_attn_workspace_bytes",
     "sva_attn_prepare_v", "sva_block_sparse_attn_fwd_prepared", "sva_gather_tokens", "sva_scatter_tokens",
-    "sva_quantize_qk_fp4", "sva_block_sparse_attn_fwd_fp4", "sva_attn_remainder_workspace_bytes", "sva_block_sparse_attn_remainder_fwd", "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
+    "sva_attn_one_call_workspace_bytes", "sva_quantize_qk_fp4", "sva_block_sparse_attn_fwd_fp4", "sva_attn_remainder_workspace_bytes", "sva_block_sparse_attn_remainder_fwd", "sva_smooth_workspace_bytes", "sva_quantize_qk_fp8_smooth_k", "sva_block_select_pooled", "sva_qk_norm_rope_pool", "sva_pool_qk",
 ]
 DEBUG_EXPORTS = ["sva_debug_set_prof_buffer", "sva_debug_set_mode", "sva_debug_set_wait_limit"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -67,6 +67,8 @@ def lib():
         L.sva_block_select_noalloc.restype = C.c_int
         L.sva_block_select_noalloc.argtypes = [C.POINTER(Problem), C.POINTER(Select), vp, vp, vp, vp, vp, vp,
                                                vp, vp]
+        L.sva_attn_one_call_workspace_bytes.restype = C.c_size_t
+        L.sva_attn_one_call_workspace_bytes.argtypes = [C.POINTER(Problem)]
         L.sva_attn_workspace_bytes.restype = C.c_size_t
         L.sva_attn_workspace_bytes.argtypes = [C.POINTER(Problem)]
         L.sva_block_sparse_attn_fwd.restype = C.c_int
@@ -348,3 +350,8 @@ def block_sparse_attn_fwd_fp4(p: Problem, q4, k4, q_sf, k_sf, q_g, k_g, v, row_p
                                              _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_fwd_fp4")
+
+
+def attn_one_call_workspace_bytes(p: Problem) -> int:
+    """Workspace the one-call attention entry points need (e4m3 Q/K: just the row counters and tile lists)."""
+    return int(lib().sva_attn_one_call_workspace_bytes(C.byref(p)))

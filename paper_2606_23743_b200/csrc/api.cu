@@ -178,6 +178,11 @@ size_t sva_attn_workspace_bytes(const sva_problem_t* p) {
   return attn_ts_workspace_bytes(m);
 }
 
+size_t sva_attn_one_call_workspace_bytes(const sva_problem_t* p) {
+  if (validate_problem(p)) return 0;
+  return attn_ts_one_call_workspace_bytes(make_dims(p));
+}
+
 int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
                               const float* q_scale, const float* k_scale, const int32_t* row_ptr,
                               const int32_t* col_idx, void* o, float* lse, int32_t* device_status,

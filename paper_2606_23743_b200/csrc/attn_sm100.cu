@@ -186,7 +186,10 @@ __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int
 // block-scaled 4-bit MMA whose operands both come from shared memory (the Q tile is fetched by TMA once per row
 // instead of being written to tensor memory; tm_kp is the map of the Q codes), with the scale factors copied
 // into the tensor-memory columns the bf16 Q would have used.  128-token blocks, d = 128 only.
-template <bool B64, bool F8, bool REM, bool F4 = false>
+// VMN: V is read where it lies ([keys][d], d contiguous) and enters P V as an MN-major B operand -- another
+// instruction descriptor than S, which costs a tensor-pipe drain per switch, but no transposed copy of V and no
+// workspace for it.  Used where S and P V differ in kind anyway (e4m3 and 4-bit Q/K); tm_vt is then the map of V.
+template <bool B64, bool F8, bool REM, bool F4 = false, bool VMN = false>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_kp,
@@ -387,7 +390,20 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const uint32_t e = list_block<B64, REM>(prm, beg, j, n_own);
             const uint32_t dst = sbase + OFF_V + s * TILE;
             mbar_expect_tx(bar_v_full + 8 * s, TILE);
-            if (REM && j >= n_own) {
+            if (VMN) {
+              // V itself: two d-panels of [128 keys][64 d] (64-token blocks: each panel's two halves from two key blocks)
+              if (B64) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  const int Jh = (int)((e >> (16 * h)) & 0x3fffu);
+                  tma_load_4d(dst + h * (TILE / 4), &tm_vt, bar_v_full + 8 * s, 0, Jh * KB, hh, bb);
+                  tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_vt, bar_v_full + 8 * s, 64, Jh * KB, hh, bb);
+                }
+              } else {
+                tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)e * BS, hh, bb);
+                tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, (int)e * BS, hh, bb);
+              }
+            } else if (REM && j >= n_own) {
               // pooled tile: the block means of V, transposed ([128 d rows][128 blocks]; blocks beyond Nb zero)
               const int c = j - n_own;
               tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
@@ -467,7 +483,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     } else {
       // ---------------------------------------------------------- P V issuer (one lane)
       if (lane == 0) {
-        const uint64_t vd0 = smem_desc(sbase + OFF_V, 16, 1024);
+        // (VMN: 64 d-values contiguous, the next 64 one panel = 16 KB on, 8 keys 1 KB apart)
+        const uint64_t vd0 = VMN ? smem_desc(sbase + OFF_V, TILE / 2, 1024) : smem_desc(sbase + OFF_V, 16, 1024);
+        constexpr uint32_t IDESC_PV = VMN ? instr_desc(128, 128, 1, true) : IDESC;
         int s = 0;
         uint32_t ph = 0;
         uint32_t cp[2] = {0, 0};            // P V groups issued so far for parity w
@@ -489,8 +507,9 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < BS / 16; ++kk) {
-              const uint64_t off = (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
-              tc_mma_ts(tmem_base + COL_O, tmem_base + COL_P + 8 * kk, vd + off, IDESC, (j > 0 || kk > 0) ? 1u : 0u, 1u);
+              const uint64_t off = VMN ? (uint64_t)(kk * 128)            // 16 keys = 16 rows of 128 bytes
+                                       : (uint64_t)((kk / 4) * PANEL16 + (kk % 4) * 2);
+              tc_mma_ts(tmem_base + COL_O, tmem_base + COL_P + 8 * kk, vd + off, IDESC_PV, (j > 0 || kk > 0) ? 1u : 0u, 1u);
             }
             SVA_STAMP(3, i, j, 2);
             tc_commit(bar_v_empty + 8 * s, 1u);
@@ -1059,17 +1078,17 @@ static int g_debug_ts = 0;
 static constexpr int TS_MAX_DEVICES = 64;
 static std::mutex g_ts_mutex;
 static int g_ts_sms[TS_MAX_DEVICES];
-static bool g_ts_attr[TS_MAX_DEVICES][9];
+static bool g_ts_attr[TS_MAX_DEVICES][16];
 
-template <bool B64, bool F8, bool REM = false, bool F4 = false>
+template <bool B64, bool F8, bool REM = false, bool F4 = false, bool VMN = false>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                      const CUtensorMap& tkp, const CUtensorMap& tvp, const TsParams& prm, cudaStream_t st) {
-  auto kern = attn_ts_kernel<B64, F8, REM, F4>;
+  auto kern = attn_ts_kernel<B64, F8, REM, F4, VMN>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
   {
     std::lock_guard<std::mutex> lock(g_ts_mutex);
-    constexpr int variant = F4 ? 8 : (REM ? 4 : 0) + (B64 ? 2 : 0) + (F8 ? 1 : 0);
+    constexpr int variant = F4 ? 8 : (VMN ? 9 : 0) + (REM ? 4 : 0) + (B64 ? 2 : 0) + (F8 ? 1 : 0);
     if (!g_ts_attr[dev][variant]) {
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ts::SMEM_BYTES) != cudaSuccess)
         return SVA_ERR_CUDA;
@@ -1094,9 +1113,10 @@ struct TsLayout {
   long long cap;
   int R2, Nt;
 };
-static TsLayout ts_layout(const Dims& m) {
+// (no_vt: V is read where it lies -- no transposed copy, the rest moves to the front)
+static TsLayout ts_layout(const Dims& m, bool no_vt = false) {
   TsLayout L;
-  L.vt_bytes = (size_t)m.B * m.H * m.Nb * m.block * ts::D * 2;      // (d = 64: tiles are padded to 128 d-rows)
+  L.vt_bytes = no_vt ? 0 : (size_t)m.B * m.H * m.Nb * m.block * ts::D * 2;      // (d = 64: tiles are padded to 128 d-rows)
   L.counter_off = L.vt_bytes;
   L.Nt = m.block == 64 ? (m.Nb + 1) / 2 : m.Nb;
   L.R2 = m.B * m.H * L.Nt;
@@ -1128,6 +1148,13 @@ size_t attn_ts_remainder_workspace_bytes(const Dims& m) {
   return attn_ts_remainder_serves(m) ? ts_layout(m).total_rem : 0;
 }
 
+// What the one-call entry points need: e4m3 Q/K read V where it lies, so only the row counters (and the tile
+// lists of 64-token blocks) remain; bf16 Q/K as attn_ts_workspace_bytes.
+size_t attn_ts_one_call_workspace_bytes(const Dims& m) {
+  if (!attn_ts_serves(m)) return 0;
+  return m.fp8 ? ts_layout(m, true).total : attn_ts_workspace_bytes(m);
+}
+
 size_t attn_ts_workspace_bytes(const Dims& m) {
   if (!attn_ts_serves(m)) return 0;
   size_t bytes = ts_layout(m).total;
@@ -1140,9 +1167,9 @@ size_t attn_ts_workspace_bytes(const Dims& m) {
   return bytes;
 }
 
-static int check_ts_workspace(const Dims& m, const void* ws, size_t ws_bytes) {
+static int check_ts_workspace(const Dims& m, const void* ws, size_t ws_bytes, bool one_call = false) {
   if (!attn_ts_serves(m)) return SVA_ERR_UNSUPPORTED;
-  if (!ws || ws_bytes < attn_ts_workspace_bytes(m)) return SVA_ERR_WORKSPACE;
+  if (!ws || ws_bytes < (one_call ? attn_ts_one_call_workspace_bytes(m) : attn_ts_workspace_bytes(m))) return SVA_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
   return SVA_OK;
 }
@@ -1166,7 +1193,7 @@ int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, vo
 int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
                    void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order) {
-  int rc = check_ts_workspace(m_in, ws, ws_bytes);
+  int rc = check_ts_workspace(m_in, ws, ws_bytes, v != nullptr);
   if (rc) return rc;
   const bool rem = remainder_order >= 0;
   if (rem) {
@@ -1181,7 +1208,10 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     m.R = m.B * m.H * m.Nb;
   }
   const bool b64 = m.block == 64;
-  const TsLayout L = ts_layout(m);
+  // e4m3 Q/K with V at hand: V is read where it lies (S and P V differ in kind anyway), no transposed copy.
+  // (bf16: only on request, bit 5 of the debug mode, to measure what the copy buys.)
+  const bool vmn = v != nullptr && remainder_order < 0 && (m.fp8 || ((g_debug_ts & 32) && !b64));
+  const TsLayout L = ts_layout(m, vmn && m.fp8);
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
@@ -1213,7 +1243,14 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     if ((rc = make_map_ts(&tvp, vtp, BS, prow, m.H, m.B, (cuuint64_t)BS * 2, prow * BS * 2, prow * BS * 2 * m.H, BS)) != SVA_OK)
       return rc;
   }
-  if (v) {
+  if (vmn) {
+    const Strides sv = make_strides(p->v_stride);
+    if ((rc = make_map_ts(&tv, v, m.d, m.N, m.H, m.B, (cuuint64_t)sv.n * 2, (cuuint64_t)sv.h * 2, (cuuint64_t)sv.b * 2,
+                          m.block)) != SVA_OK)
+      return rc;
+    tvp = tv;
+    if (cudaMemsetAsync(wsb + L.counter_off, 0, 256, st) != cudaSuccess) return SVA_ERR_CUDA;
+  } else if (v) {
     // (the transposed copy is laid out for the block size of this launch)
     const Strides sv = make_strides(p->v_stride);
     dim3 tg((m.Nb * m.block + 63) / 64, ts::D / 64, m.B * m.H);    // every key slot of every tile, also those beyond N (zeros)
@@ -1252,12 +1289,15 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
       if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     }
     if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-    return m.fp8 ? launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
-                 : launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+    if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
+                          : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
   }
   if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-  if (m.fp8) return launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-  return launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+  if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
+                        : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+  return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
+             : launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
 }
 
 // 4-bit Q/K: packed codes [B*H][Nb*128][64], tiled scale factors, one fp32 scale per (b,h); V bf16 as always.
@@ -1268,9 +1308,10 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
                        const int32_t* col_idx, void* o, float* lse, int32_t* status, void* ws, size_t ws_bytes,
                        cudaStream_t st) {
   if (!attn_ts_fp4_serves(m)) return SVA_ERR_UNSUPPORTED;
-  int rc = check_ts_workspace(m, ws, ws_bytes);
-  if (rc) return rc;
-  const TsLayout L = ts_layout(m);
+  const TsLayout L = ts_layout(m, true);                      // V is read where it lies: the row counters only
+  if (!ws || ws_bytes < L.total) return SVA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SVA_ERR_ALIGNMENT;
+  int rc;
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides so = make_strides(p->o_stride);
   CUtensorMap tk, tv, to, tq;
@@ -1279,15 +1320,11 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
   const cuuint64_t crow = (cuuint64_t)m.Nb * BS;              // token rows of the code tensors (padded to whole blocks)
   if ((rc = make_map_ts(&tk, k4, 64, crow, m.H, m.B, 64, crow * 64, crow * 64 * m.H, BS, 1, 64)) != SVA_OK) return rc;
   if ((rc = make_map_ts(&tq, q4, 64, crow, m.H, m.B, 64, crow * 64, crow * 64 * m.H, BS, 1, 64)) != SVA_OK) return rc;
-  const cuuint64_t vrows = (cuuint64_t)m.Nb * ts::D;
-  if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
-                        vrows * m.block * 2 * m.H, BS)) != SVA_OK)
-    return rc;
   const Strides sv = make_strides(p->v_stride);
-  dim3 tg((m.Nb * m.block + 63) / 64, ts::D / 64, m.B * m.H);
-  transpose_v_kernel<<<tg, 256, 0, st>>>((const __nv_bfloat16*)v, sv, (__nv_bfloat16*)ws, m.H, m.N, m.Nb, m.d, m.block,
-                                         reinterpret_cast<int32_t*>(wsb + L.counter_off));
-  if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
+  if ((rc = make_map_ts(&tv, v, m.d, m.N, m.H, m.B, (cuuint64_t)sv.n * 2, (cuuint64_t)sv.h * 2, (cuuint64_t)sv.b * 2,
+                        BS)) != SVA_OK)
+    return rc;
+  if (cudaMemsetAsync(wsb + L.counter_off, 0, 256, st) != cudaSuccess) return SVA_ERR_CUDA;
   TsParams prm = {};
   prm.q = nullptr; prm.sq = Strides{0, 0, 0};
   prm.q_scale = q_g; prm.k_scale = k_g;
@@ -1302,7 +1339,7 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
   prm.np = 0; prm.log2_block = 7.f; prm.tail_bias = 0.f;
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
-  return launch_ts<false, false, false, true>(L.R2, tk, tv, to, tq, tv, prm, st);
+  return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }

@@ -97,6 +97,7 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
                        cudaStream_t st);
 bool attn_ts_fp4_serves(const Dims& m);
 size_t attn_ts_workspace_bytes(const Dims& m);
+size_t attn_ts_one_call_workspace_bytes(const Dims& m);
 size_t attn_ts_remainder_workspace_bytes(const Dims& m);
 bool attn_ts_remainder_serves(const Dims& m);
 bool attn_ts_serves(const Dims& m);    // d = 128 or 64, bf16 or e4m3 Q/K, 128- or 64-token blocks

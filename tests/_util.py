@@ -70,7 +70,7 @@ def gpu_attn(w: Workload, q, k, v, row_ptr, col_idx, N=None, simt=False, dense=F
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(q, k, v, o, N, w.block, 0.0, fp8)
     # (0xff bytes are NaNs as bf16: whatever the kernels do not write themselves shows up in the output)
-    ws = torch.full((max(B.attn_workspace_bytes(p), 256),), 0xFF, dtype=torch.uint8, device="cuda")
+    ws = torch.full((max(B.attn_one_call_workspace_bytes(p), 256),), 0xFF, dtype=torch.uint8, device="cuda")
     if dense and not simt:
         B.dense_attn_fwd(p, q, k, v, o, lse, status, q_scale, k_scale, workspace=ws)
     else:
