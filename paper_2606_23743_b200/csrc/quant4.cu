@@ -27,9 +27,16 @@ amax_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
   const __nv_bfloat16* base = (which ? k : q) + (long long)(bh / H) * s.b + (long long)(bh % H) * s.h;
   const int lo = I * 128, cnt = min(128, N - lo);
   uint32_t m = 0u;                                            // max of the |x| bit patterns (bf16 in the upper half)
-  for (int i = threadIdx.x; i < cnt * 16; i += Q4_THREADS) {  // 16 vectors of 8 elements per token
-    const uint4 u = __ldg(reinterpret_cast<const uint4*>(base + (long long)(lo + (i >> 4)) * s.n) + (i & 15));
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+  uint4 u[8];                                                 // 16 vectors of 8 elements per token: 8 loads in flight per thread
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const int i = threadIdx.x + r * Q4_THREADS;
+    u[r] = make_uint4(0u, 0u, 0u, 0u);
+    if (i < cnt * 16) u[r] = __ldg(reinterpret_cast<const uint4*>(base + (long long)(lo + (i >> 4)) * s.n) + (i & 15));
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t w[4] = {u[r].x, u[r].y, u[r].z, u[r].w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       m = max(m, (w[e] << 16) & 0x7fffffffu);
@@ -72,10 +79,16 @@ quantize4_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
       const float sd = e4m3_to_float(sf);
       if (sd > 0.f) {
         const float sc = __fmul_rn(sd, g);
+        // x / sc: the correctly rounded quotient from one reciprocal per scale block (div_fast), a true
+        // division where that sequence is not exact
+        const bool fast = div_fast_ok(sc);
+        const float rc = __frcp_rn(sc);
         uint32_t pk[2] = {0u, 0u};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const float2 y = make_float2(__fdiv_rn(bf16lo(w[e]), sc), __fdiv_rn(bf16hi(w[e]), sc));
+          const float x0 = bf16lo(w[e]), x1 = bf16hi(w[e]);
+          const float2 y = fast ? make_float2(div_fast(x0, sc, rc), div_fast(x1, sc, rc))
+                                : make_float2(__fdiv_rn(x0, sc), __fdiv_rn(x1, sc));
           const uint32_t byte = (uint32_t)__nv_cvt_float2_to_fp4x2(y, __NV_E2M1, cudaRoundNearest);
           pk[e >> 2] |= (byte & 0xffu) << (8 * (e & 3));
         }
