@@ -206,6 +206,8 @@ def main():
     ap.add_argument("--remainder", action="store_true",
                     help="extended step: attention with the approximate remainder of the dropped blocks (order 0) "
                          "instead of exact-only attention; `value` still counts the selected blocks' FLOPs only")
+    ap.add_argument("--remainder-order", type=int, default=0, choices=[0, 1],
+                    help="with --remainder: 0 = block-mean term only, 1 = plus the first-order term")
     ap.add_argument("--sustained-seconds", type=float, default=2.5,
                     help="length of the second, back-to-back leg whose clocks NVML can follow (0 = skip)")
     ap.add_argument("--prologue", action="store_true",
@@ -260,9 +262,12 @@ def main():
         qg = torch.zeros(BH, dtype=torch.float32, device=dev); kg = torch.zeros_like(qg)
         ws4 = torch.zeros(max(8 * BH, 256), dtype=torch.uint8, device=dev)
     # e4m3 and 4-bit Q/K: the kernel reads V where it lies, the one-call entry point needs only its row counters
-    aws_bytes = (B.attn_remainder_workspace_bytes(p) if args.remainder else 256 if args.fp4 else
+    aws_bytes = (B.attn_remainder_workspace_bytes(p, args.remainder_order) if args.remainder else 256 if args.fp4 else
                  B.attn_one_call_workspace_bytes(p) if w.fp8 else B.attn_workspace_bytes(p))
     aws = torch.empty(max(aws_bytes, 256), dtype=torch.uint8, device=dev)
+    # the first-order term of the remainder weighs the dropped blocks by the routing's scores
+    scores_buf = (torch.empty(w.B, w.H, w.Nb, w.Nb, dtype=torch.float32, device=dev)
+                  if args.remainder and args.remainder_order == 1 else None)
     variable_rows = w.mode == 1 or (w.win_t >= 0 and w.k < (2 * w.win_t + 1) * (2 * w.win_s + 1))
     # routing kernels (pooling, scores, selection; CSR assembly when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
@@ -274,7 +279,7 @@ def main():
     if args.fp4:            # + amax and cast kernels of the 4-bit quantiser
         launches_per_step += 2
     if args.remainder:      # + the block means of K and V (the memset before it is not a kernel of this library)
-        launches_per_step += 1
+        launches_per_step += 1 + (3 if args.remainder_order == 1 else 0)       # order 1: + C_J, weights, aggregation
 
     # V is prepared (tiled transposed copy) on a second stream while routing, which never reads V, runs
     # (lower priority: its CTAs fill the SMs that the latency-bound selection kernel leaves idle instead of
@@ -312,7 +317,7 @@ def main():
         else:
             if two_step:
                 prepare_v(vv)
-            B.block_select(p, s, qq, kk, row_ptr, col_idx, ws)
+            B.block_select(p, s, qq, kk, row_ptr, col_idx, ws, block_scores=scores_buf)
 
     def attend(qq, kk, vv, oo):
         if args.prologue:
@@ -321,7 +326,8 @@ def main():
             B.quantize_qk_fp4(pq, qq, kk, q4, k4, qsf, ksf, qg, kg, ws4)
             B.block_sparse_attn_fwd_fp4(p, q4, k4, qsf, ksf, qg, kg, vv, row_ptr, col_idx, oo, None, status, aws)
         elif args.remainder:
-            B.block_sparse_attn_remainder_fwd(p, qq, kk, vv, row_ptr, col_idx, oo, None, status, 0, aws)
+            B.block_sparse_attn_remainder_fwd(p, qq, kk, vv, row_ptr, col_idx, oo, None, status, args.remainder_order, aws,
+                                              scores_buf)
         elif w.fp8 and two_step:
             torch.cuda.current_stream().wait_event(v_ready)
             B.block_sparse_attn_fwd_prepared(p, q8, k8, row_ptr, col_idx, oo, None, status, workspace=aws,
@@ -506,7 +512,9 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "block": w.block,
                    "rule": "mass>=%.2f cap %d" % (w.tau, w.k) if w.mode == 1 else "top-%d" % w.k,
                    "nnz_tiles": nnz, "parallelism": f"replicas x{world}", "prologue": bool(args.prologue),
-                   "remainder": "order 0: +%d pooled tiles per query-block row" % (-(-w.Nb // 128)) if args.remainder else None,
+                   "remainder": ("order %d: +%d pooled%s tiles per query-block row" % (
+                       args.remainder_order, -(-w.Nb // 128), " +%d first-order" % (2 if w.block == 64 else 1)
+                       if args.remainder_order else "")) if args.remainder else None,
                    "l2": "inputs (%.0f MB) larger than L2; no flush" % (3 * sel_bytes / 2 / 1e6)},
         "tokens_per_s": world * w.B * w.N / (ms_per_step * 1e-3),
         "attention_ms": attn_ms, "select_ms": sel_ms,

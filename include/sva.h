@@ -226,18 +226,23 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
  * order 0 stops there: a dropped block acts as n_J copies of its mean key carrying its mean value.  On the
  * device the dropped blocks cost ceil(Nb/128) extra tiles per query block, whose "keys" and "values" are the
  * bf16-rounded block means (written into the workspace by this call), the kept blocks masked out.
- * order 1 adds scale * exp(sbar_IJ) * C_J^T q_i per dropped block, C_J = sum_j (k_j - kbar_J) v_j^T weighted at
- * the query block's mean query so that the dropped blocks collapse into one d x d matrix per query block: not
- * built on the device yet (SVA_ERR_UNSUPPORTED).
+ * order 1 adds scale * exp(sbar_IJ) * C_J^T q_i per dropped block, C_J = sum_j (k_j - kbar_J) v_j^T, weighted at
+ * the query block's mean query (sbar_IJ is the routing score) so that the dropped blocks collapse into one d x d
+ * matrix per query block, A_I = sum_J exp(sbar_IJ) C_J.  On the device: C_J per key block (one tensor-core product
+ * K_J^T V_J, centred), the weights from `block_scores` and the CSR, A_I as a [Nb x Nb] x [Nb x d*d] GEMM per head
+ * (2*Nb^2*d^2 FLOP), all bf16 in the workspace, and one more tile per row in the attention kernel whose "P" are the
+ * scaled query values and whose "V^T" is A_I^T (two such tiles per tile row with 64-token blocks).
+ *   block_scores : order 1 only: the [B,H,Nb,Nb] fp32 score matrix sva_block_select wrote for this Q, K
+ *                  (16-byte aligned); ignored (may be NULL) for order 0
  * Supported: bf16 Q/K, d = 128, 128- or 64-token blocks; otherwise SVA_ERR_UNSUPPORTED.  A query block that
  * drops nothing gets exactly the result of sva_block_sparse_attn_fwd.  workspace: >=
- * sva_attn_remainder_workspace_bytes(p), 256-byte aligned, rewritten by every call.  Everything else as for
- * sva_block_sparse_attn_fwd.
+ * sva_attn_remainder_workspace_bytes(p, order), 256-byte aligned, rewritten by every call (order 1 holds two
+ * d x d bf16 matrices per block row there: 2 * 32 KB * R).  Everything else as for sva_block_sparse_attn_fwd.
  */
-size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p);
+size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p, int32_t order);
 int sva_block_sparse_attn_remainder_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
-                                        const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
-                                        int32_t* device_status, int32_t order, void* workspace,
+                                        const int32_t* row_ptr, const int32_t* col_idx, const float* block_scores,
+                                        void* o, float* lse, int32_t* device_status, int32_t order, void* workspace,
                                         size_t workspace_bytes, void* stream);
 
 /* The dense fallback: every block kept, no CSR read. */

@@ -79,9 +79,9 @@ def lib():
         L.sva_dense_attn_fwd.restype = C.c_int
         L.sva_dense_attn_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.sva_attn_remainder_workspace_bytes.restype = C.c_size_t
-        L.sva_attn_remainder_workspace_bytes.argtypes = [C.POINTER(Problem)]
+        L.sva_attn_remainder_workspace_bytes.argtypes = [C.POINTER(Problem), C.c_int32]
         L.sva_block_sparse_attn_remainder_fwd.restype = C.c_int
-        L.sva_block_sparse_attn_remainder_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp,
+        L.sva_block_sparse_attn_remainder_fwd.argtypes = [C.POINTER(Problem), vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp,
                                                           C.c_size_t, vp]
         L.sva_attn_prepare_v.restype = C.c_int
         L.sva_attn_prepare_v.argtypes = [C.POINTER(Problem), vp, vp, C.c_size_t, vp]
@@ -320,16 +320,17 @@ def debug_set_wait_limit(cycles: int) -> None:
         raise RuntimeError("sva_debug_set_wait_limit failed")
 
 
-def attn_remainder_workspace_bytes(p: Problem) -> int:
-    return int(lib().sva_attn_remainder_workspace_bytes(C.byref(p)))
+def attn_remainder_workspace_bytes(p: Problem, order: int = 0) -> int:
+    return int(lib().sva_attn_remainder_workspace_bytes(C.byref(p), int(order)))
 
 
 def block_sparse_attn_remainder_fwd(p: Problem, q, k, v, row_ptr, col_idx, o, lse=None, status=None, order: int = 0,
-                                    workspace=None) -> None:
-    """Exact attention over the kept blocks plus the approximate remainder of the dropped ones (order 0)."""
+                                    workspace=None, block_scores=None) -> None:
+    """Exact attention over the kept blocks plus the approximate remainder of the dropped ones (order 0: block means;
+    order 1: plus the first-order term, which needs the routing's score matrix)."""
     rc = lib().sva_block_sparse_attn_remainder_fwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(row_ptr), _ptr(col_idx),
-                                                   _ptr(o), _ptr(lse), _ptr(status), int(order), _ptr(workspace),
-                                                   _ws_bytes(workspace), _stream())
+                                                   _ptr(block_scores), _ptr(o), _ptr(lse), _ptr(status), int(order),
+                                                   _ptr(workspace), _ws_bytes(workspace), _stream())
     if rc != SVA_OK:
         raise SvaError(rc, "sva_block_sparse_attn_remainder_fwd")
 

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsva.so")
-SOURCES = ["api.cu", "select.cu", "quant.cu", "quant4.cu", "prologue.cu", "gather.cu", "attn_simt.cu", "attn_sm100.cu"]
+SOURCES = ["api.cu", "select.cu", "quant.cu", "quant4.cu", "remainder.cu", "prologue.cu", "gather.cu", "attn_simt.cu", "attn_sm100.cu"]
 HEADERS = ["common.cuh", "tc_ptx.cuh", os.path.join("..", "..", "include", "sva.h")]
 
 

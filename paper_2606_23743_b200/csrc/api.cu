@@ -198,23 +198,24 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
                           (cudaStream_t)stream);
 }
 
-size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p) {
-  if (validate_problem(p)) return 0;
-  return attn_ts_remainder_workspace_bytes(make_dims(p));
+size_t sva_attn_remainder_workspace_bytes(const sva_problem_t* p, int32_t order) {
+  if (validate_problem(p) || (order != 0 && order != 1)) return 0;
+  return attn_ts_remainder_workspace_bytes(make_dims(p), order);
 }
 
 int sva_block_sparse_attn_remainder_fwd(const sva_problem_t* p, const void* q, const void* k, const void* v,
-                                        const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse,
-                                        int32_t* device_status, int32_t order, void* workspace,
+                                        const int32_t* row_ptr, const int32_t* col_idx, const float* block_scores,
+                                        void* o, float* lse, int32_t* device_status, int32_t order, void* workspace,
                                         size_t workspace_bytes, void* stream) {
   int rc = validate_attn(p, q, k, v, nullptr, nullptr, o);
   if (rc) return rc;
   if (!row_ptr || !col_idx) return SVA_ERR_INVALID_ARG;
   if (order != 0 && order != 1) return SVA_ERR_INVALID_ARG;
   Dims m = make_dims(p);
-  if (!attn_ts_remainder_serves(m) || order != 0) return SVA_ERR_UNSUPPORTED;
+  if (!attn_ts_remainder_serves(m)) return SVA_ERR_UNSUPPORTED;
+  if (order == 1 && (!block_scores || !aligned16(block_scores))) return SVA_ERR_INVALID_ARG;
   return launch_attn_ts(m, p, q, k, v, nullptr, nullptr, row_ptr, col_idx, o, lse, device_status, workspace,
-                        workspace_bytes, (cudaStream_t)stream, order);
+                        workspace_bytes, (cudaStream_t)stream, order, block_scores);
 }
 
 int sva_block_sparse_attn_fwd_fp4(const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,

@@ -91,6 +91,8 @@ struct TsParams {
   int32_t* next_row;          // two device counters (both start at 0): the next row to hand out, CTAs done drawing
   // approximate remainder (REM kernels): every row's list is followed by np tiles whose "keys" are the
   // block means of K (and whose "values" the block means of V), 128 blocks per tile
+  int n1;                     // first-order tiles after them: 0 (order 0), 1, or 2 with 64-token blocks (one per query block)
+  const float* mu;            // first-order term: the reference mu_I of every query block's weights, [R of the CSR]
   int np;                     // pooled tiles per head = ceil(Nb / 128); 0 = no remainder
   float log2_block;           // log2(tokens per block): a block mean stands for that many keys
   float tail_bias;            // (log2(keys of the last block) - log2_block) / scale_log2: added to the last block's pooled logit
@@ -142,27 +144,33 @@ template <bool B64, bool REM = false>
 __device__ __forceinline__ bool row_list(const TsParams& prm, int r, int nnz_bound, int& n, int& beg) {
   if (B64) {
     if (prm.row_ptr == nullptr) { n = (prm.Nb + 1) >> 1; beg = 0; return true; }     // dense: every pair of key blocks
-    n = __ldg(prm.tile_cnt + r) + (REM ? prm.np : 0); beg = __ldg(prm.tile_beg + r);
+    n = __ldg(prm.tile_cnt + r) + (REM ? prm.np + prm.n1 : 0); beg = __ldg(prm.tile_beg + r);
     return true;
   }
   if (prm.row_ptr == nullptr) { n = prm.Nb; beg = 0; return true; }
   beg = __ldg(prm.row_ptr + r);
   const int end = __ldg(prm.row_ptr + r + 1);
   n = end - beg;
-  if (beg < 0 || end < beg || n > prm.Nb || end > nnz_bound) { n = REM ? prm.np : 0; beg = 0; return false; }
-  if (REM) n += prm.np;
+  if (beg < 0 || end < beg || n > prm.Nb || end > nnz_bound) { n = REM ? prm.np + prm.n1 : 0; beg = 0; return false; }
+  if (REM) n += prm.np + prm.n1;
   return true;
 }
 // Pooled tiles (REM) are marked in their list entry: bit 31 (128-token blocks) resp. an upper half of
 // 0xffff (64-token blocks: block index 0x3fff cannot occur, Nb <= 16383); the low 16 bits are the chunk.
+// First-order tiles: bit 30 resp. an upper half of 0xfffe; the low bits say which query block of the tile row.
 template <bool B64>
 __device__ __forceinline__ bool entry_is_pooled(uint32_t e) {
   return B64 ? (e >> 16) == 0xffffu : (e >> 31) != 0u;
+}
+template <bool B64>
+__device__ __forceinline__ bool entry_is_first_order(uint32_t e) {
+  return B64 ? (e >> 16) == 0xfffeu : (e >> 30) == 1u;
 }
 // Entry j of a work list.  128-token blocks: the key block (an out-of-range entry is replaced by block 0;
 // the producer reports it).  64-token blocks: the tile descriptor.
 template <bool B64, bool REM = false>
 __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int j, int n_own = 0) {
+  if (REM && j >= n_own + prm.np) return (B64 ? 0xfffe0000u : 0x40000000u) | (uint32_t)(j - n_own - prm.np);
   if (REM && j >= n_own) return (B64 ? 0xffff0000u : 0x80000000u) | (uint32_t)(j - n_own);
   if (B64) {
     if (prm.row_ptr == nullptr) {        // dense: key blocks 2j and 2j+1 (if it exists), kept by both query blocks
@@ -193,7 +201,7 @@ template <bool B64, bool F8, bool REM, bool F4 = false, bool VMN = false>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_kp,
-               const __grid_constant__ CUtensorMap tm_vtp, const TsParams prm) {
+               const __grid_constant__ CUtensorMap tm_vtp, const __grid_constant__ CUtensorMap tm_at, const TsParams prm) {
   using namespace ts;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -249,7 +257,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 8 && lane == 0) { prefetch_tmap(&tm_k); if (REM) prefetch_tmap(&tm_kp); }
-  if (warp == 11 && lane == 0) { prefetch_tmap(&tm_vt); if (REM) prefetch_tmap(&tm_vtp); }
+  if (warp == 11 && lane == 0) { prefetch_tmap(&tm_vt); if (REM) { prefetch_tmap(&tm_vtp); prefetch_tmap(&tm_at); } }
   if (warp == 0 && lane == 0) prefetch_tmap(&tm_o);
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -311,7 +319,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
           }
           uint32_t e0 = 0u, e1 = 0u;
-          const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);        // entries of the row's own list
+          const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);        // entries of the row's own list
           if (r < prm.R) { e0 = list_block<B64, REM>(prm, beg, 0, n_own); if (n > 1) e1 = list_block<B64, REM>(prm, beg, 1, n_own); }
           rowq[8 * slot] = r;
           rowq[8 * slot + 1] = n;
@@ -346,7 +354,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               bulk_load(dst + 8192, prm.k_sf + ((long long)bh * prm.Nb + J) * 1024, 1024, bar_k_full + 8 * s);
             } else if (REM && j >= n_own) {
               // pooled tile: 128 block means of K (rows beyond Nb are zero in the pooled tensor)
-              const int c = j - n_own;
+              // (a first-order tile has no logits of its own: its S is computed from pooled tile 0 and ignored)
+              const int c = j - n_own < prm.np ? j - n_own : 0;
               tma_load_4d(dst, &tm_kp, bar_k_full + 8 * s, 0, c * BS, hh, bb);
               tma_load_4d(dst + TILE / 2, &tm_kp, bar_k_full + 8 * s, 64, c * BS, hh, bb);
             } else if (B64) {
@@ -384,7 +393,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           uint32_t e0, e1;
           if (!fetch_row(i, r, n, beg, e0, e1, true) || r >= prm.R) break;
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
-          const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);
+          const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);
           for (int j = 0; j < n; ++j) {
             if (!mbar_wait(bar_v_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
             const uint32_t e = list_block<B64, REM>(prm, beg, j, n_own);
@@ -406,8 +415,15 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             } else if (REM && j >= n_own) {
               // pooled tile: the block means of V, transposed ([128 d rows][128 blocks]; blocks beyond Nb zero)
               const int c = j - n_own;
-              tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
-              tma_load_4d(dst + TILE / 2, &tm_vtp, bar_v_full + 8 * s, 64, c * BS, hh, bb);
+              if (c < prm.np) {
+                tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
+                tma_load_4d(dst + TILE / 2, &tm_vtp, bar_v_full + 8 * s, 64, c * BS, hh, bb);
+              } else {
+                // first-order tile: A^T of the query block (64-token blocks: of the tile row's first / second one)
+                const int qb = B64 ? min(2 * (r % Nb) + (c - prm.np), prm.Nb - 1) : r % Nb;
+                tma_load_4d(dst, &tm_at, bar_v_full + 8 * s, 0, qb * BS, hh, bb);
+                tma_load_4d(dst + TILE / 2, &tm_at, bar_v_full + 8 * s, 64, qb * BS, hh, bb);
+              }
             } else if (B64) {
               // each 64-key panel of the tile is one key block's transposed V: [128 d rows][64 keys]
               tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)(e & 0x3fffu) * D, hh, bb);
@@ -615,7 +631,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         qs_row = __ldg(prm.q_scale + (long long)bh * prm.Nb + qb) * prm.scale_log2;
         if (w < n) load_ks(J);
       }
-      const int n_own = n - ((REM && prm.row_ptr) ? prm.np : 0);      // entries of the row's own list
+      const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);      // entries of the row's own list
       for (int j = w; j < n; j += 2) {
         const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
         const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
@@ -624,7 +640,10 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         int v0, v1;
         const bool pooled = REM && entry_is_pooled<B64>(J);          // a tile of block means (the remainder)
         const int pc = (int)(J & 0xffffu);                            // ... and which 128 blocks it holds
-        if (pooled) {
+        const bool fo = REM && entry_is_first_order<B64>(J);          // the first-order tile: P = scaled q, "V^T" = A^T
+        if (fo) {
+          v0 = B64 ? 64 : BS; v1 = B64 ? 64 : 0;
+        } else if (pooled) {
           const int vn = min(BS, prm.Nb - BS * pc);                   // blocks that exist in this tile
           v0 = B64 ? min(64, vn) : vn;
           v1 = B64 ? max(vn - 64, 0) : 0;
@@ -691,11 +710,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           tc_wait_st();
         }
         uint32_t sv[128];
-        tmem_ld32(s_tmem + 0, sv + 0);
-        tmem_ld32(s_tmem + 32, sv + 32);
-        tmem_ld32(s_tmem + 64, sv + 64);
-        tmem_ld32(s_tmem + 96, sv + 96);
-        tc_wait_ld();
+        if (!(REM && fo)) {                                           // (a first-order tile's S is a dummy: not read)
+          tmem_ld32(s_tmem + 0, sv + 0);
+          tmem_ld32(s_tmem + 32, sv + 32);
+          tmem_ld32(s_tmem + 64, sv + 64);
+          tmem_ld32(s_tmem + 96, sv + 96);
+          tc_wait_ld();
+        }
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 2);
@@ -724,7 +745,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         // (e4m3 with 64-token blocks: each half has its own scale; a half that is not kept stays -inf)
         // (a pooled logit carries + log2(keys per block): a block mean stands for that many keys)
-        const float mx = (B64 && F8) ? fmaxf(v0 > 0 ? mx0 * c : -INFINITY, v1 > 0 ? mx1 * c1 : -INFINITY)
+        const float mx = (REM && fo) ? -INFINITY
+                       : (B64 && F8) ? fmaxf(v0 > 0 ? mx0 * c : -INFINITY, v1 > 0 ? mx1 * c1 : -INFINITY)
                                      : fmaxf(mx0, mx1) * c + ((REM && pooled) ? prm.log2_block : 0.f);
         // reference exponent left by block j-1 (other group)
         float m_prev = -INFINITY;
@@ -768,7 +790,24 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm), nm2h1 = B64 ? pack2(nmh1, nmh1) : nm2;
         const uint64_t c2h1 = (B64 && F8) ? pack2(c1, c1) : c2;
         uint64_t sum2 = pack2(0.f, 0.f);
-        if (!(prm.debug & 1)) {
+        if (REM && fo) {
+          // P'[i][c] = scale * q_i[c] * exp(mu - m): the row's own query values, for the rows of the query block this
+          // tile belongs to (64-token blocks: the other half of the tile row gets zeros); nothing joins the row sum
+          const int qb = B64 ? min(2 * I + qh, prm.Nb - 1) : I;
+          const bool mine_rows = (qi < prm.N) && (!B64 || qh == (int)(J & 1u)) && m_new != -INFINITY;
+          const float f = mine_rows ? prm.scale_log2 * 0.6931471805599453f *
+                                          ex2(__ldg(prm.mu + (long long)bh * prm.Nb + qb) * 1.4426950408889634f - m_new)
+                                    : 0.f;
+          const uint4* src = reinterpret_cast<const uint4*>(prm.q + (long long)bb * prm.sq.b + (long long)hh * prm.sq.h +
+                                                            (long long)min(qi, prm.N - 1) * prm.sq.n);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const uint4 u = __ldg(src + e);
+            const uint32_t wd[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) sv[4 * e + t] = pack_bf16(bf16lo(wd[t]) * f, bf16hi(wd[t]) * f);
+          }
+        } else if (!(prm.debug & 1)) {
 #pragma unroll
           for (int e = 0; e < 128; e += 2) {
             float x0, x1;
@@ -1082,7 +1121,8 @@ static bool g_ts_attr[TS_MAX_DEVICES][16];
 
 template <bool B64, bool F8, bool REM = false, bool F4 = false, bool VMN = false>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                     const CUtensorMap& tkp, const CUtensorMap& tvp, const TsParams& prm, cudaStream_t st) {
+                     const CUtensorMap& tkp, const CUtensorMap& tvp, const CUtensorMap& tat, const TsParams& prm,
+                     cudaStream_t st) {
   auto kern = attn_ts_kernel<B64, F8, REM, F4, VMN>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
@@ -1100,7 +1140,7 @@ static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, con
     sms = g_ts_sms[dev];
   }
   const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
-  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, tkp, tvp, prm);
+  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, tkp, tvp, tat, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
@@ -1144,8 +1184,14 @@ bool attn_ts_serves(const Dims& m) {
 
 // The remainder variant: bf16 Q/K, d = 128, a CSR (the dense form drops nothing).
 bool attn_ts_remainder_serves(const Dims& m) { return attn_ts_serves(m) && m.d == ts::D && !m.fp8; }
-size_t attn_ts_remainder_workspace_bytes(const Dims& m) {
-  return attn_ts_remainder_serves(m) ? ts_layout(m).total_rem : 0;
+size_t remainder1_bytes(const Dims& m);
+int launch_remainder1(const Dims& m, const sva_problem_t* p, const void* k, const void* v, const float* scores,
+                      const int32_t* row_ptr, const int32_t* col_idx, void* buf, const __nv_bfloat16** at_out,
+                      const float** mu_out, int32_t* status, cudaStream_t st);
+// (order 1 adds the buffers of the first-order term behind those of order 0)
+size_t attn_ts_remainder_workspace_bytes(const Dims& m, int order) {
+  if (!attn_ts_remainder_serves(m)) return 0;
+  return ts_layout(m).total_rem + (order >= 1 ? remainder1_bytes(m) : 0);
 }
 
 // What the one-call entry points need: e4m3 Q/K read V where it lies, so only the row counters (and the tile
@@ -1189,16 +1235,18 @@ int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, vo
 
 // v == nullptr: the workspace has been prepared by launch_prepare_v_ts (once per attention call).
 // remainder_order < 0: exact attention over the kept blocks only.  0: plus the block-mean remainder of the
-// dropped blocks (needs v, a CSR and the larger workspace of attn_ts_remainder_workspace_bytes).
+// dropped blocks (needs v, a CSR and the larger workspace of attn_ts_remainder_workspace_bytes).  1: plus the
+// first-order term (needs the routing's score matrix as well).
 int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order) {
+                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order, const float* block_scores) {
   int rc = check_ts_workspace(m_in, ws, ws_bytes, v != nullptr);
   if (rc) return rc;
   const bool rem = remainder_order >= 0;
   if (rem) {
-    if (remainder_order != 0 || !attn_ts_remainder_serves(m_in) || !row_ptr || !v) return SVA_ERR_UNSUPPORTED;
-    if (ws_bytes < attn_ts_remainder_workspace_bytes(m_in)) return SVA_ERR_WORKSPACE;
+    if (remainder_order > 1 || !attn_ts_remainder_serves(m_in) || !row_ptr || !v) return SVA_ERR_UNSUPPORTED;
+    if (remainder_order == 1 && !block_scores) return SVA_ERR_INVALID_ARG;
+    if (ws_bytes < attn_ts_remainder_workspace_bytes(m_in, remainder_order)) return SVA_ERR_WORKSPACE;
   }
   // dense attention does not depend on the block size: 64-token blocks run as 128-token blocks
   Dims m = m_in;
@@ -1215,7 +1263,8 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
-  CUtensorMap tk, tv, to, tkp, tvp;
+  CUtensorMap tk, tv, to, tkp, tvp, tat;
+  const float* mu_dev = nullptr;
   if ((rc = make_map_ts(&to, o, m.d, m.N, m.H, m.B, (cuuint64_t)so.n * 2, (cuuint64_t)so.h * 2, (cuuint64_t)so.b * 2, BS)) != SVA_OK)
     return rc;
   const int eb = m.fp8 ? 1 : 2;
@@ -1227,7 +1276,16 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   if ((rc = make_map_ts(&tv, ws, m.block, vrows, m.H, m.B, (cuuint64_t)m.block * 2, vrows * m.block * 2,
                         vrows * m.block * 2 * m.H, BS)) != SVA_OK)
     return rc;
-  tkp = tk; tvp = tv;            // (placeholders when there is no remainder: the kernel never touches them)
+  tkp = tk; tvp = tv; tat = tv;  // (placeholders when there is no remainder: the kernel never touches them)
+  if (rem && remainder_order == 1) {
+    // first-order term: C_J, weights, A_I (remainder.cu) into the buffers behind those of order 0
+    const __nv_bfloat16* at = nullptr;
+    if ((rc = launch_remainder1(m, p, k, v, block_scores, row_ptr, col_idx, wsb + L.total_rem, &at, &mu_dev, status, st)) != SVA_OK)
+      return rc;
+    const cuuint64_t arow = (cuuint64_t)m.Nb * BS;               // per head: Nb matrices of 128 rows x 128 bf16
+    if ((rc = make_map_ts(&tat, at, BS, arow, m.H, m.B, (cuuint64_t)BS * 2, arow * BS * 2, arow * BS * 2 * m.H, BS)) != SVA_OK)
+      return rc;
+  }
   if (rem) {
     // block means of K ([Nbp rows][128], rows >= Nb zero) and of V (transposed tiles), then their maps
     __nv_bfloat16* kp = reinterpret_cast<__nv_bfloat16*>(wsb + L.kp_off);
@@ -1274,6 +1332,8 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   prm.scale_log2 = m.scale * 1.4426950408889634f;
   prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
   prm.np = rem ? L.np : 0;
+  prm.n1 = (rem && remainder_order == 1) ? (b64 ? 2 : 1) : 0;
+  prm.mu = mu_dev;
   prm.log2_block = log2f((float)m.block);
   {
     const int tail = m.N - (m.Nb - 1) * m.block;
@@ -1288,16 +1348,16 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
           reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
       if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     }
-    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-    if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
-                          : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+    if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
+                          : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
   }
-  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-  if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
-                        : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st);
-  return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, prm, st)
-             : launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, prm, st);
+  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+  if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
+                        : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+  return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
+             : launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
 }
 
 // 4-bit Q/K: packed codes [B*H][Nb*128][64], tiled scale factors, one fp32 scale per (b,h); V bf16 as always.
@@ -1336,10 +1396,10 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
   prm.tile_cnt = nullptr; prm.tile_beg = nullptr; prm.tile_desc = nullptr;
   prm.scale_log2 = m.scale * 1.4426950408889634f;
   prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
-  prm.np = 0; prm.log2_block = 7.f; prm.tail_bias = 0.f;
+  prm.np = 0; prm.n1 = 0; prm.mu = nullptr; prm.log2_block = 7.f; prm.tail_bias = 0.f;
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
-  return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, prm, st);
+  return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, tv, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }

@@ -90,7 +90,8 @@ int launch_attn_simt(const Dims& m, const sva_problem_t* p, const void* q, const
                      const int32_t* col_idx, void* o, float* lse, int32_t* status, cudaStream_t st);
 int launch_attn_ts(const Dims& m, const sva_problem_t* p, const void* q, const void* k, const void* v,
                    const float* q_scale, const float* k_scale, const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int32_t* status,
-                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order = -1);
+                   void* ws, size_t ws_bytes, cudaStream_t st, int remainder_order = -1,
+                   const float* block_scores = nullptr);
 int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, const void* k4, const void* q_sf,
                        const void* k_sf, const float* q_g, const float* k_g, const void* v, const int32_t* row_ptr,
                        const int32_t* col_idx, void* o, float* lse, int32_t* status, void* ws, size_t ws_bytes,
@@ -98,7 +99,7 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
 bool attn_ts_fp4_serves(const Dims& m);
 size_t attn_ts_workspace_bytes(const Dims& m);
 size_t attn_ts_one_call_workspace_bytes(const Dims& m);
-size_t attn_ts_remainder_workspace_bytes(const Dims& m);
+size_t attn_ts_remainder_workspace_bytes(const Dims& m, int order);
 bool attn_ts_remainder_serves(const Dims& m);
 bool attn_ts_serves(const Dims& m);    // d = 128 or 64, bf16 or e4m3 Q/K, 128- or 64-token blocks
 int launch_prepare_v_ts(const Dims& m, const sva_problem_t* p, const void* v, void* ws, size_t ws_bytes,

@@ -148,20 +148,34 @@ def test_full_size_prologue():
     assert torch.equal(rp, rp2) and torch.equal(ci[: int(rp[-1])], ci2)
 
 
-@pytest.mark.parametrize("name", ["large", "large_b64"])
-def test_full_size_remainder(name):
-    """Piecewise attention with the order-0 remainder at full size in the launch configuration
-    `bench.py --remainder` times: per head, block 0, the ragged last block and 3 random ones against the oracle."""
+@pytest.mark.parametrize("name,order", [("large", 0), ("large_b64", 0), ("large", 1), ("large_b64", 1)])
+def test_full_size_remainder(name, order):
+    """Piecewise attention with the remainder at full size in the launch configuration `bench.py --remainder
+    [--remainder-order 1]` times: per head, block 0, the ragged last block and 3 random ones against the oracle
+    (order 1: four heads -- the oracle's d x d block statistics are numpy)."""
     from test_gpu_remainder import check_vs_oracle, gpu_remainder
     w = WORKLOADS[name]
     (q, k, v), (qb, kb, vb) = U.host_inputs(w)
     qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
-    rp, ci, _ = U.gpu_select(w, qd, kd)
-    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci)
+    rp, ci, scores = U.gpu_select(w, qd, kd, want_scores=order == 1)
+    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci, order, scores=scores)
     assert st == 0
-    rows = U.sample_rows_per_head(w.B * w.H, w.Nb, 3, seed=w.cfg)
-    r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
-    print(f"{name} + remainder: oracle sample {len(rows)} of {w.R} query blocks: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
+    if order == 0:
+        rows = U.sample_rows_per_head(w.B * w.H, w.Nb, 3, seed=w.cfg)
+        r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
+    else:
+        from paper_2606_23743_b200.workloads import shrink
+        r = (0.0, 0.0, 0.0)
+        rows = []
+        for h in (0, 9, 17, w.H - 1):
+            w1 = shrink(w, H=1)
+            rp_h = (rp[h * w.Nb:(h + 1) * w.Nb + 1] - rp[h * w.Nb]).cpu()
+            ci_h = ci[int(rp[h * w.Nb]):int(rp[(h + 1) * w.Nb])].cpu()
+            rows_h = U.sample_rows_per_head(1, w.Nb, 3, seed=h)
+            rh = check_vs_oracle(w1, qb[:, h:h + 1], kb[:, h:h + 1], vb[:, h:h + 1], rp_h, ci_h, o[:, h:h + 1], lse[:, h:h + 1],
+                                 rows_h, 1)
+            r = tuple(max(a, b) for a, b in zip(r, rh)); rows += rows_h
+    print(f"{name} + remainder order {order}: oracle sample {len(rows)} of {w.R} query blocks: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
     assert torch.isfinite(o[:, :, :w.N].float()).all() and torch.isfinite(lse).all()
     if w.n_alloc > w.N:
         assert (o[:, :, w.N:] == 7.0).all()

@@ -1,4 +1,4 @@
-"""Piecewise attention with the approximate remainder (order 0) through the C ABI against the oracle's
+"""Piecewise attention with the approximate remainder (orders 0 and 1) through the C ABI against the oracle's
 remainder formula with bf16-rounded block statistics, the same CSR on both sides.  bf16 tolerances."""
 import numpy as np
 import pytest
@@ -12,14 +12,14 @@ from paper_2606_23743_b200.workloads import WORKLOADS, shrink
 pytestmark = pytest.mark.gpu
 
 
-def gpu_remainder(w, q, k, v, rp, ci, order=0, N=None):
+def gpu_remainder(w, q, k, v, rp, ci, order=0, N=None, scores=None):
     N = w.N if N is None else N
     o = torch.full(v.shape, 7.0, dtype=torch.bfloat16, device="cuda")
     lse = torch.full((q.shape[0], q.shape[1], N), 7.0, dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = B.make_problem(q, k, v, o, N, w.block)
-    ws = torch.full((B.attn_remainder_workspace_bytes(p),), 0xFF, dtype=torch.uint8, device="cuda")
-    B.block_sparse_attn_remainder_fwd(p, q, k, v, rp, ci, o, lse, status, order, ws)
+    ws = torch.full((B.attn_remainder_workspace_bytes(p, order),), 0xFF, dtype=torch.uint8, device="cuda")
+    B.block_sparse_attn_remainder_fwd(p, q, k, v, rp, ci, o, lse, status, order, ws, scores)
     torch.cuda.synchronize()
     return o, lse, int(status.item())
 
@@ -46,19 +46,50 @@ CASES = {
 }
 
 
+@pytest.mark.parametrize("order", [0, 1])
 @pytest.mark.parametrize("name", list(CASES))
-def test_remainder_matches_oracle(name):
+def test_remainder_matches_oracle(name, order):
     w = CASES[name]
     (q, k, v), (qb, kb, vb) = U.host_inputs(w)
     qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
-    rp, ci, _ = U.gpu_select(w, qd, kd)
-    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci)
+    rp, ci, scores = U.gpu_select(w, qd, kd, want_scores=order == 1)
+    o, lse, st = gpu_remainder(w, qd, kd, vd, rp, ci, order, scores=scores)
     assert st == 0
     rows = list(range(w.R)) if w.R <= 160 else U.sample_rows_per_head(w.B * w.H, w.Nb, 6, seed=1)
-    r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows)
-    print(f"{name}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
+    r = check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows, order)
+    print(f"{name} order {order}: max_abs {r[0]:.2e} rel_l2 {r[1]:.2e} lse {r[2]:.2e}")
     if w.n_alloc > w.N:
         assert (o[:, :, w.N:] == 7.0).all()
+
+
+@pytest.mark.parametrize("name", ["medium_h2", "b64_odd_nb", "two_pooled_tiles"])
+def test_first_order_term_where_it_matters(name):
+    """V correlated with K inside every block (v += 4 k), so that C_J = sum (k - kbar) v^T is large and the
+    first-order term moves the output by more than twice the tolerance: a missing term, a wrong sign, a transposed C_J or A_I, a wrong
+    weight or reference would all fail here (on the plain workloads the term is smaller than the bf16 noise)."""
+    from paper_2606_23743_b200.workloads import bf16_bits
+    w = CASES[name]
+    (q, k, v), (qb, kb, _) = U.host_inputs(w)
+    v = (v.float() + 4.0 * k.float()).to(torch.bfloat16)
+    vb = bf16_bits(v)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, scores = U.gpu_select(w, qd, kd, want_scores=True)
+    o1, lse1, st = gpu_remainder(w, qd, kd, vd, rp, ci, 1, scores=scores)
+    assert st == 0
+    rows = list(range(w.R)) if w.R <= 160 else U.sample_rows_per_head(w.B * w.H, w.Nb, 6, seed=1)
+    rpn, cin = rp.cpu().numpy(), ci.cpu().numpy()
+    ref0, _ = oracle.attn_remainder_rows(qb, kb, vb, w.N, w.block, w.scale, rpn, cin, rows, order=0, stats="bf16")
+    ref1, l1 = oracle.attn_remainder_rows(qb, kb, vb, w.N, w.block, w.scale, rpn, cin, rows, order=1, stats="bf16")
+    ok = ~np.isnan(ref1)
+    moved = np.linalg.norm((ref1 - ref0)[ok]) / np.linalg.norm(ref1[ok])
+    assert moved > 2 * U.BF16_REL_L2, moved                  # the term is worth more than two tolerances here (a flipped sign: four)
+    o0, _, _ = gpu_remainder(w, qd, kd, vd, rp, ci, 0)
+    d_gpu = U.attn_errors(o1, None, ref0, l1, rows, w.N, w.block, o1.shape[1])[1]        # rel-L2 of GPU order 1 to oracle order 0
+    assert d_gpu > 1.5 * U.BF16_REL_L2, d_gpu                # ... and the GPU's order 1 is not order 0
+    max_abs, rel, lse_err = U.attn_errors(o1, lse1, ref1, l1, rows, w.N, w.block, o1.shape[1])
+    print(f"{name}: first-order term moves the output by rel-L2 {moved:.3f}; GPU vs oracle rel_l2 {rel:.2e} max_abs {max_abs:.2e}")
+    assert rel <= U.BF16_REL_L2 and lse_err <= 2e-3
+    assert max_abs <= max(U.BF16_MAX_ABS, 2.0 ** -7 * float(np.nanmax(np.abs(ref1))))     # (outputs of magnitude > 2.5: one bf16 unit)
 
 
 def test_rows_that_drop_nothing_equal_the_exact_call_and_empty_rows_are_all_remainder():
@@ -100,10 +131,14 @@ def test_unsupported_forms_are_refused_on_the_host():
     rp, ci, _ = U.gpu_select(w2, qd, kd)
     p2 = B.make_problem(qd, kd, vd, torch.empty_like(vd), w2.N, w2.block)
     ws = torch.empty(B.attn_remainder_workspace_bytes(p2), dtype=torch.uint8, device="cuda")
-    with pytest.raises(B.SvaError) as e:                      # first-order term: not built on the device
+    with pytest.raises(B.SvaError) as e:                      # first-order term without the score matrix
         B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 1, ws)
-    assert e.value.status == 2
+    assert e.value.status == 1
     with pytest.raises(B.SvaError) as e:                      # the exact call's workspace is too small
         B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 0,
                                           ws[: B.attn_workspace_bytes(p2)])
+    assert e.value.status == 3
+    with pytest.raises(B.SvaError) as e:                      # order 1 needs more than order 0's workspace
+        sc = torch.zeros(w2.B, w2.H, w2.Nb, w2.Nb, dtype=torch.float32, device="cuda")
+        B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 1, ws, sc)
     assert e.value.status == 3
