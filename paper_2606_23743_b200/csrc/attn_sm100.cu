@@ -713,15 +713,26 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (!(REM && fo)) {                                           // (a first-order tile's S is a dummy: not read)
           tmem_ld32(s_tmem + 0, sv + 0);
           tmem_ld32(s_tmem + 32, sv + 32);
+          tc_wait_ld();
           tmem_ld32(s_tmem + 64, sv + 64);
           tmem_ld32(s_tmem + 96, sv + 96);
-          tc_wait_ld();
         }
+        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+        float mx0, mx1;
+        if (!B64) {
+          // (the first half's maximum while the second half is still on its way from tensor memory)
+#pragma unroll
+          for (int e = 0; e < 64; e += 8) {
+            mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
+            mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+            mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
+            mxd = max3(mxd, __uint_as_float(sv[e + 6]), __uint_as_float(sv[e + 7]));
+          }
+        }
+        if (!(REM && fo)) tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + 8 * w);                     // the S issuer may refill this buffer
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 2);
-        float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
-        float mx0, mx1;
         if (B64) {                                           // a, b: keys 0..63; c, d: keys 64..127
 #pragma unroll
           for (int e = 0; e < 64; e += 4) {
@@ -734,7 +745,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           mx1 = v1 > 0 ? fmaxf(mxc, mxd) : -INFINITY;
         } else {
 #pragma unroll
-          for (int e = 0; e < 128; e += 8) {
+          for (int e = 64; e < 128; e += 8) {
             mxa = max3(mxa, __uint_as_float(sv[e + 0]), __uint_as_float(sv[e + 1]));
             mxb = max3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
             mxc = max3(mxc, __uint_as_float(sv[e + 4]), __uint_as_float(sv[e + 5]));
