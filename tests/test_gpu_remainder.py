@@ -114,6 +114,25 @@ def test_rows_that_drop_nothing_equal_the_exact_call_and_empty_rows_are_all_rema
         assert torch.equal(o[sl], o_e[sl]) and torch.equal(lse[sl], lse_e[sl])
 
 
+@pytest.mark.parametrize("block", [128, 64])
+def test_bad_csr_entries_are_reported_not_trapped(block):
+    """An out-of-range col_idx entry and a corrupt row_ptr pair under the remainder (both orders): flagged in
+    device_status, nothing faults, rows that the damage does not touch still match the oracle."""
+    w = shrink(WORKLOADS["medium"], H=2, T=2, k=3, block=block)
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, scores = U.gpu_select(w, qd, kd, want_scores=True)
+    rp_h = rp.cpu()
+    ci_bad = ci.clone(); ci_bad[int(rp_h[5])] = 9999
+    rp_bad = rp_h.clone(); rp_bad[9] = int(rp_h[8]) - 3                      # not monotone
+    for order in (0, 1):
+        for rpx, cix, touched in ((rp, ci_bad, {4, 5}), (rp_bad.cuda(), ci, {8, 9})):
+            o, lse, st = gpu_remainder(w, qd, kd, vd, rpx, cix, order, scores=scores)
+            assert st & B.SVA_DEV_BAD_INDEX and not (st & B.SVA_DEV_TIMEOUT)
+            rows = [r for r in range(w.R) if r not in touched and (r ^ 1) not in touched][:10]
+            check_vs_oracle(w, qb, kb, vb, rp, ci, o, lse, rows, order)
+
+
 def test_unsupported_forms_are_refused_on_the_host():
     w = shrink(WORKLOADS["tiny"], H=2)                        # d = 64
     (q, k, v), _ = U.host_inputs(w)
