@@ -48,6 +48,7 @@
 // loops, TMEM is released and the kernel returns.  Parity waits never run a whole phase ahead of
 // their barrier (each wait on a barrier is preceded by a wait on its previous phase).
 #include <mutex>
+#include <type_traits>
 
 #include "tc_ptx.cuh"
 
@@ -632,15 +633,18 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (w < n) load_ks(J);
       }
       const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);      // entries of the row's own list
-      for (int j = w; j < n; j += 2) {
+      // One tile of the row (KIND 0: a kept key block, 1: a tile of block means, 2: the first-order tile).  The
+      // kinds are separate instantiations, so the hot one carries none of the remainder's code; false: a wait ran out.
+      auto tile = [&](auto kind_tag, const int j) -> bool {
+        constexpr int KIND = decltype(kind_tag)::value;
         const uint32_t mine = cnt[w] + (uint32_t)(j >> 1);            // my barriers' phase index for block j
         const uint32_t prev = cnt[w ^ 1] + (uint32_t)((j - 1) >> 1);  // other group's phase index for block j-1
         // valid keys of the tile's two 64-key halves (64-token blocks: a half whose key block this
         // thread's query block does not keep counts as 0; uniform over a warp)
         int v0, v1;
-        const bool pooled = REM && entry_is_pooled<B64>(J);          // a tile of block means (the remainder)
+        constexpr bool pooled = REM && KIND == 1;                     // a tile of block means (the remainder)
         const int pc = (int)(J & 0xffffu);                            // ... and which 128 blocks it holds
-        const bool fo = REM && entry_is_first_order<B64>(J);          // the first-order tile: P = scaled q, "V^T" = A^T
+        constexpr bool fo = REM && KIND == 2;                         // the first-order tile: P = scaled q, "V^T" = A^T
         if (fo) {
           v0 = B64 ? 64 : BS; v1 = B64 ? 64 : 0;
         } else if (pooled) {
@@ -661,7 +665,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (F8) load_ks(J);
         }
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 0);
-        if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) { ok = false; break; }
+        if (!mbar_wait(bar_s_full + 8 * w, mine & 1u, abort_flag, prm.status)) return false;
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 1);
         tc_fence_after();
         if (B64 ? (v0 + v1 < BS) : (v0 < BS)) {
@@ -762,7 +766,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // reference exponent left by block j-1 (other group)
         float m_prev = -INFINITY;
         if (j > 0) {
-          if (!mbar_wait(bar_ref + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          if (!mbar_wait(bar_ref + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) return false;
           m_prev = ref[(w ^ 1) * 128 + row];
         }
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 3);
@@ -774,7 +778,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         bool pv_waited = false;
         if (j > 0 && __any_sync(0xffffffffu, m_new != m_prev)) {
           // rescale this row of O once P V(j-1) has completed (O is then quiescent: P V(j) waits for us)
-          if (!mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+          if (!mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) return false;
           pv_waited = true;
           tc_fence_after();
           const float alpha = ex2(m_prev - m_new);
@@ -837,7 +841,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // the P columns are free once P V(j-1) has completed (block 0: the previous row's last P V
         // was waited for in that row's epilogue)
         if (j > 0 && !pv_waited &&
-            !mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) { ok = false; break; }
+            !mbar_wait(bar_pv_done + 8 * (w ^ 1), prev & 1u, abort_flag, prm.status)) return false;
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 5);
         tc_fence_after();
         tmem_st32(p_tmem, sv);
@@ -846,6 +850,12 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         tc_fence_before();
         mbar_arrive(bar_p_full + 8 * w);
         if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, j, 6);
+        return true;
+      };
+      for (int j = w; j < n && ok; j += 2) {
+        if (!REM || j < n_own) ok = tile(std::integral_constant<int, 0>{}, j);
+        else if (j < n_own + prm.np) ok = tile(std::integral_constant<int, 1>{}, j);
+        else ok = tile(std::integral_constant<int, 2>{}, j);
       }
       if (!ok) break;
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 7);
