@@ -232,7 +232,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
 #endif
   if (threadIdx.x == 0) {
-    mbar_init(bar_q_ready, 256);
+    mbar_init(bar_q_ready, (!F4 && !B64) ? 128 : 256);   // (128-token blocks, bf16 / e4m3 Q: one softmax group writes a row's Q)
     mbar_init(bar_o_free, 256);
     mbar_init(bar_xch, 256);
     for (int w = 0; w < 2; ++w) {
@@ -322,6 +322,19 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           uint32_t e0 = 0u, e1 = 0u;
           const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);        // entries of the row's own list
           if (r < prm.R) { e0 = list_block<B64, REM>(prm, beg, 0, n_own); if (n > 1) e1 = list_block<B64, REM>(prm, beg, 1, n_own); }
+          if (!F4 && !B64 && r < prm.R) {
+            // the row's Q will be read by a softmax group about a row from now: start it on its way into the L2
+            const int I = r % Nb, bh0 = r / Nb, rows = min(BS, prm.N - I * BS);
+            const uint32_t eb = F8 ? 1u : 2u, row_bytes = (uint32_t)prm.d * eb;
+            const uint8_t* qrow = reinterpret_cast<const uint8_t*>(prm.q) +
+                                  ((long long)(bh0 / prm.H) * prm.sq.b + (long long)(bh0 % prm.H) * prm.sq.h +
+                                   (long long)I * BS * prm.sq.n) * eb;
+            if (prm.sq.n * (long long)eb == (long long)row_bytes) {
+              bulk_prefetch_l2(qrow, (uint32_t)rows * row_bytes);
+            } else {
+              for (int t = 0; t < rows; ++t) bulk_prefetch_l2(qrow + (long long)t * prm.sq.n * eb, row_bytes);
+            }
+          }
           rowq[8 * slot] = r;
           rowq[8 * slot + 1] = n;
           rowq[8 * slot + 2] = beg;
@@ -593,6 +606,37 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_arrive(bar_q_ready);
     };
 
+    // 128-token blocks (bf16 / e4m3 Q): ONE group writes the whole Q of the next row -- the group that does not take
+    // the current row's last tile, as soon as that last S has been computed, about a tile before the row ends -- so
+    // that the S issuer starts on the next row while this one is still finishing.  (The K producer has asked for
+    // those bytes to be brought into the L2 when it drew the row.)
+    constexpr bool EARLYQ = !F4 && !B64;
+    constexpr int QWF = F8 ? 32 : 64;                                   // 32-bit words of a whole row of Q
+    const uint32_t q_tmem_full = tmem_base + lane_addr + COL_Q;
+    auto load_q_full = [&](int r, uint32_t* qv) {
+#pragma unroll
+      for (int e = 0; e < QWF; ++e) qv[e] = 0u;
+      const int bh = r / Nb, qi = (r % Nb) * BS + row;
+      if (qi >= prm.N) return;
+      const long long eoff = (long long)(bh / prm.H) * prm.sq.b + (long long)(bh % prm.H) * prm.sq.h +
+                             (long long)qi * prm.sq.n;                    // in elements
+      const uint4* src = F8 ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(prm.q) + eoff)
+                            : reinterpret_cast<const uint4*>(prm.q + eoff);
+#pragma unroll
+      for (int e = 0; e < QWF / 4; ++e) {
+        if (e * (F8 ? 16 : 8) >= prm.d) break;                            // (d = 64: the upper half of Q is zero)
+        const uint4 u = __ldg(src + e);
+        qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
+      }
+    };
+    auto store_q_full = [&](const uint32_t* qv) {
+      tmem_st32(q_tmem_full, qv);
+      if (!F8) tmem_st32(q_tmem_full + 32, qv + 32);
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_q_ready);
+    };
+
     // The row sequence comes from the queue the K producer fills.  The entry after the current one is
     // read in the epilogue (the producer has published it by then: it runs about two blocks ahead),
     // so the next row's Q and first list entries are at hand when the row changes.
@@ -600,7 +644,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     int r_c = prm.R, n_c = 0, beg_c = 0;
     uint32_t e0_c = 0u, e1_c = 0u;
     if (!fetch_row(0, r_c, n_c, beg_c, e0_c, e1_c, signs)) ok = false;
-    if (ok && r_c < prm.R) {
+    if (EARLYQ) {
+      if (ok && r_c < prm.R && w == 1) {
+        uint32_t qv[QWF];
+        load_q_full(r_c, qv);
+        store_q_full(qv);
+      }
+    } else if (ok && r_c < prm.R) {
       // first row: its Q goes in right away
       uint32_t qv[32];
       load_q(r_c, qv);
@@ -859,12 +909,26 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
       if (!ok) break;
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 7);
+      if (EARLYQ) {
+        if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
+        if (w != wl) {
+          // The row's last S tile (the other group's) has been computed, and with it every S of the row: Q is free.
+          // (Its barrier's previous phase completed before the S tile this group has just worked on, or in an earlier row.)
+          if (!mbar_wait(bar_s_full + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+          if (r_c < prm.R) {
+            uint32_t qe[QWF];
+            load_q_full(r_c, qe);
+            store_q_full(qe);
+          }
+          if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
+        }
+      }
       // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
       // normalise and store (each group half of d)
-      if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
+      if (!EARLYQ && !fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
       const int r_next = r_c;                                         // (the queue holds non-empty rows only)
       uint32_t qn[32];
-      load_q(r_next, qn);                                             // in flight during the waits below
+      if (!EARLYQ) load_q(r_next, qn);                                // in flight during the waits below
       if (!mbar_wait(bar_ref + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
       const float m_fin = ref[wl * 128 + row];
       if (m_mine != m_fin) { l *= ex2(m_mine - m_fin); m_mine = m_fin; }        // l = 0 for a group without blocks
@@ -874,8 +938,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_arrive(bar_xch);
       if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
       // both groups have seen all their S tiles: no MMA reads Q any more
-      if (r_next < prm.R) store_q(qn, r_next);
-      if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
+      if (!EARLYQ && r_next < prm.R) store_q(qn, r_next);
+      if (!EARLYQ && (threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
       if (!mbar_wait(bar_pv_done + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 9);
       tc_fence_after();
