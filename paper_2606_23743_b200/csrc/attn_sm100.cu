@@ -131,7 +131,7 @@ constexpr float LAZY_LOG2 = 32.0f;
 // control block (bytes from OFF_CTRL):
 //   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
 //   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
-//   216 tmem_base | 220 abort | 224 o_staged[2] | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
+//   216 tmem_base | 220 abort | 224 o_staged[2] | 240 q_staged | 248 q_copied | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
 //   3328 row queue: QD entries {row, count, start, first entry, second entry, -, -, -} | 3456 rq_full[QD] | 3488 rq_empty[QD]
 
 // Work list of row r (a 128-query tile): count and start; returns false for a corrupt row_ptr pair.
@@ -202,7 +202,8 @@ template <bool B64, bool F8, bool REM, bool F4 = false, bool VMN = false>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
                const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_kp,
-               const __grid_constant__ CUtensorMap tm_vtp, const __grid_constant__ CUtensorMap tm_at, const TsParams prm) {
+               const __grid_constant__ CUtensorMap tm_vtp, const __grid_constant__ CUtensorMap tm_at,
+               const __grid_constant__ CUtensorMap tm_q, const TsParams prm) {
   using namespace ts;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -212,7 +213,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
                  bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
                  bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
-                 bar_ost = cb + 224, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
+                 bar_ost = cb + 224, bar_qs = cb + 240, bar_qg = cb + 248, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
   volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
   volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
@@ -235,6 +236,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     mbar_init(bar_q_ready, (!F4 && !B64) ? 128 : 256);   // (128-token blocks, bf16 / e4m3 Q: one softmax group writes a row's Q)
     mbar_init(bar_o_free, 256);
     mbar_init(bar_xch, 256);
+    mbar_init(bar_qs, 1);
+    mbar_init(bar_qg, 128);
     for (int w = 0; w < 2; ++w) {
       mbar_init(bar_s_full + 8 * w, 1);
       mbar_init(bar_p_full + 8 * w, 128);
@@ -259,7 +262,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   if (warp == 8 && lane == 0) { prefetch_tmap(&tm_k); if (REM) prefetch_tmap(&tm_kp); }
   if (warp == 11 && lane == 0) { prefetch_tmap(&tm_vt); if (REM) { prefetch_tmap(&tm_vtp); prefetch_tmap(&tm_at); } }
-  if (warp == 0 && lane == 0) prefetch_tmap(&tm_o);
+  if (warp == 0 && lane == 0) { prefetch_tmap(&tm_o); if (!F4 && !B64) prefetch_tmap(&tm_q); }
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(cb + 216), "r"(512u) : "memory");
@@ -323,7 +326,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int n_own = n - ((REM && prm.row_ptr) ? prm.np + prm.n1 : 0);        // entries of the row's own list
           if (r < prm.R) { e0 = list_block<B64, REM>(prm, beg, 0, n_own); if (n > 1) e1 = list_block<B64, REM>(prm, beg, 1, n_own); }
           if (!F4 && !B64 && r < prm.R) {
-            // the row's Q will be read by a softmax group about a row from now: start it on its way into the L2
+            // the row's Q tile will be fetched about a row from now: start it on its way into the L2
             const int I = r % Nb, bh0 = r / Nb, rows = min(BS, prm.N - I * BS);
             const uint32_t eb = F8 ? 1u : 2u, row_bytes = (uint32_t)prm.d * eb;
             const uint8_t* qrow = reinterpret_cast<const uint8_t*>(prm.q) +
@@ -608,33 +611,41 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
     // 128-token blocks (bf16 / e4m3 Q): ONE group writes the whole Q of the next row -- the group that does not take
     // the current row's last tile, as soon as that last S has been computed, about a tile before the row ends -- so
-    // that the S issuer starts on the next row while this one is still finishing.  (The K producer has asked for
-    // those bytes to be brought into the L2 when it drew the row.)
+    // that the S issuer starts on the next row while this one is still finishing.  The Q tile comes through the
+    // group's own output staging panel (idle between two epilogues), one 64-column half of d at a time: a TMA load
+    // (a thread-per-row read of Q from global memory costs 32 cache lines per load instruction, and that
+    // load/store-unit time stood in the way of the other group's last P store), then each thread copies its row
+    // of the half from shared memory into tensor memory.  `use` counts these copies over the CTA's rows (the
+    // first row's is copy 0), which gives the two barriers' phases.
     constexpr bool EARLYQ = !F4 && !B64;
-    constexpr int QWF = F8 ? 32 : 64;                                   // 32-bit words of a whole row of Q
-    const uint32_t q_tmem_full = tmem_base + lane_addr + COL_Q;
-    auto load_q_full = [&](int r, uint32_t* qv) {
+    constexpr int QPASS = F8 ? 1 : 2;                                   // halves of d (e4m3: the 128 bytes of a row are one)
+    auto copy_q = [&](int r, uint32_t use) -> bool {
+      const int bh = r / Nb, I = r % Nb;
+      const uint32_t panel = sbase + OFF_O + w * (TILE / 2);
+      const uint8_t* prow = smem + OFF_O + w * (TILE / 2) + row * 128;    // 128-byte rows, 16-byte chunks swizzled by row % 8
 #pragma unroll
-      for (int e = 0; e < QWF; ++e) qv[e] = 0u;
-      const int bh = r / Nb, qi = (r % Nb) * BS + row;
-      if (qi >= prm.N) return;
-      const long long eoff = (long long)(bh / prm.H) * prm.sq.b + (long long)(bh % prm.H) * prm.sq.h +
-                             (long long)qi * prm.sq.n;                    // in elements
-      const uint4* src = F8 ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(prm.q) + eoff)
-                            : reinterpret_cast<const uint4*>(prm.q + eoff);
+      for (int ps = 0; ps < QPASS; ++ps) {
+        const uint32_t k = use * QPASS + ps;                              // loads so far
+        if ((threadIdx.x & 127) == 0) {
+          if (ps == 0) bulk_wait_read0();                                 // my previous output store has read the panel
+          else if (!mbar_wait(bar_qg, (k - 1u) & 1u, abort_flag, prm.status)) return false;   // the group has copied the first half
+          mbar_expect_tx(bar_qs, TILE / 2);
+          tma_load_4d(panel, &tm_q, bar_qs, 64 * ps, I * BS, bh % prm.H, bh / prm.H);
+        }
+        if (!mbar_wait(bar_qs, k & 1u, abort_flag, prm.status)) return false;
+        uint32_t qv[32];
 #pragma unroll
-      for (int e = 0; e < QWF / 4; ++e) {
-        if (e * (F8 ? 16 : 8) >= prm.d) break;                            // (d = 64: the upper half of Q is zero)
-        const uint4 u = __ldg(src + e);
-        qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
+        for (int e = 0; e < 8; ++e) {
+          const uint4 u = *reinterpret_cast<const uint4*>(prow + ((e ^ (row & 7)) << 4));
+          qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
+        }
+        mbar_arrive(bar_qg);
+        tmem_st32(tmem_base + lane_addr + COL_Q + 32 * ps, qv);
       }
-    };
-    auto store_q_full = [&](const uint32_t* qv) {
-      tmem_st32(q_tmem_full, qv);
-      if (!F8) tmem_st32(q_tmem_full + 32, qv + 32);
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_q_ready);
+      return true;
     };
 
     // The row sequence comes from the queue the K producer fills.  The entry after the current one is
@@ -645,11 +656,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     uint32_t e0_c = 0u, e1_c = 0u;
     if (!fetch_row(0, r_c, n_c, beg_c, e0_c, e1_c, signs)) ok = false;
     if (EARLYQ) {
-      if (ok && r_c < prm.R && w == 1) {
-        uint32_t qv[QWF];
-        load_q_full(r_c, qv);
-        store_q_full(qv);
-      }
+      if (ok && r_c < prm.R && w == 1) ok = copy_q(r_c, 0u);
     } else if (ok && r_c < prm.R) {
       // first row: its Q goes in right away
       uint32_t qv[32];
@@ -909,20 +916,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
       if (!ok) break;
       if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 7);
-      if (EARLYQ) {
-        if (!fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
-        if (w != wl) {
-          // The row's last S tile (the other group's) has been computed, and with it every S of the row: Q is free.
-          // (Its barrier's previous phase completed before the S tile this group has just worked on, or in an earlier row.)
-          if (!mbar_wait(bar_s_full + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
-          if (r_c < prm.R) {
-            uint32_t qe[QWF];
-            load_q_full(r_c, qe);
-            store_q_full(qe);
-          }
-          if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
-        }
-      }
+      if (EARLYQ && !fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
       // ---- epilogue: merge the two groups' row sums, hand the next row's Q to the S issuer,
       // normalise and store (each group half of d)
       if (!EARLYQ && !fetch_row(rows_done + 1u, r_c, n_c, beg_c, e0_c, e1_c, signs)) { ok = false; break; }   // the row after this one, or the end mark
@@ -936,6 +930,14 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       lxr[w * 128 + row] = l;
       if ((threadIdx.x & 127) == 0) bulk_wait_read0();                // the previous row's store has read the staging panel
       mbar_arrive(bar_xch);
+      if (EARLYQ && w != wl) {
+        // (after this group's row sums are out, so that the other group's epilogue does not wait for the copy)
+        // The row's last S tile (the other group's) has been computed, and with it every S of the row: Q is free.
+        // (Its barrier's previous phase completed before the S tile this group has just worked on, or in an earlier row.)
+        if (!mbar_wait(bar_s_full + 8 * wl, last & 1u, abort_flag, prm.status)) { ok = false; break; }
+        if (r_next < prm.R && !copy_q(r_next, rows_done + 1u)) { ok = false; break; }
+        if ((threadIdx.x & 127) == 0) SVA_STAMP(w, rows_done, 255, 8);
+      }
       if (!mbar_wait(bar_xch, rows_done & 1u, abort_flag, prm.status)) { ok = false; break; }
       // both groups have seen all their S tiles: no MMA reads Q any more
       if (!EARLYQ && r_next < prm.R) store_q(qn, r_next);
@@ -1206,8 +1208,8 @@ static bool g_ts_attr[TS_MAX_DEVICES][16];
 
 template <bool B64, bool F8, bool REM = false, bool F4 = false, bool VMN = false>
 static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                     const CUtensorMap& tkp, const CUtensorMap& tvp, const CUtensorMap& tat, const TsParams& prm,
-                     cudaStream_t st) {
+                     const CUtensorMap& tkp, const CUtensorMap& tvp, const CUtensorMap& tat, const CUtensorMap& tq,
+                     const TsParams& prm, cudaStream_t st) {
   auto kern = attn_ts_kernel<B64, F8, REM, F4, VMN>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TS_MAX_DEVICES) return SVA_ERR_CUDA;
@@ -1225,7 +1227,7 @@ static int launch_ts(int rows, const CUtensorMap& tk, const CUtensorMap& tv, con
     sms = g_ts_sms[dev];
   }
   const int grid = rows < sms ? rows : sms;        // persistent: one CTA per SM, rows drawn from a counter
-  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, tkp, tvp, tat, prm);
+  kern<<<grid, ts::THREADS, ts::SMEM_BYTES, st>>>(tk, tv, to, tkp, tvp, tat, tq, prm);
   return cudaGetLastError() == cudaSuccess ? SVA_OK : SVA_ERR_CUDA;
 }
 
@@ -1362,6 +1364,14 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
                         vrows * m.block * 2 * m.H, BS)) != SVA_OK)
     return rc;
   tkp = tk; tvp = tv; tat = tv;  // (placeholders when there is no remainder: the kernel never touches them)
+  // Q as 128-row tiles, like K (128-token blocks: a row's Q reaches the kernel by TMA; otherwise unused)
+  CUtensorMap tq = tk;
+  if (!b64) {
+    const Strides sq = make_strides(p->q_stride);
+    if ((rc = make_map_ts(&tq, q, m.d, m.N, m.H, m.B, (cuuint64_t)sq.n * eb, (cuuint64_t)sq.h * eb, (cuuint64_t)sq.b * eb,
+                          m.block, eb)) != SVA_OK)
+      return rc;
+  }
   if (rem && remainder_order == 1) {
     // first-order term: C_J, weights, A_I (remainder.cu) into the buffers behind those of order 0
     const __nv_bfloat16* at = nullptr;
@@ -1433,16 +1443,16 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
           reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
       if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     }
-    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
-    if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
-                          : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
-    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+    if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+                          : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   }
-  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
-  if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
-                        : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
-  return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st)
-             : launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, tat, prm, st);
+  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+  if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+                        : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+  return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+             : launch_ts<false, false>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
 }
 
 // 4-bit Q/K: packed codes [B*H][Nb*128][64], tiled scale factors, one fp32 scale per (b,h); V bf16 as always.
@@ -1484,7 +1494,7 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
   prm.np = 0; prm.n1 = 0; prm.mu = nullptr; prm.log2_block = 7.f; prm.tail_bias = 0.f;
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
-  return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, tv, prm, st);
+  return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, tv, tq, prm, st);
 }
 
 void ts_set_prof_buffer(void* p) { g_prof_ts = (long long*)p; }
