@@ -5,7 +5,9 @@
 // A operand from shared memory vs tensor memory, or another instruction descriptor.  Here both
 // S = Q K^T and O += P V have the same form -- A from TENSOR memory (Q resp. P, bf16 pairs), B
 // from shared memory, K-major, M = N = 128 -- so the pipe never drains:
-//   * Q is written into TMEM once per row by the softmax threads (straight from global memory);
+//   * Q is written into TMEM once per row by the softmax threads (128-token blocks: by the group that finishes
+//     the row first, about a tile before the row ends, from a tile that TMA has put into the group's idle output
+//     staging panel; otherwise by both groups in the epilogue, straight from global memory);
 //   * V is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed copy
 //     that a small kernel writes into the caller's workspace first.
 // The kernel is persistent: one CTA per SM takes rows (one row = one query block of one head, 128
