@@ -55,12 +55,12 @@
 #include "tc_ptx.cuh"
 
 // Timeline stamps for tuning builds only (-DSVA_TIMELINE; never in the shipped library): CTA 0 appends
-// {cycle << 20 | role << 16 | row << 12 | tile << 4 | event} to prof[512..] for its rows 2..4.
+// {cycle << 20 | role << 16 | row << 12 | tile << 4 | event} to prof[512..] for its rows 2..4 (350 per role).
 #ifdef SVA_TIMELINE
 #define SVA_STAMP(role, row, j, ev)                                                                       \
   do {                                                                                                    \
-    if (blockIdx.x == 0 && (row) >= 2 && (row) <= 4 && stamp_n < 800u) {                                  \
-      stamp_buf[(role) * 800 + stamp_n++] = ((unsigned long long)(unsigned)clock() << 20) |               \
+    if (blockIdx.x == 0 && (row) >= 2 && (row) <= 4 && stamp_n < 350u) {                                  \
+      stamp_buf[(role) * 350 + stamp_n++] = ((unsigned long long)(unsigned)clock() << 20) |               \
           ((unsigned long long)(role) << 16) | ((unsigned long long)((row) & 15) << 12) |                 \
           ((unsigned long long)((j) & 255) << 4) | (unsigned long long)(ev);                              \
     }                                                                                                     \
@@ -117,10 +117,11 @@ constexpr int OFF_O = OFF_V + VS * TILE;    // output staging: two [128 rows][12
 constexpr int OFF_CTRL = OFF_O + TILE;      // 6 tiles = 192 KB
 constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers, reference exponents, row sums (two rows), row queue
 constexpr int OFF_Q4 = OFF_CTRL + 4096;     // 4-bit variant: the row's Q codes (8 KB) and their scale factors (1 KB)
+constexpr int OFF_QS = OFF_CTRL + 4096;     // bf16, 128-token blocks: staging of the second half (d 64..127) of a row's Q tile (16 KB)
 #ifdef SVA_TIMELINE
-constexpr int SMEM_BYTES = OFF_CTRL + CTRL_BYTES + 1024 + 3200 * 8;
+constexpr int SMEM_BYTES = OFF_QS + 16384 + 1024 + 1400 * 8;
 #else
-constexpr int SMEM_BYTES = OFF_Q4 + 8192 + 1024 + 1024;      // + alignment slack
+constexpr int SMEM_BYTES = OFF_QS + 16384 + 1024;            // + alignment slack
 #endif
 constexpr uint32_t COL_SFA = 384, COL_SFB = 392;              // 4-bit variant: scale factors in the Q columns (8 + 2 x 8)
 constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
@@ -133,7 +134,7 @@ constexpr float LAZY_LOG2 = 32.0f;
 // control block (bytes from OFF_CTRL):
 //   0 q_ready | 8 o_free | 16 s_full[2] | 32 p_full[2] | 48 pv_done[2] | 64 ref_ready[2] | 80 xch
 //   96 s_free[2] | 112 k_full[3] | 136 k_empty[3] | 160 v_full[3] | 184 v_empty[3]
-//   216 tmem_base | 220 abort | 224 o_staged[2] | 240 q_staged | 248 q_copied | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
+//   216 tmem_base | 220 abort | 224 o_staged[2] | 240 q_staged | 256 ref[2][128] floats | 1280 lx[2 rows][2][128] floats
 //   3328 row queue: QD entries {row, count, start, first entry, second entry, -, -, -} | 3456 rq_full[QD] | 3488 rq_empty[QD]
 
 // Work list of row r (a 128-query tile): count and start; returns false for a corrupt row_ptr pair.
@@ -215,7 +216,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t bar_q_ready = cb + 0, bar_o_free = cb + 8, bar_s_full = cb + 16, bar_p_full = cb + 32,
                  bar_pv_done = cb + 48, bar_ref = cb + 64, bar_xch = cb + 80, bar_s_free = cb + 96,
                  bar_k_full = cb + 112, bar_k_empty = cb + 136, bar_v_full = cb + 160, bar_v_empty = cb + 184,
-                 bar_ost = cb + 224, bar_qs = cb + 240, bar_qg = cb + 248, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
+                 bar_ost = cb + 224, bar_qs = cb + 240, bar_rq_full = cb + 3456, bar_rq_empty = cb + 3488;
   volatile uint32_t* tmem_base_p = reinterpret_cast<volatile uint32_t*>(ctrl + 216);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 220);
   volatile float* ref = reinterpret_cast<volatile float*>(ctrl + 256);      // [2][128]
@@ -230,8 +231,8 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const long long t_cta0 = prm.prof ? clock64() : 0;
 #ifdef SVA_TIMELINE
   uint32_t stamp_n = 0;
-  unsigned long long* stamp_buf = reinterpret_cast<unsigned long long*>(smem + OFF_CTRL + CTRL_BYTES);   // 3200 entries
-  if (blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 3200; i_ += THREADS) stamp_buf[i_] = 0ull;
+  unsigned long long* stamp_buf = reinterpret_cast<unsigned long long*>(smem + OFF_QS + 16384);   // 1400 entries
+  if (blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 1400; i_ += THREADS) stamp_buf[i_] = 0ull;
   __syncthreads();
 #endif
   if (threadIdx.x == 0) {
@@ -239,7 +240,6 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     mbar_init(bar_o_free, 256);
     mbar_init(bar_xch, 256);
     mbar_init(bar_qs, 1);
-    mbar_init(bar_qg, 128);
     for (int w = 0; w < 2; ++w) {
       mbar_init(bar_s_full + 8 * w, 1);
       mbar_init(bar_p_full + 8 * w, 128);
@@ -613,35 +613,32 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
     // 128-token blocks (bf16 / e4m3 Q): ONE group writes the whole Q of the next row -- the group that does not take
     // the current row's last tile, as soon as that last S has been computed, about a tile before the row ends -- so
-    // that the S issuer starts on the next row while this one is still finishing.  The Q tile comes through the
-    // group's own output staging panel (idle between two epilogues), one 64-column half of d at a time: a TMA load
-    // (a thread-per-row read of Q from global memory costs 32 cache lines per load instruction, and that
-    // load/store-unit time stood in the way of the other group's last P store), then each thread copies its row
-    // of the half from shared memory into tensor memory.  `use` counts these copies over the CTA's rows (the
-    // first row's is copy 0), which gives the two barriers' phases.
+    // that the S issuer starts on the next row while this one is still finishing.  The Q tile comes by TMA (a
+    // thread-per-row read of Q from global memory costs 32 cache lines per load instruction, and that
+    // load/store-unit time stood in the way of the other group's last P store): the first 64 columns of d into
+    // the group's own output staging panel (idle between two epilogues), the other 64 into a 16 KB buffer behind
+    // the control block, both loads in flight together; each thread then copies its row from shared memory into
+    // tensor memory.  `use` counts these copies over the CTA's rows (the first row's is copy 0): the barrier's phase.
     constexpr bool EARLYQ = !F4 && !B64;
-    constexpr int QPASS = F8 ? 1 : 2;                                   // halves of d (e4m3: the 128 bytes of a row are one)
     auto copy_q = [&](int r, uint32_t use) -> bool {
       const int bh = r / Nb, I = r % Nb;
-      const uint32_t panel = sbase + OFF_O + w * (TILE / 2);
-      const uint8_t* prow = smem + OFF_O + w * (TILE / 2) + row * 128;    // 128-byte rows, 16-byte chunks swizzled by row % 8
+      if ((threadIdx.x & 127) == 0) {
+        bulk_wait_read0();                                                // my previous output store has read the panel
+        mbar_expect_tx(bar_qs, F8 ? TILE / 2 : TILE);
+        tma_load_4d(sbase + OFF_O + w * (TILE / 2), &tm_q, bar_qs, 0, I * BS, bh % prm.H, bh / prm.H);
+        if (!F8) tma_load_4d(sbase + OFF_QS, &tm_q, bar_qs, 64, I * BS, bh % prm.H, bh / prm.H);
+      }
+      if (!mbar_wait(bar_qs, use & 1u, abort_flag, prm.status)) return false;
 #pragma unroll
-      for (int ps = 0; ps < QPASS; ++ps) {
-        const uint32_t k = use * QPASS + ps;                              // loads so far
-        if ((threadIdx.x & 127) == 0) {
-          if (ps == 0) bulk_wait_read0();                                 // my previous output store has read the panel
-          else if (!mbar_wait(bar_qg, (k - 1u) & 1u, abort_flag, prm.status)) return false;   // the group has copied the first half
-          mbar_expect_tx(bar_qs, TILE / 2);
-          tma_load_4d(panel, &tm_q, bar_qs, 64 * ps, I * BS, bh % prm.H, bh / prm.H);
-        }
-        if (!mbar_wait(bar_qs, k & 1u, abort_flag, prm.status)) return false;
+      for (int ps = 0; ps < (F8 ? 1 : 2); ++ps) {
+        // 128-byte rows, 16-byte chunks swizzled by row % 8
+        const uint8_t* prow = smem + (ps == 0 ? OFF_O + w * (TILE / 2) : OFF_QS) + row * 128;
         uint32_t qv[32];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const uint4 u = *reinterpret_cast<const uint4*>(prow + ((e ^ (row & 7)) << 4));
           qv[4 * e] = u.x; qv[4 * e + 1] = u.y; qv[4 * e + 2] = u.z; qv[4 * e + 3] = u.w;
         }
-        mbar_arrive(bar_qg);
         tmem_st32(tmem_base + lane_addr + COL_Q + 32 * ps, qv);
       }
       tc_wait_st();
@@ -992,7 +989,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     atomicMax(reinterpret_cast<unsigned long long*>(prm.prof + 319), (unsigned long long)(clock64() - t_cta0));
 #ifdef SVA_TIMELINE
   __syncthreads();
-  if (prm.prof && blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 3200; i_ += THREADS) prm.prof[512 + i_] = (long long)stamp_buf[i_];
+  if (prm.prof && blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 1400; i_ += THREADS) prm.prof[512 + i_] = (long long)stamp_buf[i_];
 #endif
   if (*abort_flag) {
     // give copies and MMAs still in flight time to land before shared memory and TMEM go away
