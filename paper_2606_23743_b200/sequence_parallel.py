@@ -46,14 +46,16 @@ def _check(x: torch.Tensor, world: int, shard_sizes: Sequence[int]):
         raise ValueError(f"{len(shard_sizes)} shard sizes for a group of {world}")
 
 
-def _exchange(send, recv_counts, group):
+def _exchange(send, recv_counts, group, src=None):
     """One all-to-all of flat chunks: send[g] goes to rank g, the result's entry s came from rank s.
-    (The single-buffer form with split sizes: both the NCCL and the gloo backend have it.)"""
-    src = torch.cat(send)
+    (The single-buffer form with split sizes: both the NCCL and the gloo backend have it.)
+    `src`: the chunks as one flat buffer, when the caller's tensor already is that (no staging copy)."""
+    if src is None:
+        src = torch.cat(send)
     dst = src.new_empty(sum(recv_counts))
     dist.all_to_all_single(dst, src, output_split_sizes=list(recv_counts),
                            input_split_sizes=[t.numel() for t in send], group=group)
-    return list(torch.split(dst, list(recv_counts)))
+    return dst, list(torch.split(dst, list(recv_counts)))
 
 
 def seq_to_head_shard(x_local: torch.Tensor, shard_sizes: Sequence[int], group=None) -> torch.Tensor:
@@ -67,7 +69,9 @@ def seq_to_head_shard(x_local: torch.Tensor, shard_sizes: Sequence[int], group=N
         raise ValueError(f"rank {rank} holds {n} tokens, shard_sizes says {shard_sizes[rank]}")
     hg = H // world
     send = [x_local[:, g * hg:(g + 1) * hg].reshape(-1) for g in range(world)]
-    recv = _exchange(send, [Bq * hg * shard_sizes[s] * d for s in range(world)], group)
+    # (one batch entry, contiguous: the head groups lie one behind the other already)
+    flat = x_local.reshape(-1) if Bq == 1 and x_local.is_contiguous() else None
+    _, recv = _exchange(send, [Bq * hg * shard_sizes[s] * d for s in range(world)], group, flat)
     return torch.cat([r.view(Bq, hg, shard_sizes[s], d) for s, r in enumerate(recv)], dim=2)
 
 
@@ -79,7 +83,9 @@ def head_to_seq_shard(x_heads: torch.Tensor, shard_sizes: Sequence[int], group=N
     if N != sum(shard_sizes):
         raise ValueError(f"{N} tokens, shard sizes add up to {sum(shard_sizes)}")
     send = [x_heads[:, :, lo:hi].reshape(-1) for lo, hi in shard_bounds(shard_sizes)]
-    recv = _exchange(send, [Bq * hg * shard_sizes[rank] * d] * world, group)
+    dst, recv = _exchange(send, [Bq * hg * shard_sizes[rank] * d] * world, group)
+    if Bq == 1:                                  # the received head groups already lie in head order
+        return dst.view(1, hg * world, shard_sizes[rank], d)
     return torch.cat([r.view(Bq, hg, shard_sizes[rank], d) for r in recv], dim=1)
 
 
