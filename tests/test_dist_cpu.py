@@ -41,7 +41,7 @@ def test_single_process_is_identity():
 
 
 # ------------------------------------------------------------------ sequence-parallel exchange (world 2 and 3, gloo)
-def _sp_worker(rank, world, port, q, N, H):
+def _sp_worker(rank, world, port, q, N, H, B_=2):
     os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
                       MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     import torch
@@ -49,7 +49,7 @@ def _sp_worker(rank, world, port, q, N, H):
     from paper_2606_23743_b200 import sequence_parallel as SP
     D.init("gloo")
     g = torch.Generator().manual_seed(5)
-    B_, d = 2, 8
+    d = 8
     full = [torch.randn(B_, H, N, d, generator=g) for _ in range(3)]          # the same on every rank
     sizes = SP.even_shards(N, world)
     lo, hi = SP.shard_bounds(sizes)[rank]
@@ -82,11 +82,11 @@ def _sp_worker(rank, world, port, q, N, H):
     q.put((rank, ok_fwd, ok_back, tuple(o.shape), err, bad))
 
 
-def _run_sp(world, N, H):
+def _run_sp(world, N, H, B_=2):
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    ps = [ctx.Process(target=_sp_worker, args=(r, world, port, q, N, H)) for r in range(world)]
+    ps = [ctx.Process(target=_sp_worker, args=(r, world, port, q, N, H, B_)) for r in range(world)]
     for p in ps:
         p.start()
     out = sorted(q.get(timeout=180) for _ in ps)
@@ -107,6 +107,15 @@ def test_sequence_parallel_exchange_three_ranks_ragged():
     """N = 50 over 3 ranks: shards of 17, 17, 16 tokens; 6 heads -> 2 per rank."""
     out = _run_sp(3, 50, 6)
     assert [o[3][2] for o in out] == [17, 17, 16]
+    for rank, ok_fwd, ok_back, shape, err, bad in out:
+        assert ok_fwd and ok_back and bad == 2 and err < 1e-5
+
+
+def test_sequence_parallel_exchange_one_batch_entry_ragged():
+    """B = 1 takes the forms of the two exchanges that skip a staging copy (the head groups of a contiguous
+    one-entry tensor already lie one behind the other): same checks, 3 ranks, ragged shards."""
+    out = _run_sp(3, 50, 6, 1)
+    assert [o[3] for o in out] == [(1, 6, 17, 8), (1, 6, 17, 8), (1, 6, 16, 8)]
     for rank, ok_fwd, ok_back, shape, err, bad in out:
         assert ok_fwd and ok_back and bad == 2 and err < 1e-5
 
