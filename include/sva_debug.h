@@ -26,6 +26,9 @@ void sva_debug_set_prof_buffer(void* buf);
  *   bit 0: skip the exponentials (tuning aid: timing only, results are wrong);
  *   bit 4: test aid: the K producer withholds a row's tiles after the first, so that a bounded pipeline wait
  *          runs out and the kernel takes its give-up path (SVA_DEV_TIMEOUT) -- nothing faults or hangs.
+ *   bit 5: measurement aid: bf16 attention reads V where it lies (MN-major operand) instead of the transposed copy;
+ *   bit 7: test aid: the remainder call masks the kept blocks of a block-mean tile by looking them up in the CSR
+ *          (the form that serves more than 1024 key blocks) even where the kept-block bit masks would serve.
  */
 void sva_debug_set_mode(int bits);
 

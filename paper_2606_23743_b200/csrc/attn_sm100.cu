@@ -97,11 +97,13 @@ struct TsParams {
   int n1;                     // first-order tiles after them: 0 (order 0), 1, or 2 with 64-token blocks (one per query block)
   const float* mu;            // first-order term: the reference mu_I of every query block's weights, [R of the CSR]
   int np;                     // pooled tiles per head = ceil(Nb / 128); 0 = no remainder
+  int rem_mask;               // 1: the K producer leaves a bit mask of every row's kept blocks in shared memory (Nb <= 1024)
   float log2_block;           // log2(tokens per block): a block mean stands for that many keys
   float tail_bias;            // (log2(keys of the last block) - log2_block) / scale_log2: added to the last block's pooled logit
   long long* prof;            // tuning aid, normally null: entry 319 receives the longest CTA's cycle count
   int debug;                  // bit0: skip the exponentials (tuning aid, wrong results);
                               // bit4: starve the pipeline so that a wait runs out (test aid)
+                              // (bit 7 acts in the launcher: the remainder looks kept blocks up in the CSR, without the mask)
 };
 
 namespace ts {
@@ -119,9 +121,11 @@ constexpr int CTRL_BYTES = 256 + 2 * 128 * 4 + 4 * 128 * 4 + 256;   // barriers,
 constexpr int OFF_Q4 = OFF_CTRL + 4096;     // 4-bit variant: the row's Q codes (8 KB) and their scale factors (1 KB)
 constexpr int OFF_QS = OFF_CTRL + 4096;     // bf16, 128-token blocks: staging of the second half (d 64..127) of a row's Q tile (16 KB)
 #ifdef SVA_TIMELINE
-constexpr int SMEM_BYTES = OFF_QS + 16384 + 1024 + 1400 * 8;
+constexpr int OFF_KMASK = OFF_QS + 16384;   // remainder: kept-block bit masks, [8 rows in flight][32 words]
+constexpr int SMEM_BYTES = OFF_KMASK + 1024 + 1024 + 1400 * 8;
 #else
-constexpr int SMEM_BYTES = OFF_QS + 16384 + 1024;            // + alignment slack
+constexpr int OFF_KMASK = OFF_QS + 16384;   // remainder: kept-block bit masks, [8 rows in flight][32 words]
+constexpr int SMEM_BYTES = OFF_KMASK + 1024 + 1024;          // + alignment slack
 #endif
 constexpr uint32_t COL_SFA = 384, COL_SFB = 392;              // 4-bit variant: scale factors in the Q columns (8 + 2 x 8)
 constexpr uint32_t COL_O = 256, COL_Q = 384, COL_P = 448;
@@ -226,12 +230,13 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int Nb = prm.Nt;             // row index arithmetic: rows per head
   constexpr int KB = B64 ? 64 : BS;  // tokens per key block
+  constexpr bool RMASK = REM && !B64; // remainder, 128-token blocks: kept-block bit masks (64-token blocks: the CSR look-up measured faster)
 
   // ---------------------------------------------------------------- set-up
   const long long t_cta0 = prm.prof ? clock64() : 0;
 #ifdef SVA_TIMELINE
   uint32_t stamp_n = 0;
-  unsigned long long* stamp_buf = reinterpret_cast<unsigned long long*>(smem + OFF_QS + 16384);   // 1400 entries
+  unsigned long long* stamp_buf = reinterpret_cast<unsigned long long*>(smem + OFF_KMASK + 1024);   // 1400 entries
   if (blockIdx.x == 0) for (int i_ = threadIdx.x; i_ < 1400; i_ += THREADS) stamp_buf[i_] = 0ull;
   __syncthreads();
 #endif
@@ -357,6 +362,15 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
           // ---- K tiles of the row
           const int bh = r / Nb, hh = bh % prm.H, bb = bh / prm.H;
+          // Remainder (128-token blocks): while walking the row's list this lane leaves a bit mask of the kept blocks
+          // for the softmax warps, which mask those columns of the block-mean tiles.  Eight masks in
+          // rotation: this lane is at most four tiles (two K slots, two S buffers) -- so at most four rows -- ahead.
+          // The masks are complete before the first block-mean tile's load is issued, which orders them before the
+          // softmax warps' read (expect_tx arrive -> k_full -> S MMA -> s_full).
+          volatile uint32_t* kmask = reinterpret_cast<volatile uint32_t*>(smem + OFF_KMASK) + (i & 7u) * 32;
+          if (RMASK && prm.rem_mask) {
+            for (int t = 0; t < 32; ++t) kmask[t] = 0u;
+          }
           for (int j = 0; j < n; ++j) {
             if ((prm.debug & 16) && j >= 1) { ok = false; break; }   // test aid: starve the pipeline so that a wait runs out
             if (!mbar_wait(bar_k_empty + 8 * s, ph ^ 1u, abort_flag, prm.status)) { ok = false; break; }
@@ -384,6 +398,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
                 const int J = (int)((dsc >> (16 * h)) & 0x3fffu);
+
                 tma_load_4d(dst + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 0, J * KB, hh, bb);
                 if (!F8) tma_load_4d(dst + TILE / 2 + h * (TILE / 4), &tm_k, bar_k_full + 8 * s, 64, J * KB, hh, bb);
               }
@@ -392,6 +407,7 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (prm.row_ptr) {
                 J = __ldg(prm.col_idx + beg + j);
                 if (J < 0 || J >= prm.Nb) { J = 0; if (prm.status) atomicOr(prm.status, SVA_DEV_BAD_INDEX); }
+                if (RMASK && prm.rem_mask) kmask[J >> 5] |= 1u << (J & 31);
               }
               tma_load_4d(dst, &tm_k, bar_k_full + 8 * s, 0, J * BS, hh, bb);      // e4m3: the whole tile (128 x 128 bytes)
               if (!F8) tma_load_4d(dst + TILE / 2, &tm_k, bar_k_full + 8 * s, 64, J * BS, hh, bb);
@@ -747,8 +763,23 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           // The remainder stands for the DROPPED blocks only: the blocks this thread's query block keeps become
           // -inf (one warp-wide TMEM store each; the row's CSR entries are the same for a whole warp), and the
           // ragged last block's mean stands for fewer keys than the others.
+          if (RMASK && prm.rem_mask) {
+            // (the K producer left the kept blocks of this row as a bit mask: four words for this tile's 128 blocks)
+            const volatile uint32_t* mk = reinterpret_cast<const volatile uint32_t*>(smem + OFF_KMASK) +
+                                          (rows_done & 7u) * 32 + 4 * pc;
+#pragma unroll 1
+            for (int kw = 0; kw < 4; ++kw) {
+              uint32_t mword = mk[kw];
+              while (mword) {
+                const int bit = __ffs(mword) - 1;
+                mword &= mword - 1u;
+                tmem_st1(s_tmem + 32 * kw + bit, 0xff800000u);
+              }
+            }
+          }
           const int rq = B64 ? bh * prm.Nb + min(2 * I + qh, prm.Nb - 1) : r;      // my query block's CSR row
-          int cb = __ldg(prm.row_ptr + rq), ce = __ldg(prm.row_ptr + rq + 1);
+          int cb = 0, ce = 0;                                          // (more than 1024 key blocks: from the CSR itself)
+          if (!(RMASK && prm.rem_mask)) { cb = __ldg(prm.row_ptr + rq); ce = __ldg(prm.row_ptr + rq + 1); }
           if (cb < 0 || ce < cb || ce - cb > prm.Nb || ce > nnz_total) ce = cb;      // corrupt pair (reported elsewhere)
 #pragma unroll 1
           for (int t0 = cb; t0 < ce; t0 += 32) {                       // 32 entries at a time, one per lane
@@ -1426,6 +1457,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   prm.scale_log2 = m.scale * 1.4426950408889634f;
   prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
   prm.np = rem ? L.np : 0;
+  prm.rem_mask = (rem && !b64 && m.Nb <= 1024 && !(g_debug_ts & 128)) ? 1 : 0;
   prm.n1 = (rem && remainder_order == 1) ? (b64 ? 2 : 1) : 0;
   prm.mu = mu_dev;
   prm.log2_block = log2f((float)m.block);
@@ -1490,7 +1522,7 @@ int launch_attn_ts_fp4(const Dims& m, const sva_problem_t* p, const void* q4, co
   prm.tile_cnt = nullptr; prm.tile_beg = nullptr; prm.tile_desc = nullptr;
   prm.scale_log2 = m.scale * 1.4426950408889634f;
   prm.next_row = reinterpret_cast<int32_t*>(wsb + L.counter_off);
-  prm.np = 0; prm.n1 = 0; prm.mu = nullptr; prm.log2_block = 7.f; prm.tail_bias = 0.f;
+  prm.np = 0; prm.rem_mask = 0; prm.n1 = 0; prm.mu = nullptr; prm.log2_block = 7.f; prm.tail_bias = 0.f;
   prm.prof = g_prof_ts;
   prm.debug = g_debug_ts;
   return launch_ts<false, false, false, true, true>(L.R2, tk, tv, to, tq, tv, tv, tq, prm, st);

@@ -62,6 +62,29 @@ def test_remainder_matches_oracle(name, order):
         assert (o[:, :, w.N:] == 7.0).all()
 
 
+@pytest.mark.parametrize("name", ["two_pooled_tiles", "ragged_tail", "mass_ragged_rows"])
+def test_both_ways_of_masking_the_kept_blocks_agree(name):
+    """128-token blocks, at most 1024 key blocks: the K producer leaves the kept blocks of a row as a bit mask in shared
+    memory; beyond that the softmax warps look them up in the CSR.  The second form is forced here (debug bit 7) on
+    cases the first one serves: same bytes, and the oracle check of the forced form."""
+    w = CASES[name]
+    (q, k, v), (qb, kb, vb) = U.host_inputs(w)
+    qd, kd, vd = U.dev(q), U.dev(k), U.dev(v)
+    rp, ci, scores = U.gpu_select(w, qd, kd, want_scores=True)
+    for order in (0, 1):
+        o_mask, lse_mask, st = gpu_remainder(w, qd, kd, vd, rp, ci, order, scores=scores)
+        assert st == 0
+        B.debug_set_mode(128)
+        try:
+            o_csr, lse_csr, st = gpu_remainder(w, qd, kd, vd, rp, ci, order, scores=scores)
+        finally:
+            B.debug_set_mode(0)
+        assert st == 0
+        assert torch.equal(o_mask.view(torch.int16), o_csr.view(torch.int16)) and torch.equal(lse_mask, lse_csr)
+        rows = list(range(w.R)) if w.R <= 160 else U.sample_rows_per_head(w.B * w.H, w.Nb, 4, seed=2)
+        check_vs_oracle(w, qb, kb, vb, rp, ci, o_csr, lse_csr, rows, order)
+
+
 @pytest.mark.parametrize("name", ["medium_h2", "b64_odd_nb", "two_pooled_tiles"])
 def test_first_order_term_where_it_matters(name):
     """V correlated with K inside every block (v += 4 k), so that C_J = sum (k - kbar) v^T is large and the
