@@ -213,6 +213,9 @@ def main():
                     help="with --remainder: 0 = block-mean term only, 1 = plus the first-order term")
     ap.add_argument("--sustained-seconds", type=float, default=2.5,
                     help="length of the second, back-to-back leg whose clocks NVML can follow (0 = skip)")
+    ap.add_argument("--v-copy", action="store_true",
+                    help="bf16: the two-step form -- a tiled transposed copy of V made on a second stream beside routing, "
+                         "then the attention kernel on that copy (default: one call that reads V where it lies)")
     ap.add_argument("--prologue", action="store_true",
                     help="extended step: the fused QK-norm + RoPE prologue in front (it also writes the block means, "
                          "and the e4m3 codes of an FP8 workload, so routing skips its pooling pass and the quantiser)")
@@ -264,9 +267,10 @@ def main():
         qsf = torch.zeros(BH, w.Nb, 1024, dtype=torch.uint8, device=dev); ksf = torch.zeros_like(qsf)
         qg = torch.zeros(BH, dtype=torch.float32, device=dev); kg = torch.zeros_like(qg)
         ws4 = torch.zeros(max(8 * BH, 256), dtype=torch.uint8, device=dev)
-    # e4m3 and 4-bit Q/K: the kernel reads V where it lies, the one-call entry point needs only its row counters
+    # the one-call entry points read V where it lies and need only their row counters (and tile lists);
+    # the two-step form (--v-copy) and the remainder keep a transposed copy of V in the workspace
     aws_bytes = (B.attn_remainder_workspace_bytes(p, args.remainder_order) if args.remainder else 256 if args.fp4 else
-                 B.attn_one_call_workspace_bytes(p) if w.fp8 else B.attn_workspace_bytes(p))
+                 B.attn_workspace_bytes(p) if args.v_copy else B.attn_one_call_workspace_bytes(p))
     aws = torch.empty(max(aws_bytes, 256), dtype=torch.uint8, device=dev)
     # the first-order term of the remainder weighs the dropped blocks by the routing's scores
     scores_buf = (torch.empty(w.B, w.H, w.Nb, w.Nb, dtype=torch.float32, device=dev)
@@ -275,7 +279,7 @@ def main():
     # routing kernels (pooling, scores, selection; CSR assembly when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
     launches_per_step = (4 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
-    if w.fp8 or args.fp4:   # no V transpose: V is read where it lies
+    if not (args.v_copy and not w.fp8 and not args.fp4) and not args.remainder:   # no V transpose: V is read where it lies
         launches_per_step -= 1
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
@@ -301,7 +305,7 @@ def main():
 
     # the two-step form serves what the tensor-core kernel serves (every supported shape today)
     # bf16: V is prepared (tiled transposed copy) beside routing; the other forms have no such step
-    two_step = B.attn_workspace_bytes(p) > 0 and not args.remainder and not args.fp4 and not w.fp8
+    two_step = args.v_copy and B.attn_workspace_bytes(p) > 0 and not args.remainder and not args.fp4 and not w.fp8
 
     def route(qq, kk, vv):
         if args.prologue:
@@ -527,7 +531,7 @@ def main():
                      "frac": achieved / peak, "traffic": ATTN_TRAFFIC_BYTES.get(w.name),
                      "traffic_source": "constant from one ncu capture of attn_ts_kernel on this workload, not measured by this run",
                      "traffic_with_v_transpose": (ATTN_TRAFFIC_BYTES[w.name] + TRANSPOSE_TRAFFIC_BYTES[w.name])
-                     if w.name in ATTN_TRAFFIC_BYTES and w.name in TRANSPOSE_TRAFFIC_BYTES else None,
+                     if two_step and w.name in ATTN_TRAFFIC_BYTES and w.name in TRANSPOSE_TRAFFIC_BYTES else None,
                      "algorithmic_bytes": 8.0 * w.B * w.H * w.N * w.d,
                      "frac_with_prepare": (step_flops / (inline_ms * 1e-3) / 1e12 / peak) if inline_ms else None,
                      "attention_with_prepare_ms": inline_ms,
@@ -539,7 +543,8 @@ def main():
                      "sm_mhz_implied_sustained": kernel_cycles / (sustained["attention_ms"] * 1e3)
                      if kernel_cycles and sustained else None,
                      "kernel": "attn_ts_kernel" + (" (the V transpose runs beside routing on a second stream)" if two_step
-                                                  else " with the V transpose in front of it"),
+                                                  else " on a transposed copy of V made in the same call" if args.remainder
+                                                  else ", V read where it lies"),
                      "mixed_precision_ceiling": peak * 4.0 / 3.0 if w.fp8 else None,
                      "peak_source": f"{peak_kind} bf16 burst",
                      "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"])

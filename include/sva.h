@@ -197,15 +197,12 @@ int sva_block_select_noalloc(const sva_problem_t* p, const sva_select_t* s, cons
  * (16 for e4m3 Q/K).  One tensor-core kernel (bf16 x bf16 or e4m3 x e4m3 MMA for Q K^T, bf16 for P V,
  * fp32 accumulate) serves every supported shape: d = 128 or 64 (64 is computed as 128 with a zero upper
  * half), bf16 or e4m3 Q/K, 128- or 64-token blocks.
- * workspace: >= sva_attn_workspace_bytes(p) bytes, 256-byte aligned.  The tensor-core kernel
- * keeps a tiled, transposed copy of V (2*B*H*Nb*block*128 bytes), its row counter and, for 64-token
- * blocks, its tile lists there, all rewritten by every call (so two calls that may overlap on the
- * GPU need a workspace each);
- * 0 only for an unsupported problem.
- * sva_attn_one_call_workspace_bytes(p) is what sva_block_sparse_attn_fwd and sva_dense_attn_fwd themselves need (the
- * larger figure also serves the two-step form below): the same for bf16 Q/K; for e4m3 Q/K -- whose kernel reads V
- * where it lies, S and P V being different MMA kinds anyway -- only the row counters and, for 64-token blocks, the
- * tile lists (a few KB to a few MB).  sva_block_sparse_attn_fwd_fp4 needs 256 bytes (its row counters).
+ * workspace: >= sva_attn_one_call_workspace_bytes(p) bytes, 256-byte aligned: the kernel's row counters and, for
+ * 64-token blocks, its tile lists (256 bytes to a few MB), rewritten by every call (so two calls that may overlap
+ * on the GPU need a workspace each).  These calls read V where it lies.
+ * sva_attn_workspace_bytes(p) is what the two-step form below needs: the same plus a tiled, transposed copy of V
+ * (2*B*H*Nb*block*128 bytes) that sva_attn_prepare_v writes; it also serves the one-call form.
+ * Both are 0 only for an unsupported problem.  sva_block_sparse_attn_fwd_fp4 needs 256 bytes (its row counters).
  */
 size_t sva_attn_workspace_bytes(const sva_problem_t* p);
 size_t sva_attn_one_call_workspace_bytes(const sva_problem_t* p);
@@ -251,16 +248,18 @@ int sva_dense_attn_fwd(const sva_problem_t* p, const void* q, const void* k, con
                        int32_t* device_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * The tensor-core path in two steps, for callers that can prepare V early -- on another stream
- * while routing runs (routing never reads V), or because the producer of V can be made to write
- * the prepared layout itself.  sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
+ * The tensor-core path in two steps, on a transposed copy of V: the attention kernel then needs about 1 % fewer
+ * cycles than the one-call form (both MMAs of one instruction form), at the price of the copy (a pass over V, its
+ * workspace) -- worth it where the copy can be made off the critical path, e.g. because the producer of V can be
+ * made to write the prepared layout itself; under a power cap the one-call form measured faster.
+ * sva_attn_prepare_v writes the tiled transposed copy of V (per (b,h)
  * and key block one contiguous tile [d][block keys], keys >= N zero) and resets the row counter in
  * `workspace`; sva_block_sparse_attn_fwd_prepared then runs the attention kernel alone (row_ptr ==
  * NULL means dense).  A prepared workspace serves any number of attention calls on that V that do
  * not overlap on the GPU (after a call that reported SVA_DEV_TIMEOUT, prepare again); the caller
- * orders prepare and attention (same stream, or an event).  Together they do exactly what
- * sva_block_sparse_attn_fwd / sva_dense_attn_fwd do in one call (q_scale, k_scale: as there, NULL for
- * bf16 Q/K).  SVA_ERR_UNSUPPORTED for the dense form of bf16 Q/K with 64-token blocks (it runs as
+ * orders prepare and attention (same stream, or an event).  Together they compute what
+ * sva_block_sparse_attn_fwd / sva_dense_attn_fwd compute in one call (q_scale, k_scale: as there, NULL for
+ * bf16 Q/K; the bytes agree, the P V products being the same sums).  SVA_ERR_UNSUPPORTED for the dense form of bf16 Q/K with 64-token blocks (it runs as
  * 128-token blocks, which a workspace prepared for 64-token blocks does not fit): use the one-call
  * entry point there.
  */

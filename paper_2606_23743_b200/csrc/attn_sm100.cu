@@ -1311,11 +1311,20 @@ size_t attn_ts_remainder_workspace_bytes(const Dims& m, int order) {
   return ts_layout(m).total_rem + (order >= 1 ? remainder1_bytes(m) : 0);
 }
 
-// What the one-call entry points need: e4m3 Q/K read V where it lies, so only the row counters (and the tile
-// lists of 64-token blocks) remain; bf16 Q/K as attn_ts_workspace_bytes.
+// What the one-call entry points need: they read V where it lies, so only the row counters (and the tile lists of
+// 64-token blocks) remain.  (The transposed copy in the one-call form is a measurement aid: debug bit 5, which then
+// needs the workspace of the two-step form.)
 size_t attn_ts_one_call_workspace_bytes(const Dims& m) {
   if (!attn_ts_serves(m)) return 0;
-  return m.fp8 ? ts_layout(m, true).total : attn_ts_workspace_bytes(m);
+  if (g_debug_ts & 32) return attn_ts_workspace_bytes(m);
+  size_t bytes = ts_layout(m, true).total;
+  if (m.block == 64 && !m.fp8) {            // the dense entry point runs 64-token blocks as 128-token blocks
+    Dims d = m;
+    d.block = BS; d.Nb = (m.N + BS - 1) / BS; d.R = m.B * m.H * d.Nb;
+    const size_t b2 = ts_layout(d, true).total;
+    if (b2 > bytes) bytes = b2;
+  }
+  return bytes;
 }
 
 size_t attn_ts_workspace_bytes(const Dims& m) {
@@ -1373,10 +1382,11 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     m.R = m.B * m.H * m.Nb;
   }
   const bool b64 = m.block == 64;
-  // e4m3 Q/K with V at hand: V is read where it lies (S and P V differ in kind anyway), no transposed copy.
-  // (bf16: only on request, bit 5 of the debug mode, to measure what the copy buys.)
-  const bool vmn = v != nullptr && remainder_order < 0 && (m.fp8 || ((g_debug_ts & 32) && !b64));
-  const TsLayout L = ts_layout(m, vmn && m.fp8);
+  // With V at hand it is read where it lies (an MN-major B operand): no transposed copy, no workspace for it, and
+  // under the power cap the step is faster without the copy's HBM traffic although the kernel needs 1 % more cycles.
+  // (The two-step form keeps the copy, and so does the remainder; bit 5 of the debug mode forces it here, to measure.)
+  const bool vmn = v != nullptr && remainder_order < 0 && !(g_debug_ts & 32);
+  const TsLayout L = ts_layout(m, vmn);
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
   const Strides so = make_strides(p->o_stride);
@@ -1477,7 +1487,8 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
     if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
                           : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
-    return launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+    return vmn ? launch_ts<true, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+               : launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   }
   if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
