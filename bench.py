@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, constants copied from one ncu capture each
 # (`ncu --set full --clock-control none -k regex:<kernel> -c 1` of this script on the "large" workload);
 # they are not measured by this run.  Other workloads: not captured (null).
-ATTN_TRAFFIC_BYTES = {"large": 794.5e6}           # attn_ts_kernel alone (605.1 MB read + 189.4 MB written)
+ATTN_TRAFFIC_BYTES = {"large": 793.9e6}           # attn_ts_kernel, V read where it lies (605.4 MB read + 188.5 MB written)
 TRANSPOSE_TRAFFIC_BYTES = {"large": 355.9e6}      # transpose_v_kernel (201.3 MB read + 154.6 MB written)
 SM_COUNT_FALLBACK = 148
 
