@@ -194,6 +194,11 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------ GPU arm
+def two_step_wanted(args, w):
+    """--v-copy: the two-step form of plain bf16 attention (the other forms have no such step)."""
+    return bool(args.v_copy) and not w.fp8 and not args.fp4 and not args.remainder
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -268,7 +273,7 @@ def main():
         qg = torch.zeros(BH, dtype=torch.float32, device=dev); kg = torch.zeros_like(qg)
         ws4 = torch.zeros(max(8 * BH, 256), dtype=torch.uint8, device=dev)
     # the one-call entry points read V where it lies and need only their row counters (and tile lists);
-    # the two-step form (--v-copy) and the remainder keep a transposed copy of V in the workspace
+    # the two-step form (--v-copy) keeps a transposed copy of V in the workspace
     aws_bytes = (B.attn_remainder_workspace_bytes(p, args.remainder_order) if args.remainder else 256 if args.fp4 else
                  B.attn_workspace_bytes(p) if args.v_copy else B.attn_one_call_workspace_bytes(p))
     aws = torch.empty(max(aws_bytes, 256), dtype=torch.uint8, device=dev)
@@ -279,7 +284,7 @@ def main():
     # routing kernels (pooling, scores, selection; CSR assembly when rows vary in length) + V transpose
     # + attention (+ the tile-list kernel of the 64-token-block path, + the quantiser of the FP8 variant)
     launches_per_step = (4 if variable_rows else 3) + 2 + (1 if w.block == 64 else 0) + (1 if w.fp8 else 0)
-    if not (args.v_copy and not w.fp8 and not args.fp4) and not args.remainder:   # no V transpose: V is read where it lies
+    if not two_step_wanted(args, w):   # no V transpose: V is read where it lies
         launches_per_step -= 1
     if args.prologue:       # + the prologue, - the pooling kernel, - the quantiser
         launches_per_step += 1 - 1 - (1 if w.fp8 else 0)
@@ -543,7 +548,6 @@ def main():
                      "sm_mhz_implied_sustained": kernel_cycles / (sustained["attention_ms"] * 1e3)
                      if kernel_cycles and sustained else None,
                      "kernel": "attn_ts_kernel" + (" (the V transpose runs beside routing on a second stream)" if two_step
-                                                  else " on a transposed copy of V made in the same call" if args.remainder
                                                   else ", V read where it lies"),
                      "mixed_precision_ceiling": peak * 4.0 / 3.0 if w.fp8 else None,
                      "peak_source": f"{peak_kind} bf16 burst",

@@ -228,7 +228,7 @@ int sva_block_sparse_attn_fwd(const sva_problem_t* p, const void* q, const void*
  * matrix per query block, A_I = sum_J exp(sbar_IJ) C_J.  On the device: C_J per key block (one tensor-core product
  * K_J^T V_J, centred), the weights from `block_scores` and the CSR, A_I as a [Nb x Nb] x [Nb x d*d] GEMM per head
  * (2*Nb^2*d^2 FLOP), all bf16 in the workspace, and one more tile per row in the attention kernel whose "P" are the
- * scaled query values and whose "V^T" is A_I^T (two such tiles per tile row with 64-token blocks).
+ * scaled query values and whose "V" is A_I (two such tiles per tile row with 64-token blocks).
  *   block_scores : order 1 only: the [B,H,Nb,Nb] fp32 score matrix sva_block_select wrote for this Q, K
  *                  (16-byte aligned); ignored (may be NULL) for order 0
  * Supported: bf16 Q/K, d = 128, 128- or 64-token blocks; otherwise SVA_ERR_UNSUPPORTED.  A query block that

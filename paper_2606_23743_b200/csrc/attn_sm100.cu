@@ -434,7 +434,21 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const uint32_t e = list_block<B64, REM>(prm, beg, j, n_own);
             const uint32_t dst = sbase + OFF_V + s * TILE;
             mbar_expect_tx(bar_v_full + 8 * s, TILE);
-            if (VMN) {
+            if (REM && j >= n_own) {
+              // pooled tile: the block means of V ([128 d rows][128 blocks], or [128 blocks][128 d] when V itself is
+              // read keys-major; blocks beyond Nb zero)
+              const int c = j - n_own;
+              if (c < prm.np) {
+                tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
+                tma_load_4d(dst + TILE / 2, &tm_vtp, bar_v_full + 8 * s, 64, c * BS, hh, bb);
+              } else {
+                // first-order tile: A^T (A when V is read keys-major) of the query block (64-token blocks: of the tile
+                // row's first / second one)
+                const int qb = B64 ? min(2 * (r % Nb) + (c - prm.np), prm.Nb - 1) : r % Nb;
+                tma_load_4d(dst, &tm_at, bar_v_full + 8 * s, 0, qb * BS, hh, bb);
+                tma_load_4d(dst + TILE / 2, &tm_at, bar_v_full + 8 * s, 64, qb * BS, hh, bb);
+              }
+            } else if (VMN) {
               // V itself: two d-panels of [128 keys][64 d] (64-token blocks: each panel's two halves from two key blocks)
               if (B64) {
 #pragma unroll
@@ -446,18 +460,6 @@ attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               } else {
                 tma_load_4d(dst, &tm_vt, bar_v_full + 8 * s, 0, (int)e * BS, hh, bb);
                 tma_load_4d(dst + TILE / 2, &tm_vt, bar_v_full + 8 * s, 64, (int)e * BS, hh, bb);
-              }
-            } else if (REM && j >= n_own) {
-              // pooled tile: the block means of V, transposed ([128 d rows][128 blocks]; blocks beyond Nb zero)
-              const int c = j - n_own;
-              if (c < prm.np) {
-                tma_load_4d(dst, &tm_vtp, bar_v_full + 8 * s, 0, c * BS, hh, bb);
-                tma_load_4d(dst + TILE / 2, &tm_vtp, bar_v_full + 8 * s, 64, c * BS, hh, bb);
-              } else {
-                // first-order tile: A^T of the query block (64-token blocks: of the tile row's first / second one)
-                const int qb = B64 ? min(2 * (r % Nb) + (c - prm.np), prm.Nb - 1) : r % Nb;
-                tma_load_4d(dst, &tm_at, bar_v_full + 8 * s, 0, qb * BS, hh, bb);
-                tma_load_4d(dst + TILE / 2, &tm_at, bar_v_full + 8 * s, 64, qb * BS, hh, bb);
               }
             } else if (B64) {
               // each 64-key panel of the tile is one key block's transposed V: [128 d rows][64 keys]
@@ -1152,7 +1154,7 @@ pair_lists_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict
 __global__ void __launch_bounds__(256)
 pool_kv_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, Strides sk, Strides sv,
                int H, int N, int block, int Nb, int Nbp, __nv_bfloat16* __restrict__ kp,
-               __nv_bfloat16* __restrict__ vtp) {
+               __nv_bfloat16* __restrict__ vtp, int v_rows) {
   __shared__ float part[16][ts::D + 1];
   const int J = blockIdx.x, bh = blockIdx.y, which = blockIdx.z;
   const int b = bh / H, h = bh % H;
@@ -1177,8 +1179,8 @@ pool_kv_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restr
 #pragma unroll
     for (int g = 0; g < 16; ++g) sum += part[g][threadIdx.x];
     const __nv_bfloat16 mean = __float2bfloat16_rn(sum / (float)cnt);
-    if (which == 0)
-      kp[((long long)bh * Nbp + J) * ts::D + threadIdx.x] = mean;
+    if (which == 0 || v_rows)                                 // (v_rows: the means of V laid out like those of K)
+      (which ? vtp : kp)[((long long)bh * Nbp + J) * ts::D + threadIdx.x] = mean;
     else
       vtp[(((long long)bh * (Nbp >> 7) + (J >> 7)) * ts::D + threadIdx.x) * BS + (J & 127)] = mean;
   }
@@ -1304,11 +1306,11 @@ bool attn_ts_remainder_serves(const Dims& m) { return attn_ts_serves(m) && m.d =
 size_t remainder1_bytes(const Dims& m);
 int launch_remainder1(const Dims& m, const sva_problem_t* p, const void* k, const void* v, const float* scores,
                       const int32_t* row_ptr, const int32_t* col_idx, void* buf, const __nv_bfloat16** at_out,
-                      const float** mu_out, int32_t* status, cudaStream_t st);
+                      const float** mu_out, int32_t* status, cudaStream_t st, bool natural);
 // (order 1 adds the buffers of the first-order term behind those of order 0)
 size_t attn_ts_remainder_workspace_bytes(const Dims& m, int order) {
   if (!attn_ts_remainder_serves(m)) return 0;
-  return ts_layout(m).total_rem + (order >= 1 ? remainder1_bytes(m) : 0);
+  return ts_layout(m, !(g_debug_ts & 32)).total_rem + (order >= 1 ? remainder1_bytes(m) : 0);
 }
 
 // What the one-call entry points need: they read V where it lies, so only the row counters (and the tile lists of
@@ -1385,7 +1387,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   // With V at hand it is read where it lies (an MN-major B operand): no transposed copy, no workspace for it, and
   // under the power cap the step is faster without the copy's HBM traffic although the kernel needs 1 % more cycles.
   // (The two-step form keeps the copy, and so does the remainder; bit 5 of the debug mode forces it here, to measure.)
-  const bool vmn = v != nullptr && remainder_order < 0 && !(g_debug_ts & 32);
+  const bool vmn = v != nullptr && !(g_debug_ts & 32);
   const TsLayout L = ts_layout(m, vmn);
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const Strides sk = make_strides(p->k_stride);
@@ -1415,7 +1417,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
   if (rem && remainder_order == 1) {
     // first-order term: C_J, weights, A_I (remainder.cu) into the buffers behind those of order 0
     const __nv_bfloat16* at = nullptr;
-    if ((rc = launch_remainder1(m, p, k, v, block_scores, row_ptr, col_idx, wsb + L.total_rem, &at, &mu_dev, status, st)) != SVA_OK)
+    if ((rc = launch_remainder1(m, p, k, v, block_scores, row_ptr, col_idx, wsb + L.total_rem, &at, &mu_dev, status, st, vmn)) != SVA_OK)
       return rc;
     const cuuint64_t arow = (cuuint64_t)m.Nb * BS;               // per head: Nb matrices of 128 rows x 128 bf16
     if ((rc = make_map_ts(&tat, at, BS, arow, m.H, m.B, (cuuint64_t)BS * 2, arow * BS * 2, arow * BS * 2 * m.H, BS)) != SVA_OK)
@@ -1427,12 +1429,14 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     __nv_bfloat16* vtp = reinterpret_cast<__nv_bfloat16*>(wsb + L.vtp_off);
     if (cudaMemsetAsync(kp, 0, 2 * L.pooled_bytes, st) != cudaSuccess) return SVA_ERR_CUDA;
     pool_kv_kernel<<<dim3(m.Nb, m.B * m.H, 2), 256, 0, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, sk,
-                                                            make_strides(p->v_stride), m.H, m.N, m.block, m.Nb, L.Nbp, kp, vtp);
+                                                            make_strides(p->v_stride), m.H, m.N, m.block, m.Nb, L.Nbp, kp, vtp,
+                                                            vmn ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     const cuuint64_t prow = (cuuint64_t)L.Nbp;
     if ((rc = make_map_ts(&tkp, kp, ts::D, prow, m.H, m.B, (cuuint64_t)ts::D * 2, prow * ts::D * 2,
                           prow * ts::D * 2 * m.H, BS)) != SVA_OK)
       return rc;
+    // (V read where it lies: the block means of V as rows, like those of K; else transposed, like a V^T tile)
     if ((rc = make_map_ts(&tvp, vtp, BS, prow, m.H, m.B, (cuuint64_t)BS * 2, prow * BS * 2, prow * BS * 2 * m.H, BS)) != SVA_OK)
       return rc;
   }
@@ -1441,7 +1445,7 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
     if ((rc = make_map_ts(&tv, v, m.d, m.N, m.H, m.B, (cuuint64_t)sv.n * 2, (cuuint64_t)sv.h * 2, (cuuint64_t)sv.b * 2,
                           m.block)) != SVA_OK)
       return rc;
-    tvp = tv;
+    if (!rem) tvp = tv;
     if (cudaMemsetAsync(wsb + L.counter_off, 0, 256, st) != cudaSuccess) return SVA_ERR_CUDA;
   } else if (v) {
     // (the transposed copy is laid out for the block size of this launch)
@@ -1484,13 +1488,15 @@ int launch_attn_ts(const Dims& m_in, const sva_problem_t* p, const void* q, cons
           reinterpret_cast<int32_t*>(wsb + L.beg_off), reinterpret_cast<uint32_t*>(wsb + L.desc_off), L.cap, status);
       if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
     }
-    if (rem) return launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+    if (rem) return vmn ? launch_ts<true, false, true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+                        : launch_ts<true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
     if (m.fp8) return vmn ? launch_ts<true, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
                           : launch_ts<true, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
     return vmn ? launch_ts<true, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
                : launch_ts<true, false>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   }
-  if (rem) return launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
+  if (rem) return vmn ? launch_ts<false, false, true, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
+                      : launch_ts<false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   if (m.fp8) return vmn ? launch_ts<false, true, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)
                         : launch_ts<false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st);
   return vmn ? launch_ts<false, false, false, false, true>(L.R2, tk, tv, to, tkp, tvp, tat, tq, prm, st)

@@ -2,7 +2,9 @@
 // blocks, as this build reads it): for a query block I
 //     T_i = scale * A_I^T q_i,   A_I = sum_{J dropped by I} exp(sbar_IJ) C_J,   C_J = sum_{j in J} (k_j - kbar_J) v_j^T,
 // one d x d matrix per query block.  Three kernels prepare A_I for the attention kernel, which then treats it as one
-// more tile of the row (its "P" are the scaled query values, its "V^T" is A_I^T):
+// more tile of the row (its "P" are the scaled query values, its "V" is A_I -- or, for the attention kernel that runs
+// on a transposed copy of V, its "V^T" is A_I^T; the kernels below are written for the transposed form and produce
+// the other one when the launcher hands the covariance kernel K and V in each other's place):
 //   cov_kernel        C_J^T = V_J^T K_J - n_J vbar_J kbar_J^T per key block: one 128 x 128 x block tcgen05 MMA, both
 //                     operands read where they lie (MN-major), the rank-one centring in the epilogue; bf16 out
 //   weights_kernel    W[I][J] = exp(sbar_IJ - mu_I) for the dropped J (0 for the kept ones), mu_I = their maximum
@@ -275,9 +277,11 @@ size_t remainder1_bytes(const Dims& m) {
 
 // Fills `buf` (remainder1_bytes) from K, V, the routing's score matrix and the CSR.  *at_out / *mu_out: where the
 // attention kernel finds A_I^T ([R][128 e][128 c] bf16) and mu_I.
+// natural: A_I itself ([R][128 c][128 e]) instead of its transpose -- for an attention kernel that takes its "V" tiles
+// keys-major (V read where it lies): the covariance kernel then simply gets K and V in each other's place.
 int launch_remainder1(const Dims& m, const sva_problem_t* p, const void* k, const void* v, const float* scores,
                       const int32_t* row_ptr, const int32_t* col_idx, void* buf, const __nv_bfloat16** at_out,
-                      const float** mu_out, int32_t* status, cudaStream_t st) {
+                      const float** mu_out, int32_t* status, cudaStream_t st, bool natural) {
   if (m.d != rem::D || (m.block != 128 && m.block != 64)) return SVA_ERR_UNSUPPORTED;
   const size_t mats = al256((size_t)m.R * rem::D * rem::D * 2);
   const int Nbw = (m.Nb + 63) / 64 * 64;
@@ -309,7 +313,8 @@ int launch_remainder1(const Dims& m, const sva_problem_t* p, const void* k, cons
   }
   const int smem_cov = 2 * rem::TILE + 1024, smem_agg = 128 * 128 + 2 * 64 * 128 + 1024;
   if (cudaFuncSetAttribute(cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cov) != cudaSuccess) return SVA_ERR_CUDA;
-  cov_kernel<<<dim3(m.Nb, m.B * m.H), 128, smem_cov, st>>>(tk, tv, m.H, m.N, m.block, m.Nb, ct, status);
+  if (natural) cov_kernel<<<dim3(m.Nb, m.B * m.H), 128, smem_cov, st>>>(tv, tk, m.H, m.N, m.block, m.Nb, ct, status);
+  else cov_kernel<<<dim3(m.Nb, m.B * m.H), 128, smem_cov, st>>>(tk, tv, m.H, m.N, m.block, m.Nb, ct, status);
   if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;
   weights_kernel<<<(m.R + 7) / 8, 256, 0, st>>>(scores, row_ptr, col_idx, m.R, m.Nb, Nbw, w, mu);
   if (cudaGetLastError() != cudaSuccess) return SVA_ERR_CUDA;

@@ -178,7 +178,7 @@ def test_unsupported_forms_are_refused_on_the_host():
     assert e.value.status == 1
     with pytest.raises(B.SvaError) as e:                      # the exact call's workspace is too small
         B.block_sparse_attn_remainder_fwd(p2, qd, kd, vd, rp, ci, torch.empty_like(vd), None, None, 0,
-                                          ws[: B.attn_workspace_bytes(p2)])
+                                          ws[: B.attn_one_call_workspace_bytes(p2)])
     assert e.value.status == 3
     with pytest.raises(B.SvaError) as e:                      # order 1 needs more than order 0's workspace
         sc = torch.zeros(w2.B, w2.H, w2.Nb, w2.Nb, dtype=torch.float32, device="cuda")
