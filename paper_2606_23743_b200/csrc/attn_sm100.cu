@@ -8,8 +8,11 @@
 //   * Q is written into TMEM once per row by the softmax threads (128-token blocks: by the group that finishes
 //     the row first, about a tile before the row ends, from a tile that TMA has put into the group's idle output
 //     staging panel; otherwise by both groups in the epilogue, straight from global memory);
-//   * V is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed copy
-//     that a small kernel writes into the caller's workspace first.
+//   * V: in the two-step form it is consumed transposed (V^T tiles: d rows, keys contiguous) from a tiled transposed
+//     copy that a small kernel writes into the caller's workspace first, so that P V has the form of S.  The one-call
+//     entry points read V where it lies instead (template switch VMN: an MN-major B operand, a second instruction
+//     descriptor): the pipe is idle often enough for the switch to cost 1 % of the cycles, and the step is faster
+//     without the copy's pass over the HBM.
 // The kernel is persistent: one CTA per SM takes rows (one row = one query block of one head, 128
 // query rows) from a device-wide counter until none is left.  All barriers keep running across rows
 // (every role derives the same phase counters from the same row sequence), so the producers run
