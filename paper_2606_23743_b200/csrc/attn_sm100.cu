@@ -206,8 +206,9 @@ __device__ __forceinline__ uint32_t list_block(const TsParams& prm, int beg, int
 // instead of being written to tensor memory; tm_kp is the map of the Q codes), with the scale factors copied
 // into the tensor-memory columns the bf16 Q would have used.  128-token blocks, d = 128 only.
 // VMN: V is read where it lies ([keys][d], d contiguous) and enters P V as an MN-major B operand -- another
-// instruction descriptor than S, which costs a tensor-pipe drain per switch, but no transposed copy of V and no
-// workspace for it.  Used where S and P V differ in kind anyway (e4m3 and 4-bit Q/K); tm_vt is then the map of V.
+// instruction descriptor than S, which costs a tensor-pipe drain per switch (hidden in the pipe's idle time: +1 % of
+// the cycles), but no transposed copy of V and no workspace for it.  Every one-call entry point uses it; tm_vt is then
+// the map of V (and, with REM, tm_vtp the block means of V as rows and tm_at the matrices A_I rather than their transposes).
 template <bool B64, bool F8, bool REM, bool F4 = false, bool VMN = false>
 __global__ void __launch_bounds__(384, 1)
 attn_ts_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_vt,
