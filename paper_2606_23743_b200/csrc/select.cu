@@ -447,7 +447,18 @@ static int launch_select_d(const Dims& m, const sva_problem_t* p, const sva_sele
   {
     auto kern = block_scores_kernel<D>;
     constexpr int smem = 2 * SC_TILE * (D + 4) * (int)sizeof(float);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SVA_ERR_CUDA;
+    // (the shared-memory attribute is set once per device and instantiation, not per call)
+    static std::mutex attr_mutex;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SVA_ERR_CUDA;
+    {
+      std::lock_guard<std::mutex> lock(attr_mutex);
+      if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SVA_ERR_CUDA;
+        attr_set[dev] = true;
+      }
+    }
     const int nt = (m.Nb + SC_TILE - 1) / SC_TILE;
     kern<<<dim3(nt, nt, m.B * m.H), 256, smem, st>>>(qbar, kbar, m.Nb, m.scale, scores);
   }
